@@ -1,0 +1,171 @@
+/*
+ * libdare — DARE per-layer activation-reuse attention step for bidirectional diffusion LLMs
+ * on NVIDIA B200 (sm_100a).  Plain C ABI: pointers and sizes only.
+ *
+ * One handle = one attention layer with its reuse state (previous head-0 query, K/V cache,
+ * attention-output cache, staleness counters).  One `dare_layer_step` = one denoising step of
+ * that layer:
+ *
+ *   Alg. 1 / Alg. 2, line 1   x_norm = Norm(x)                       (RMSNorm with gain)
+ *   line 2                    Q = W_Q x_norm, every token
+ *   line 3 (Sec. 3.1)         s_i = 1 - cos(Q_t[i, head 0], Q_{t-1}[i, head 0])
+ *   lines 4-5 (Eq. 2)         reuse set R = {i : s_i <= tau}; refresh set = complement,
+ *                             emitted as an ascending, compacted index list
+ *   DARE-KV (Alg. 1, Eq. 3)   K, V recomputed for the refresh set only and scattered into the cache
+ *   DARE-O  (Alg. 2, Eq. 4)   attention evaluated for the refresh set's query rows only; every other
+ *                             row keeps its cached attention output
+ *   last line                 y = W_O O
+ *   Sec. 4                    delta_i = 0 if refreshed else delta_i + 1
+ *
+ * Every step of that path runs in CUDA kernels of this library.  There is no CPU fallback.
+ *
+ * Memory and ownership
+ *   - All `const void*` / `void*` arguments are DEVICE pointers unless the name ends in `_host`.
+ *   - The library never allocates or frees device memory: the caller passes one workspace of
+ *     `dare_layer_workspace_bytes()` bytes at creation; it holds the caches and all scratch.
+ *   - Weights are borrowed for the life of the handle.  x and y belong to the caller.
+ *   - Device pointers must be 16-byte aligned (DARE_ERR_ALIGN otherwise); the workspace 256-byte.
+ *   - The handle itself is host memory owned by the library until `dare_layer_destroy`.
+ *
+ * Asynchrony
+ *   `dare_layer_step` validates on the host, enqueues kernels on the given stream and returns.  The number
+ *   of refreshed tokens never travels to the host during a step.  Results are valid once the caller has
+ *   synchronised the stream.  The observation calls (`status`, `last_selection`, `export_state`,
+ *   `import_state`, `step_host`) synchronise the stream themselves.
+ *
+ * Errors
+ *   Status codes only; nothing is thrown, nothing aborts.  Problems seen by a kernel (a bounded wait that
+ *   ran out, an index that failed its range check) are recorded in a device status word that
+ *   `dare_layer_status` returns.
+ *
+ * Threading: one host thread per handle at a time.
+ */
+#ifndef DARE_H_
+#define DARE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dare_layer dare_layer_t; /* opaque */
+
+typedef enum {
+  DARE_OK = 0,
+  DARE_ERR_INVALID_ARG = 1, /* NULL pointer, bad enum, NaN threshold, struct_size mismatch */
+  DARE_ERR_SHAPE = 2,       /* batch/seq/window outside the configured maxima, unsupported geometry */
+  DARE_ERR_STATE = 3,       /* call not legal in the handle's current state */
+  DARE_ERR_ALIGN = 4,       /* pointer alignment */
+  DARE_ERR_WORKSPACE = 5,   /* workspace too small */
+  DARE_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed */
+  DARE_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (reported by dare_layer_status) */
+  DARE_ERR_UNSUPPORTED = 8, /* configuration this build has no kernels for */
+  DARE_ERR_DEVICE_CHECK = 9 /* a device-side range check failed (reported by dare_layer_status) */
+} dare_status_t;
+
+/* mode bit 0: reuse cached K/V for tokens of the reuse set (DARE-KV, Alg. 1);
+ * mode bit 1: reuse cached attention outputs for them (DARE-O, Alg. 2).
+ * DARE_MODE_DENSE recomputes everything but still scores and updates every cache, so that a reuse
+ * step may follow (the "full dLLM" forward of Appendix E.2). */
+enum { DARE_MODE_DENSE = 0, DARE_MODE_KV = 1, DARE_MODE_O = 2, DARE_MODE_BOTH = 3 };
+
+typedef enum { DARE_F32 = 0, DARE_BF16 = 1 } dare_dtype_t;
+
+/* kernel_path: which kernel family the handle uses. */
+enum {
+  DARE_PATH_AUTO = 0,   /* tcgen05/TMEM tensor-core kernels when dtype = bf16 and head_dim = 128, else SIMT */
+  DARE_PATH_SIMT = 1,   /* plain fp32-accumulate CUDA-core kernels for every step (any supported geometry) */
+  DARE_PATH_TENSOR = 2  /* tensor-core kernels or DARE_ERR_UNSUPPORTED */
+};
+
+typedef struct {
+  uint32_t struct_size; /* sizeof(dare_layer_config_t), checked */
+  int32_t d_model;      /* = n_heads * head_dim; multiple of 8 */
+  int32_t n_heads;
+  int32_t head_dim;     /* even; 32..256 for the SIMT path, 128 for the tensor-core path */
+  int32_t max_batch;
+  int32_t max_seq;
+  float rope_theta;     /* rotary base (half-split pairing: element j rotates with j + head_dim/2) */
+  float rms_eps;
+  int32_t dtype;        /* dare_dtype_t: storage type of weights, x, y and caches; math accumulates in fp32 */
+  int32_t score_head;   /* head whose query drives the drift score; the paper uses head 0 (Sec. 3.2) */
+  int32_t kernel_path;  /* DARE_PATH_* */
+} dare_layer_config_t;
+
+typedef struct {
+  const void* w_q; /* device, row-major [d_model (out), d_model (in)], y = W x (Alg. 1 line 2) */
+  const void* w_k;
+  const void* w_v;
+  const void* w_o;
+  const float* rms_gain; /* device, float32 [d_model] */
+} dare_layer_weights_t;
+
+/* Bytes of device workspace a layer of this configuration needs; 0 if the configuration is invalid. */
+size_t dare_layer_workspace_bytes(const dare_layer_config_t* cfg);
+
+/* Creates a layer on the current CUDA device.  Fills the rotary table inside the workspace (synchronises the
+ * device once).  The first step after creation is dense whatever its mode (nothing is cached yet). */
+dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer_weights_t* weights,
+                                void* workspace, size_t workspace_bytes, dare_layer_t** out);
+
+/* One denoising step (Alg. 1 when mode = KV, Alg. 2 when mode = O, both reuse rules when mode = BOTH).
+ *   x, y        [batch, seq_act, d_model], dtype of the layer, covering positions
+ *               [pos_begin, pos_begin + seq_act) of every sequence.
+ *   threshold   tau of Eq. 2.  Negative refreshes every token, +inf reuses every token, NaN is rejected.
+ *   cuda_stream a cudaStream_t (NULL = legacy default stream).
+ * The first step after create/reset must have pos_begin = 0; it fixes batch and the cached extent
+ * kv_len = seq_act.  Later steps may cover any window inside [0, kv_len) and must keep the same batch
+ * (DARE_ERR_STATE otherwise).  Rows outside the window keep their cached K/V/O; attention always spans
+ * keys [0, kv_len). */
+dare_status_t dare_layer_step(dare_layer_t* layer, const void* x, int batch, int seq_act, int pos_begin,
+                              int mode, float threshold, void* y, void* cuda_stream);
+
+/* Same step with HOST buffers: copies x_host to the device, runs the step, copies y back and synchronises.
+ * x_host / y_host should be pinned for full copy bandwidth. */
+dare_status_t dare_layer_step_host(dare_layer_t* layer, const void* x_host, int batch, int seq_act, int pos_begin,
+                                   int mode, float threshold, void* y_host, void* cuda_stream);
+
+/* Forgets every cached activation: the next step is dense and must start at position 0.  Host-only. */
+dare_status_t dare_layer_reset(dare_layer_t* layer);
+
+dare_status_t dare_layer_destroy(dare_layer_t* layer);
+
+/* Synchronises the stream and returns the device-recorded status (DARE_OK, DARE_ERR_TIMEOUT,
+ * DARE_ERR_DEVICE_CHECK) or DARE_ERR_CUDA if the stream reports an error. */
+dare_status_t dare_layer_status(dare_layer_t* layer, void* cuda_stream);
+
+/* Selection of the last step, copied to host buffers (any of them may be NULL):
+ *   idx_host        int32[count]  ascending flat indices b*seq_act + i of the refresh set (room for batch*seq_act)
+ *   count_host      int32         |refresh set|
+ *   batch_off_host  int32[batch+1] start of each sequence's slice of idx
+ *   scores_host     float32[batch*seq_act] drift scores (+inf on a first step)
+ *   delta_host      int32[batch*seq_act] staleness counters of the window rows (Sec. 4) */
+dare_status_t dare_layer_last_selection(dare_layer_t* layer, int32_t* idx_host, int32_t* count_host,
+                                        int32_t* batch_off_host, float* scores_host, int32_t* delta_host,
+                                        void* cuda_stream);
+
+/* Raw views of the caches for tests and checkpointing: copies rows [0, kv_len) of each of the first `batch`
+ * sequences into host buffers shaped [batch, kv_len, d_model] (layer dtype); q_prev_host is float32
+ * [batch, kv_len, head_dim].  Any pointer may be NULL. */
+dare_status_t dare_layer_read_caches(dare_layer_t* layer, void* k_host, void* v_host, void* o_host,
+                                     float* q_prev_host, void* cuda_stream);
+
+/* Checkpoint / resume of the reuse state (previous query, K/V/O caches, staleness, step bookkeeping). */
+size_t dare_layer_state_bytes(const dare_layer_t* layer);
+dare_status_t dare_layer_export_state(dare_layer_t* layer, void* dst_host, size_t bytes, void* cuda_stream);
+dare_status_t dare_layer_import_state(dare_layer_t* layer, const void* src_host, size_t bytes, void* cuda_stream);
+
+/* Number of kernels the last dare_layer_step enqueued (for launch accounting in benchmarks). */
+int dare_layer_last_launch_count(const dare_layer_t* layer);
+
+const char* dare_status_string(dare_status_t s);
+
+/* Version of this ABI (bumped when a signature changes). */
+int dare_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DARE_H_ */

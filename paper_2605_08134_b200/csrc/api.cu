@@ -1,0 +1,418 @@
+// C ABI of libdare: handle life cycle, argument validation, workspace layout and the per-step kernel sequence.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "layer.h"
+
+using namespace dare;
+
+namespace {
+
+constexpr uint32_t kMagic = 0xDA2E1A7Eu;
+constexpr size_t kAlign = 256;
+
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+bool valid_config(const dare_layer_config_t* c) {
+  if (!c || c->struct_size != sizeof(dare_layer_config_t)) return false;
+  if (c->d_model <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->max_batch <= 0 || c->max_seq <= 0) return false;
+  if ((long)c->n_heads * c->head_dim != c->d_model) return false;
+  if (c->d_model % 16 != 0) return false;
+  if (c->dtype != DARE_F32 && c->dtype != DARE_BF16) return false;
+  if (c->score_head < 0 || c->score_head >= c->n_heads) return false;
+  if (c->kernel_path < DARE_PATH_AUTO || c->kernel_path > DARE_PATH_TENSOR) return false;
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return false;
+  if ((long)c->max_batch * c->max_seq > (1L << 24)) return false;
+  return true;
+}
+
+bool simt_geometry_ok(const dare_layer_config_t* c) {
+  return c->head_dim == 32 || c->head_dim == 64 || c->head_dim == 128 || c->head_dim == 256;
+}
+
+// Decides the kernel path; returns false when the configuration has no kernels.
+bool pick_path(const dare_layer_config_t* c, bool* use_tc) {
+  const bool tc = tc_supported(*c);
+  if (c->kernel_path == DARE_PATH_TENSOR) { *use_tc = true; return tc; }
+  if (c->kernel_path == DARE_PATH_SIMT) { *use_tc = false; return simt_geometry_ok(c); }
+  *use_tc = tc;
+  return tc || simt_geometry_ok(c);
+}
+
+// Carves the workspace.  With base == nullptr only the total size is computed.
+size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) {
+  const size_t Tm = (size_t)c->max_batch * c->max_seq;
+  const size_t e = c->dtype == DARE_BF16 ? 2 : 4;
+  const size_t d = c->d_model, hd = c->head_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> void* {
+    void* p = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return p;
+  };
+  Buffers tmp;
+  Buffers& B = b ? *b : tmp;
+  B.rope_cs = (float*)take((size_t)c->max_seq * (hd / 2) * 2 * sizeof(float));
+  B.xn = take(Tm * d * e);
+  B.q = take(Tm * d * e);
+  B.kc = take(Tm * d * e);
+  B.vc = take(Tm * d * e);
+  B.oc = take(Tm * d * e);
+  B.q_prev = (float*)take(Tm * hd * sizeof(float));
+  B.scores = (float*)take(Tm * sizeof(float));
+  B.idx = (int*)take(Tm * sizeof(int));
+  B.delta = (int*)take(Tm * sizeof(int));
+  B.batch_off = (int*)take(((size_t)c->max_batch + 1) * sizeof(int));
+  B.count = (int*)take(sizeof(int));
+  B.status = (int*)take(sizeof(int));
+  B.x_stage = take(Tm * d * e);
+  B.y_stage = take(Tm * d * e);
+  if (use_tc) {
+    B.xg = take((Tm + 128) * d * e);  // gathered rows of x_norm, padded to a whole tile
+    B.tmp = nullptr;
+  } else {
+    B.xg = nullptr;
+    B.tmp = (float*)take(Tm * 2 * d * sizeof(float));
+  }
+  return off;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+dare_status_t check_handle(const dare_layer_t* L) {
+  if (!L) return DARE_ERR_INVALID_ARG;
+  if (L->magic != kMagic) return DARE_ERR_STATE;
+  return DARE_OK;
+}
+
+#define CUDA_TRY(expr)                                  \
+  do {                                                  \
+    cudaError_t e_ = (expr);                            \
+    if (e_ != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; } \
+  } while (0)
+
+template <typename T>
+dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode, float tau, T* y, cudaStream_t st) {
+  const Buffers& B = L->buf;
+  const int T_ = g.tokens(), d = g.d;
+  const bool has_prev = L->has_prev;
+  const bool kv_sparse = has_prev && (mode & DARE_MODE_KV);
+  const bool o_sparse = has_prev && (mode & DARE_MODE_O);
+  int launches = 0;
+  // Alg. 1/2 line 1
+  launch_rmsnorm<T>(x, L->w.rms_gain, (T*)B.xn, T_, d, L->cfg.rms_eps, st); ++launches;
+  // line 2: dense Q projection
+  launch_gemm_simt<T>((const T*)B.xn, nullptr, nullptr, (const T*)L->w.w_q, B.tmp, T_, d, d, d, st); ++launches;
+  // line 3 + stored-query update + rotary embedding
+  launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
+  // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
+  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, B.status,
+                st); ++launches;
+  // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
+  const int* kv_idx = kv_sparse ? B.idx : nullptr;
+  const int* kv_cnt = kv_sparse ? B.count : nullptr;
+  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_k, B.tmp, T_, d, d, 2 * d, st); ++launches;
+  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_v, B.tmp + d, T_, d, d, 2 * d, st); ++launches;
+  launch_kv_post_simt<T>(B.tmp, 2 * d, kv_idx, kv_cnt, B.rope_cs, (T*)B.kc, (T*)B.vc, g, st); ++launches;
+  // attention: Alg. 1 line 10 (all rows) or Alg. 2 lines 6, 8-10 (refresh set rows, others keep the cache)
+  launch_attention_simt<T>((const T*)B.q, (const T*)B.kc, (const T*)B.vc, o_sparse ? B.idx : nullptr,
+                           o_sparse ? B.count : nullptr, (T*)B.oc, g, st); ++launches;
+  // last line: output projection of every row
+  launch_out_proj_simt<T>((const T*)B.oc, (const T*)L->w.w_o, B.tmp, y, g, st); ++launches;
+  L->last_launches = launches;
+  CUDA_TRY(cudaGetLastError());
+  return DARE_OK;
+}
+
+dare_status_t validate_step(dare_layer_t* L, const void* x, int batch, int seq_act, int pos_begin, int mode,
+                            float tau, void* y) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!x || !y) return DARE_ERR_INVALID_ARG;
+  if (mode < DARE_MODE_DENSE || mode > DARE_MODE_BOTH) return DARE_ERR_INVALID_ARG;
+  if (isnan(tau)) return DARE_ERR_INVALID_ARG;
+  if (batch <= 0 || seq_act <= 0 || pos_begin < 0) return DARE_ERR_SHAPE;
+  if (batch > L->cfg.max_batch || (long)pos_begin + seq_act > L->cfg.max_seq) return DARE_ERR_SHAPE;
+  if (L->has_prev) {
+    if (batch != L->batch) return DARE_ERR_STATE;
+    if (pos_begin + seq_act > L->kv_len) return DARE_ERR_STATE;
+  } else if (pos_begin != 0) {
+    return DARE_ERR_STATE;
+  }
+  return DARE_OK;
+}
+
+dare_status_t enqueue_step(dare_layer_t* L, const void* x, int batch, int seq_act, int pos_begin, int mode, float tau,
+                           void* y, cudaStream_t st) {
+  StepGeom g;
+  g.batch = batch; g.seq_act = seq_act; g.pos_begin = pos_begin; g.max_seq = L->cfg.max_seq;
+  g.kv_len = L->has_prev ? L->kv_len : seq_act;
+  g.d = L->cfg.d_model; g.n_heads = L->cfg.n_heads; g.head_dim = L->cfg.head_dim; g.score_head = L->cfg.score_head;
+  dare_status_t s;
+  if (L->use_tc) {
+    s = step_tc(L, x, g, mode, tau, y, st);
+  } else if (L->cfg.dtype == DARE_BF16) {
+    s = step_simt<__nv_bfloat16>(L, (const __nv_bfloat16*)x, g, mode, tau, (__nv_bfloat16*)y, st);
+  } else {
+    s = step_simt<float>(L, (const float*)x, g, mode, tau, (float*)y, st);
+  }
+  if (s != DARE_OK) return s;
+  if (!L->has_prev) { L->kv_len = seq_act; L->batch = batch; }
+  L->has_prev = true;
+  L->last_geom = g;
+  return DARE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dare_abi_version(void) { return 1; }
+
+const char* dare_status_string(dare_status_t s) {
+  switch (s) {
+    case DARE_OK: return "ok";
+    case DARE_ERR_INVALID_ARG: return "invalid argument";
+    case DARE_ERR_SHAPE: return "shape outside the configured limits";
+    case DARE_ERR_STATE: return "call not legal in this state";
+    case DARE_ERR_ALIGN: return "pointer not aligned";
+    case DARE_ERR_WORKSPACE: return "workspace too small";
+    case DARE_ERR_CUDA: return "CUDA call failed";
+    case DARE_ERR_TIMEOUT: return "device-side wait timed out";
+    case DARE_ERR_UNSUPPORTED: return "configuration not supported";
+    case DARE_ERR_DEVICE_CHECK: return "device-side range check failed";
+  }
+  return "unknown status";
+}
+
+size_t dare_layer_workspace_bytes(const dare_layer_config_t* cfg) {
+  bool use_tc = false;
+  if (!valid_config(cfg) || !pick_path(cfg, &use_tc)) return 0;
+  return carve(cfg, use_tc, nullptr, nullptr);
+}
+
+dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer_weights_t* w, void* workspace,
+                                size_t workspace_bytes, dare_layer_t** out) {
+  if (!out) return DARE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || !w || !workspace) return DARE_ERR_INVALID_ARG;
+  if (!valid_config(cfg)) return DARE_ERR_INVALID_ARG;
+  bool use_tc = false;
+  if (!pick_path(cfg, &use_tc)) return DARE_ERR_UNSUPPORTED;
+  if (!w->w_q || !w->w_k || !w->w_v || !w->w_o || !w->rms_gain) return DARE_ERR_INVALID_ARG;
+  if (!aligned16(w->w_q) || !aligned16(w->w_k) || !aligned16(w->w_v) || !aligned16(w->w_o) || !aligned16(w->rms_gain))
+    return DARE_ERR_ALIGN;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0) return DARE_ERR_ALIGN;
+  const size_t need = carve(cfg, use_tc, nullptr, nullptr);
+  if (workspace_bytes < need) return DARE_ERR_WORKSPACE;
+  dare_layer_t* L = new (std::nothrow) dare_layer_t();
+  if (!L) return DARE_ERR_INVALID_ARG;
+  L->magic = kMagic;
+  L->cfg = *cfg;
+  L->w = *w;
+  L->use_tc = use_tc;
+  L->has_prev = false;
+  L->batch = 0;
+  L->kv_len = 0;
+  L->last_launches = 0;
+  L->tc = nullptr;
+  memset(&L->last_geom, 0, sizeof(L->last_geom));
+  carve(cfg, use_tc, (char*)workspace, &L->buf);
+  L->workspace = workspace;
+  L->workspace_bytes = need;
+  cudaError_t e = cudaMemset(L->buf.status, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(L->buf.count, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(L->buf.delta, 0, (size_t)cfg->max_batch * cfg->max_seq * sizeof(int));
+  if (e == cudaSuccess) {
+    launch_rope_table(L->buf.rope_cs, cfg->max_seq, cfg->head_dim, (double)cfg->rope_theta, 0);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { cudaGetLastError(); delete L; return DARE_ERR_CUDA; }
+  if (use_tc) {
+    dare_status_t s = tc_create(L);
+    if (s != DARE_OK) { delete L; return s; }
+  }
+  *out = L;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_step(dare_layer_t* L, const void* x, int batch, int seq_act, int pos_begin, int mode,
+                              float threshold, void* y, void* cuda_stream) {
+  dare_status_t s = validate_step(L, x, batch, seq_act, pos_begin, mode, threshold, y);
+  if (s != DARE_OK) return s;
+  if (!aligned16(x) || !aligned16(y)) return DARE_ERR_ALIGN;
+  return enqueue_step(L, x, batch, seq_act, pos_begin, mode, threshold, y, (cudaStream_t)cuda_stream);
+}
+
+dare_status_t dare_layer_step_host(dare_layer_t* L, const void* x_host, int batch, int seq_act, int pos_begin, int mode,
+                                   float threshold, void* y_host, void* cuda_stream) {
+  dare_status_t s = validate_step(L, x_host, batch, seq_act, pos_begin, mode, threshold, y_host);
+  if (s != DARE_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  const size_t bytes = (size_t)batch * seq_act * L->cfg.d_model * e;
+  CUDA_TRY(cudaMemcpyAsync(L->buf.x_stage, x_host, bytes, cudaMemcpyHostToDevice, st));
+  s = enqueue_step(L, L->buf.x_stage, batch, seq_act, pos_begin, mode, threshold, L->buf.y_stage, st);
+  if (s != DARE_OK) return s;
+  CUDA_TRY(cudaMemcpyAsync(y_host, L->buf.y_stage, bytes, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_reset(dare_layer_t* L) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  L->has_prev = false;
+  L->batch = 0;
+  L->kv_len = 0;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_destroy(dare_layer_t* L) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (L->use_tc) tc_destroy(L);
+  L->magic = 0;
+  delete L;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_status(dare_layer_t* L, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int dev = 0;
+  CUDA_TRY(cudaMemcpyAsync(&dev, L->buf.status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (dev == kDevTimeout) return DARE_ERR_TIMEOUT;
+  if (dev != kDevOk) return DARE_ERR_DEVICE_CHECK;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_last_selection(dare_layer_t* L, int32_t* idx_host, int32_t* count_host,
+                                        int32_t* batch_off_host, float* scores_host, int32_t* delta_host,
+                                        void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!L->has_prev) return DARE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const StepGeom& g = L->last_geom;
+  const int T_ = g.tokens();
+  int count = 0;
+  CUDA_TRY(cudaMemcpyAsync(&count, L->buf.count, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (count < 0 || count > T_) return DARE_ERR_DEVICE_CHECK;
+  if (count_host) *count_host = count;
+  if (idx_host && count > 0)
+    CUDA_TRY(cudaMemcpyAsync(idx_host, L->buf.idx, (size_t)count * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (batch_off_host)
+    CUDA_TRY(cudaMemcpyAsync(batch_off_host, L->buf.batch_off, ((size_t)g.batch + 1) * sizeof(int),
+                             cudaMemcpyDeviceToHost, st));
+  if (scores_host)
+    CUDA_TRY(cudaMemcpyAsync(scores_host, L->buf.scores, (size_t)T_ * sizeof(float), cudaMemcpyDeviceToHost, st));
+  if (delta_host)
+    CUDA_TRY(cudaMemcpy2DAsync(delta_host, (size_t)g.seq_act * sizeof(int), L->buf.delta + g.pos_begin,
+                               (size_t)g.max_seq * sizeof(int), (size_t)g.seq_act * sizeof(int), g.batch,
+                               cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_read_caches(dare_layer_t* L, void* k_host, void* v_host, void* o_host, float* q_prev_host,
+                                     void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!L->has_prev) return DARE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  const size_t d = L->cfg.d_model, hd = L->cfg.head_dim;
+  const size_t row = d * e;
+  const void* src[3] = {L->buf.kc, L->buf.vc, L->buf.oc};
+  void* dst[3] = {k_host, v_host, o_host};
+  for (int i = 0; i < 3; ++i)
+    if (dst[i])
+      CUDA_TRY(cudaMemcpy2DAsync(dst[i], (size_t)L->kv_len * row, src[i], (size_t)L->cfg.max_seq * row,
+                                 (size_t)L->kv_len * row, L->batch, cudaMemcpyDeviceToHost, st));
+  if (q_prev_host)
+    CUDA_TRY(cudaMemcpy2DAsync(q_prev_host, (size_t)L->kv_len * hd * 4, L->buf.q_prev, (size_t)L->cfg.max_seq * hd * 4,
+                               (size_t)L->kv_len * hd * 4, L->batch, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return DARE_OK;
+}
+
+struct StateHeader {
+  uint32_t magic;
+  int32_t has_prev, batch, kv_len;
+  int32_t d_model, head_dim, max_batch, max_seq, dtype;
+  int32_t reserved[7];
+};
+
+size_t dare_layer_state_bytes(const dare_layer_t* L) {
+  if (check_handle(L) != DARE_OK) return 0;
+  const size_t Tm = (size_t)L->cfg.max_batch * L->cfg.max_seq;
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  return sizeof(StateHeader) + Tm * L->cfg.head_dim * 4 + 3 * Tm * L->cfg.d_model * e + Tm * 4;
+}
+
+dare_status_t dare_layer_export_state(dare_layer_t* L, void* dst_host, size_t bytes, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!dst_host) return DARE_ERR_INVALID_ARG;
+  if (bytes < dare_layer_state_bytes(L)) return DARE_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t Tm = (size_t)L->cfg.max_batch * L->cfg.max_seq;
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  StateHeader h;
+  memset(&h, 0, sizeof(h));
+  h.magic = kMagic; h.has_prev = L->has_prev; h.batch = L->batch; h.kv_len = L->kv_len;
+  h.d_model = L->cfg.d_model; h.head_dim = L->cfg.head_dim; h.max_batch = L->cfg.max_batch; h.max_seq = L->cfg.max_seq;
+  h.dtype = L->cfg.dtype;
+  char* p = (char*)dst_host;
+  memcpy(p, &h, sizeof(h)); p += sizeof(h);
+  const void* src[5] = {L->buf.q_prev, L->buf.kc, L->buf.vc, L->buf.oc, L->buf.delta};
+  const size_t sz[5] = {Tm * L->cfg.head_dim * 4, Tm * L->cfg.d_model * e, Tm * L->cfg.d_model * e,
+                        Tm * L->cfg.d_model * e, Tm * 4};
+  for (int i = 0; i < 5; ++i) {
+    CUDA_TRY(cudaMemcpyAsync(p, src[i], sz[i], cudaMemcpyDeviceToHost, st));
+    p += sz[i];
+  }
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_import_state(dare_layer_t* L, const void* src_host, size_t bytes, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!src_host) return DARE_ERR_INVALID_ARG;
+  if (bytes < dare_layer_state_bytes(L)) return DARE_ERR_WORKSPACE;
+  StateHeader h;
+  memcpy(&h, src_host, sizeof(h));
+  if (h.magic != kMagic || h.d_model != L->cfg.d_model || h.head_dim != L->cfg.head_dim ||
+      h.max_batch != L->cfg.max_batch || h.max_seq != L->cfg.max_seq || h.dtype != L->cfg.dtype)
+    return DARE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t Tm = (size_t)L->cfg.max_batch * L->cfg.max_seq;
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  const char* p = (const char*)src_host + sizeof(h);
+  void* dst[5] = {L->buf.q_prev, L->buf.kc, L->buf.vc, L->buf.oc, L->buf.delta};
+  const size_t sz[5] = {Tm * L->cfg.head_dim * 4, Tm * L->cfg.d_model * e, Tm * L->cfg.d_model * e,
+                        Tm * L->cfg.d_model * e, Tm * 4};
+  for (int i = 0; i < 5; ++i) {
+    CUDA_TRY(cudaMemcpyAsync(dst[i], p, sz[i], cudaMemcpyHostToDevice, st));
+    p += sz[i];
+  }
+  CUDA_TRY(cudaStreamSynchronize(st));
+  L->has_prev = h.has_prev != 0;
+  L->batch = h.batch;
+  L->kv_len = h.kv_len;
+  return DARE_OK;
+}
+
+int dare_layer_last_launch_count(const dare_layer_t* L) {
+  if (check_handle(L) != DARE_OK) return 0;
+  return L->last_launches;
+}
+
+}  // extern "C"

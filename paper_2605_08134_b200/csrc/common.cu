@@ -1,0 +1,229 @@
+// Memory-bound kernels shared by both kernel paths: rotary table, RMSNorm, threshold + compaction, row gather.
+#include "dare_internal.h"
+
+namespace dare {
+
+// ------------------------------------------------------------------------------------------------ rotary table
+// cs[pos][j] = (cos, sin)(pos * theta^(-2j/head_dim)), evaluated in fp64 and stored as fp32.
+__global__ void rope_table_kernel(float2* cs, int max_seq, int half, double theta, int head_dim) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= max_seq * half) return;
+  int pos = i / half, j = i % half;
+  double inv_freq = pow(theta, -2.0 * (double)j / (double)head_dim);
+  double s, c;
+  sincos((double)pos * inv_freq, &s, &c);
+  cs[i] = make_float2((float)c, (float)s);
+}
+
+void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaStream_t st) {
+  int half = head_dim / 2;
+  int n = max_seq * half;
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(reinterpret_cast<float2*>(cs), max_seq, half, theta, head_dim);
+}
+
+// ------------------------------------------------------------------------------------------------ RMSNorm
+// Alg. 1/2 line 1.  One CTA per token row, 16-byte accesses, the row held in registers between the two passes.
+template <typename T>
+struct Vec16;
+template <>
+struct Vec16<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
+    float4 t = *reinterpret_cast<const float4*>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  static __device__ __forceinline__ void store(float* p, const float (&v)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+};
+template <>
+struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
+    uint4 t = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(h[i]);
+      v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
+    uint4 t;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    *reinterpret_cast<uint4*>(p) = t;
+  }
+};
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = (lane < nw) ? red[lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  __syncthreads();
+  return t;
+}
+
+template <typename T, int MAXV>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, const float* __restrict__ gain,
+                                                      T* __restrict__ xn, int d, float eps) {
+  constexpr int N = Vec16<T>::N;
+  __shared__ float red[32];
+  const size_t row = blockIdx.x;
+  const T* xr = x + row * d;
+  T* yr = xn + row * d;
+  const int nvec = d / N;
+  float v[MAXV][N];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      Vec16<T>::load(xr + vi * N, v[i]);
+#pragma unroll
+      for (int e = 0; e < N; ++e) ss += v[i][e] * v[i][e];
+    }
+  }
+  for (int vi = threadIdx.x + MAXV * blockDim.x; vi < nvec; vi += blockDim.x) {  // rows wider than the register file
+    float t[N];
+    Vec16<T>::load(xr + vi * N, t);
+#pragma unroll
+    for (int e = 0; e < N; ++e) ss += t[e] * t[e];
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      float g[N];
+      if (N == 4) {
+        float4 t = *reinterpret_cast<const float4*>(gain + vi * N);
+        g[0] = t.x; g[1] = t.y; g[2] = t.z; g[3] = t.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < N; e += 4) {
+          float4 t = *reinterpret_cast<const float4*>(gain + vi * N + e);
+          g[e] = t.x; g[e + 1] = t.y; g[e + 2] = t.z; g[e + 3] = t.w;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < N; ++e) v[i][e] = v[i][e] * r * g[e];
+      Vec16<T>::store(yr + vi * N, v[i]);
+    }
+  }
+  for (int vi = threadIdx.x + MAXV * blockDim.x; vi < nvec; vi += blockDim.x) {
+    float t[N];
+    Vec16<T>::load(xr + vi * N, t);
+#pragma unroll
+    for (int e = 0; e < N; ++e) t[e] = t[e] * r * gain[vi * N + e];
+    Vec16<T>::store(yr + vi * N, t);
+  }
+}
+
+template <typename T>
+void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st) {
+  if (rows <= 0) return;
+  int nvec = d / Vec16<T>::N;
+  int threads = nvec >= 512 ? 256 : (nvec >= 128 ? 128 : ((nvec + 31) / 32) * 32);
+  if (threads > 256) threads = 256;
+  rmsnorm_kernel<T, 2><<<rows, threads, 0, st>>>(x, gain, xn, d, eps);
+}
+template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t);
+template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, __nv_bfloat16*, int, int, float,
+                                            cudaStream_t);
+
+// ------------------------------------------------------------------------------------------------ selection
+// Eq. 2 and its complement: token t is refreshed iff !(s_t <= tau) (a NaN score refreshes).  The refresh set is
+// written as an ascending index list by warp ballot + popcount + a block prefix sum over warp totals; the
+// staleness counters of Sec. 4 are updated in the same pass.  One CTA walks the tokens in chunks of 1024, which
+// keeps the list ordered without any inter-CTA hand-off (T <= a few 10^4 per layer step).
+__global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
+                                                      StepGeom g, int* __restrict__ idx, int* __restrict__ count,
+                                                      int* __restrict__ batch_off, int* __restrict__ delta) {
+  __shared__ int warp_excl[32];
+  __shared__ int chunk_total;
+  const int T = g.tokens();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int base = 0;
+  for (int start = 0; start < T; start += 1024) {
+    const int t = start + threadIdx.x;
+    const bool valid = t < T;
+    bool sel = false;
+    if (valid) sel = select_all ? true : !(scores[t] <= tau);
+    const unsigned bal = __ballot_sync(0xffffffffu, sel);
+    const int lane_prefix = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_excl[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      int v = warp_excl[lane], inc = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      warp_excl[lane] = inc - v;
+      if (lane == 31) chunk_total = inc;
+    }
+    __syncthreads();
+    if (sel) idx[base + warp_excl[warp] + lane_prefix] = t;
+    if (valid) {
+      const int cr = g.cache_row(t);
+      delta[cr] = sel ? 0 : delta[cr] + 1;
+    }
+    base += chunk_total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *count = base;
+  // start of each sequence's slice: lower bound of b*seq_act in the ascending list
+  for (int b = threadIdx.x; b <= g.batch; b += blockDim.x) {
+    const int key = b * g.seq_act;
+    int lo = 0, hi = base;
+    while (lo < hi) {
+      int mid = (lo + hi) >> 1;
+      if (idx[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    batch_off[b] = lo;
+  }
+}
+
+void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
+                   int* batch_off, int* delta, int* status, cudaStream_t st) {
+  (void)status;
+  select_kernel<<<1, 1024, 0, st>>>(scores, tau, (select_all || scores == nullptr) ? 1 : 0, g, idx, count, batch_off,
+                                    delta);
+}
+
+// ------------------------------------------------------------------------------------------------ row gather
+// dst[r, :] = src[idx[r], :] for r < *count (Alg. 1 line 6: x_norm restricted to the refresh set).
+template <typename T>
+__global__ void __launch_bounds__(256) gather_rows_kernel(const T* __restrict__ src, const int* __restrict__ idx,
+                                                          const int* __restrict__ count, T* __restrict__ dst,
+                                                          int max_rows, int d) {
+  const int n = min(*count, max_rows);
+  constexpr int N = 16 / sizeof(T);
+  const int nvec = d / N;
+  for (int r = blockIdx.x; r < n; r += gridDim.x) {
+    const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)idx[r] * d);
+    uint4* o = reinterpret_cast<uint4*>(dst + (size_t)r * d);
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) o[v] = s[v];
+  }
+}
+
+template <typename T>
+void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st) {
+  if (max_rows <= 0) return;
+  int grid = max_rows < 148 * 8 ? max_rows : 148 * 8;
+  gather_rows_kernel<T><<<grid, 256, 0, st>>>(src, idx, count, dst, max_rows, d);
+}
+template void launch_gather_rows<float>(const float*, const int*, const int*, float*, int, int, cudaStream_t);
+template void launch_gather_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*, int, int,
+                                                cudaStream_t);
+
+}  // namespace dare

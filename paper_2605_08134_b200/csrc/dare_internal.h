@@ -1,0 +1,73 @@
+// Internal declarations shared by the translation units of libdare (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dare.h"
+
+namespace dare {
+
+// Device status word values (mirrors dare_status_t for the two device-reported codes).
+constexpr int kDevOk = 0;
+constexpr int kDevTimeout = DARE_ERR_TIMEOUT;
+constexpr int kDevCheck = DARE_ERR_DEVICE_CHECK;
+
+// Geometry of one step, passed by value to kernels.
+struct StepGeom {
+  int batch;      // B
+  int seq_act;    // rows of each sequence covered by this step
+  int pos_begin;  // first covered position
+  int max_seq;    // row stride between sequences inside the caches
+  int kv_len;     // keys [0, kv_len) of each sequence are valid
+  int d;          // d_model
+  int n_heads;
+  int head_dim;
+  int score_head;
+  __host__ __device__ int tokens() const { return batch * seq_act; }
+  // flat active index -> row inside the [max_batch*max_seq] caches
+  __host__ __device__ int cache_row(int t) const { return (t / seq_act) * max_seq + pos_begin + (t % seq_act); }
+  __host__ __device__ int position(int t) const { return pos_begin + (t % seq_act); }
+};
+
+// ---- kernels common to both paths (common.cu) -------------------------------------------------------------
+void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaStream_t st);
+template <typename T>
+void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st);
+// Threshold + ballot/prefix-sum compaction + staleness update.  `scores == nullptr` or `select_all` selects all.
+void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
+                   int* batch_off, int* delta, int* status, cudaStream_t st);
+template <typename T>
+void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
+
+// ---- SIMT path (simt.cu) ----------------------------------------------------------------------------------
+// C[m, n] (fp32, ld = ldc) = sum_k A[arow(m), k] * W[n, k];  arow(m) = a_idx ? a_idx[m] : m;
+// rows m >= *count (when count != nullptr) are skipped.
+template <typename T>
+void launch_gemm_simt(const T* a, const int* a_idx, const int* count, const T* w, float* c, int m_max, int n, int k,
+                      int ldc, cudaStream_t st);
+// Q post-pass: score of the scoring head against q_prev (fp32, cache rows), q_prev update, rotary embedding,
+// store Q in the layer dtype.
+template <typename T>
+void launch_q_post_simt(const float* qf, int ldq, const float* rope_cs, float* q_prev, float* scores, bool has_prev,
+                        T* q, const StepGeom& g, cudaStream_t st);
+// K/V post-pass: rows r < *count (or all when idx == nullptr): rotary embedding on K, store K and V to cache rows.
+template <typename T>
+void launch_kv_post_simt(const float* kvf, int ld, const int* idx, const int* count, const float* rope_cs, T* kc,
+                         T* vc, const StepGeom& g, cudaStream_t st);
+// Attention: query rows = idx[0..count) (or all rows when idx == nullptr), one warp per (row, head);
+// output rows go to the O cache.
+template <typename T>
+void launch_attention_simt(const T* q, const T* kc, const T* vc, const int* idx, const int* count, T* oc,
+                           const StepGeom& g, cudaStream_t st);
+// y[t, :] = W_O oc[cache_row(t), :]
+template <typename T>
+void launch_out_proj_simt(const T* oc, const T* w_o, float* tmp, T* y, const StepGeom& g, cudaStream_t st);
+
+// ---- tensor-core path (gemm_tc.cu, attn_tc.cu) -----------------------------------------------------------
+struct TcLayerMaps;  // tensor maps and launch state, owned by the handle
+bool tc_supported(const dare_layer_config_t& cfg);
+size_t tc_maps_bytes();
+
+}  // namespace dare

@@ -1,0 +1,250 @@
+"""ctypes binding of libdare: the same entry points as include/dare.h, argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used by callers for device memory and streams.
+Importing this module loads the shared library and fails loudly if it is missing (there is no fallback).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdare.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_STATE, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, \
+    ERR_DEVICE_CHECK = range(1, 10)
+MODE_DENSE, MODE_KV, MODE_O, MODE_BOTH = 0, 1, 2, 3
+F32, BF16 = 0, 1
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+
+
+class LayerConfig(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("d_model", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("rope_theta", C.c_float), ("rms_eps", C.c_float),
+                ("dtype", C.c_int32), ("score_head", C.c_int32), ("kernel_path", C.c_int32)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [("w_q", C.c_void_p), ("w_k", C.c_void_p), ("w_v", C.c_void_p), ("w_o", C.c_void_p),
+                ("rms_gain", C.c_void_p)]
+
+
+class DareError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2605_08134_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, f32, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+    sig = {
+        "dare_abi_version": (C.c_int, []),
+        "dare_status_string": (C.c_char_p, [C.c_int]),
+        "dare_layer_workspace_bytes": (sz, [C.POINTER(LayerConfig)]),
+        "dare_layer_create": (C.c_int, [C.POINTER(LayerConfig), C.POINTER(LayerWeights), vp, sz, C.POINTER(vp)]),
+        "dare_layer_step": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
+        "dare_layer_step_host": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
+        "dare_layer_reset": (C.c_int, [vp]),
+        "dare_layer_destroy": (C.c_int, [vp]),
+        "dare_layer_status": (C.c_int, [vp, vp]),
+        "dare_layer_last_selection": (C.c_int, [vp, vp, vp, vp, vp, vp, vp]),
+        "dare_layer_read_caches": (C.c_int, [vp, vp, vp, vp, vp, vp]),
+        "dare_layer_state_bytes": (sz, [vp]),
+        "dare_layer_export_state": (C.c_int, [vp, vp, sz, vp]),
+        "dare_layer_import_state": (C.c_int, [vp, vp, sz, vp]),
+        "dare_layer_last_launch_count": (C.c_int, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib, tuple(sig)
+
+
+_lib, EXPORTS = _load()
+
+
+def status_string(status: int) -> str:
+    return _lib.dare_status_string(status).decode()
+
+
+def abi_version() -> int:
+    return _lib.dare_abi_version()
+
+
+def make_config(d_model, n_heads, head_dim, max_batch, max_seq, rope_theta, rms_eps, dtype, score_head=0,
+                kernel_path=PATH_AUTO) -> LayerConfig:
+    return LayerConfig(C.sizeof(LayerConfig), d_model, n_heads, head_dim, max_batch, max_seq, rope_theta, rms_eps,
+                       dtype, score_head, kernel_path)
+
+
+def dare_layer_workspace_bytes(cfg: LayerConfig) -> int:
+    return _lib.dare_layer_workspace_bytes(C.byref(cfg))
+
+
+def dare_layer_create(cfg: LayerConfig, weights: LayerWeights, workspace_ptr: int, workspace_bytes: int):
+    """-> (status, handle)"""
+    out = C.c_void_p()
+    st = _lib.dare_layer_create(C.byref(cfg) if cfg is not None else None,
+                                C.byref(weights) if weights is not None else None,
+                                workspace_ptr, workspace_bytes, C.byref(out))
+    return st, out.value
+
+
+def dare_layer_step(handle, x_ptr, batch, seq_act, pos_begin, mode, threshold, y_ptr, stream=0) -> int:
+    return _lib.dare_layer_step(handle, x_ptr, batch, seq_act, pos_begin, mode, threshold, y_ptr, stream)
+
+
+def dare_layer_step_host(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr, stream=0) -> int:
+    return _lib.dare_layer_step_host(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr, stream)
+
+
+def dare_layer_reset(handle) -> int:
+    return _lib.dare_layer_reset(handle)
+
+
+def dare_layer_destroy(handle) -> int:
+    return _lib.dare_layer_destroy(handle)
+
+
+def dare_layer_status(handle, stream=0) -> int:
+    return _lib.dare_layer_status(handle, stream)
+
+
+def dare_layer_last_selection(handle, idx_ptr, count_ptr, batch_off_ptr, scores_ptr, delta_ptr, stream=0) -> int:
+    return _lib.dare_layer_last_selection(handle, idx_ptr, count_ptr, batch_off_ptr, scores_ptr, delta_ptr, stream)
+
+
+def dare_layer_read_caches(handle, k_ptr, v_ptr, o_ptr, q_prev_ptr, stream=0) -> int:
+    return _lib.dare_layer_read_caches(handle, k_ptr, v_ptr, o_ptr, q_prev_ptr, stream)
+
+
+def dare_layer_state_bytes(handle) -> int:
+    return _lib.dare_layer_state_bytes(handle)
+
+
+def dare_layer_export_state(handle, dst_ptr, nbytes, stream=0) -> int:
+    return _lib.dare_layer_export_state(handle, dst_ptr, nbytes, stream)
+
+
+def dare_layer_import_state(handle, src_ptr, nbytes, stream=0) -> int:
+    return _lib.dare_layer_import_state(handle, src_ptr, nbytes, stream)
+
+
+def dare_layer_last_launch_count(handle) -> int:
+    return _lib.dare_layer_last_launch_count(handle)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+class Layer:
+    """Convenience wrapper: owns the torch tensors behind a handle (weights, workspace) and marshals pointers.
+
+    No arithmetic happens here.  `x`/`y` are torch CUDA tensors (or pinned host tensors for `step_host`).
+    """
+
+    def __init__(self, shape, weights: dict, device="cuda:0", kernel_path=PATH_AUTO, max_batch=None, max_seq=None):
+        import numpy as np
+        import torch
+        self.torch = torch
+        self.shape = shape
+        self.device = torch.device(device)
+        self.tdtype = torch.bfloat16 if shape.dtype == BF16 else torch.float32
+        self.max_batch = max_batch or shape.batch
+        self.max_seq = max_seq or shape.seq
+        self.cfg = make_config(shape.d_model, shape.n_heads, shape.head_dim, self.max_batch, self.max_seq,
+                               shape.rope_theta, shape.rms_eps, shape.dtype, 0, kernel_path)
+        self._w = {}
+        for k in ("w_q", "w_k", "w_v", "w_o"):
+            v = weights[k]
+            t = v if isinstance(v, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(v, np.float32))
+            self._w[k] = t.to(self.device, self.tdtype).contiguous()
+        g = weights["rms_gain"]
+        g = g if isinstance(g, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(g, np.float32))
+        self._w["rms_gain"] = g.to(self.device, torch.float32).contiguous()
+        self.wstruct = LayerWeights(*(self._w[k].data_ptr() for k in ("w_q", "w_k", "w_v", "w_o", "rms_gain")))
+        nbytes = dare_layer_workspace_bytes(self.cfg)
+        if nbytes == 0:
+            raise DareError(ERR_UNSUPPORTED, "dare_layer_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        with torch.cuda.device(self.device):
+            st, self.handle = dare_layer_create(self.cfg, self.wstruct, base, nbytes)
+        if st != OK:
+            raise DareError(st, "dare_layer_create")
+
+    def _stream(self):
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def step(self, x, mode, threshold, y=None, pos_begin=0):
+        torch = self.torch
+        assert x.is_cuda and x.dtype == self.tdtype and x.is_contiguous()
+        if y is None:
+            y = torch.empty_like(x)
+        st = dare_layer_step(self.handle, x.data_ptr(), x.shape[0], x.shape[1], pos_begin, mode, threshold,
+                             y.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_step")
+        return y
+
+    def step_host(self, x_host, mode, threshold, y_host, pos_begin=0):
+        st = dare_layer_step_host(self.handle, x_host.data_ptr(), x_host.shape[0], x_host.shape[1], pos_begin, mode,
+                                  threshold, y_host.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_step_host")
+        return y_host
+
+    def reset(self):
+        st = dare_layer_reset(self.handle)
+        if st != OK:
+            raise DareError(st, "dare_layer_reset")
+
+    def status(self) -> int:
+        return dare_layer_status(self.handle, self._stream())
+
+    def last_selection(self, batch, seq_act):
+        """-> dict(idx, count, batch_off, scores, delta) as numpy arrays."""
+        import numpy as np
+        T = batch * seq_act
+        idx = np.zeros(T, np.int32)
+        cnt = np.zeros(1, np.int32)
+        boff = np.zeros(batch + 1, np.int32)
+        sc = np.zeros(T, np.float32)
+        dl = np.zeros(T, np.int32)
+        st = dare_layer_last_selection(self.handle, idx.ctypes.data, cnt.ctypes.data, boff.ctypes.data,
+                                       sc.ctypes.data, dl.ctypes.data, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_last_selection")
+        n = int(cnt[0])
+        return {"idx": idx[:n].copy(), "count": n, "batch_off": boff, "scores": sc, "delta": dl.reshape(batch, seq_act)}
+
+    def read_caches(self, batch, kv_len):
+        """-> dict(k, v, o, q_prev) as float32 numpy arrays [batch, kv_len, ...]."""
+        import numpy as np
+        torch = self.torch
+        d, hd = self.shape.d_model, self.shape.head_dim
+        host = [torch.empty((batch, kv_len, d), dtype=self.tdtype) for _ in range(3)]
+        qp = np.zeros((batch, kv_len, hd), np.float32)
+        st = dare_layer_read_caches(self.handle, host[0].data_ptr(), host[1].data_ptr(), host[2].data_ptr(),
+                                    qp.ctypes.data, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_read_caches")
+        k, v, o = (h.float().numpy() for h in host)
+        return {"k": k, "v": v, "o": o, "q_prev": qp}
+
+    def launch_count(self) -> int:
+        return dare_layer_last_launch_count(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            dare_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

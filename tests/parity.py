@@ -1,0 +1,84 @@
+"""Helpers shared by the GPU parity tests: drive the CUDA library and the fp64 oracle with the same arrays."""
+import numpy as np
+
+from oracle import dare_oracle as orc
+from paper_2605_08134_b200 import workloads as wl
+
+TOL_F32 = 1e-4     # fp32 path: max-abs and RMS error, relative to max(1, RMS(oracle))
+TOL_BF16 = 2e-2    # bf16 path
+SCORE_ATOL = {wl.DTYPE_F32: 2e-6, wl.DTYPE_BF16: 1e-3}
+MARGIN = 1e-3      # every oracle score must be at least this far from tau for the index set to be bit-exact
+
+
+def tol_of(dtype):
+    return TOL_BF16 if dtype == wl.DTYPE_BF16 else TOL_F32
+
+
+def assert_close(name, got, want, tol):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    assert got.shape == want.shape, (name, got.shape, want.shape)
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    rms_o = float(np.sqrt(np.mean(want ** 2))) if want.size else 0.0
+    bound = tol * max(1.0, rms_o)
+    err = got - want
+    max_abs = float(np.max(np.abs(err))) if err.size else 0.0
+    rms = float(np.sqrt(np.mean(err ** 2))) if err.size else 0.0
+    assert max_abs <= bound, f"{name}: max-abs {max_abs:.3e} > {bound:.3e} (rms(o)={rms_o:.3e})"
+    assert rms <= bound, f"{name}: rms {rms:.3e} > {bound:.3e}"
+    return max_abs, rms, rms_o
+
+
+def oracle_layer(shape, w, max_batch=None, max_seq=None):
+    return orc.OracleLayer(shape.d_model, shape.n_heads, shape.head_dim, max_batch or shape.batch,
+                           max_seq or shape.seq, shape.rope_theta, shape.rms_eps,
+                           w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"])
+
+
+def to_device(x, shape, device="cuda:0"):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(device)
+    return t.to(torch.bfloat16) if shape.dtype == wl.DTYPE_BF16 else t
+
+
+def check_margin(scores, tau):
+    s = np.asarray(scores, np.float64)
+    s = s[np.isfinite(s)]
+    if s.size:
+        gap = np.min(np.abs(s - tau))
+        assert gap >= MARGIN, f"workload puts a score {gap:.2e} from tau; the index set would not be well defined"
+
+
+def compare_step(glayer, olayer, x, mode, tau, shape, pos_begin=0, check_caches=True, first=False, stats=None):
+    """One step on both sides, then element-by-element comparison of everything the step defines."""
+    import torch
+    B, S_act = x.shape[0], x.shape[1]
+    xd = to_device(x, shape)
+    yg = glayer.step(xd, mode, tau, pos_begin=pos_begin)
+    torch.cuda.synchronize()
+    yo = olayer.step(x, mode, tau, pos_begin=pos_begin)
+    assert glayer.status() == 0
+    tol = tol_of(shape.dtype)
+    sel = glayer.last_selection(B, S_act)
+    if not first and mode != orc.MODE_DENSE:
+        check_margin(olayer.last_scores, tau)
+    # index set: bit-exact, ascending
+    np.testing.assert_array_equal(sel["idx"], olayer.last_idx)
+    assert sel["count"] == len(olayer.last_idx)
+    np.testing.assert_array_equal(sel["batch_off"], olayer.last_batch_off)
+    np.testing.assert_array_equal(sel["delta"], olayer.delta[:B, pos_begin:pos_begin + S_act])
+    if first:
+        assert np.isinf(sel["scores"]).all()
+    else:
+        np.testing.assert_allclose(sel["scores"], olayer.last_scores, rtol=0, atol=SCORE_ATOL[shape.dtype])
+    res = {"y": assert_close("y", yg.float().cpu().numpy(), yo, tol)}
+    if check_caches:
+        kv_len = olayer.kv_len
+        c = glayer.read_caches(B, kv_len)
+        res["k"] = assert_close("k_cache", c["k"], olayer.k_cache[:B, :kv_len], tol)
+        res["v"] = assert_close("v_cache", c["v"], olayer.v_cache[:B, :kv_len], tol)
+        res["o"] = assert_close("o_cache", c["o"], olayer.o_cache[:B, :kv_len], tol)
+        assert_close("q_prev", c["q_prev"], olayer.q_prev[:B, :kv_len], tol)
+    if stats is not None:
+        stats.append(res)
+    return yg, yo
