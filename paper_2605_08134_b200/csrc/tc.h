@@ -1,0 +1,38 @@
+// Declarations of the tensor-core path (tcgen05 GEMM and attention kernels) shared between its translation units.
+#pragma once
+
+#include <cuda.h>
+
+#include "dare_internal.h"
+
+namespace dare {
+
+enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2 };
+
+struct GemmParams {
+  int K;                 // reduction length (multiple of 64)
+  int m_total;           // dense: tokens of the step; gathered: capacity of the row list
+  int seq_act;           // dense row mapping: rows per sequence ...
+  int tiles_per_seq;     // ... and 128-row tiles per sequence
+  int a_seq_stride;      // rows between sequences in A's row space
+  int a_row0;            // first row of the window in A's row space
+  const int* idx;        // gathered: token of each A row (ascending refresh set), else nullptr
+  const int* count;      // gathered: device count of rows, else nullptr
+  StepGeom g;
+  int hd_map;            // head width used for the column mapping of a tile
+  int n_split;           // tiles [0, n_split) use B0/out0, the rest B1/out1
+  __nv_bfloat16* out0;
+  __nv_bfloat16* out1;
+  int ld_out;
+  int out_is_cache;      // output rows addressed by cache row (1) or by flat token index (0)
+  const float2* rope;
+  float* q_prev;
+  float* scores;
+  int has_prev;
+  int* status;
+};
+
+cudaError_t launch_gemm_tc(int bn, int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
+                           const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st);
+
+}  // namespace dare

@@ -6,7 +6,7 @@ from paper_2605_08134_b200 import workloads as wl
 
 TOL_F32 = 1e-4     # fp32 path: max-abs and RMS error, relative to max(1, RMS(oracle))
 TOL_BF16 = 2e-2    # bf16 path
-SCORE_ATOL = {wl.DTYPE_F32: 2e-6, wl.DTYPE_BF16: 1e-3}
+SCORE_ATOL = {wl.DTYPE_F32: 2e-6, wl.DTYPE_BF16: 5e-3}   # diagnostic only; bf16 x_norm rounding moves a cosine by ~2^-8/sqrt(head_dim)
 MARGIN = 1e-3      # every oracle score must be at least this far from tau for the index set to be bit-exact
 
 

@@ -1,0 +1,95 @@
+"""GPU parity of the tensor-core kernel path (tcgen05 / TMEM / TMA) against the fp64 oracle."""
+import copy
+
+import numpy as np
+import pytest
+
+from paper_2605_08134_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+MODES = {"kv": 1, "o": 2, "both": 3, "dense": 0}
+
+
+@pytest.fixture(scope="module")
+def dare():
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare as d
+    return d
+
+
+@pytest.mark.parametrize("mode", list(MODES))
+def test_small_llada_shaped_layer_ragged(dare, mode):
+    """4 heads x 128, batch 2, seq 320 (2.5 row tiles per sequence), three steps."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=512, n_heads=4, batch=2, seq=320, prompt=160)
+    w = wl.make_weights(shape, 21)
+    hs = wl.HiddenStream(shape, 21)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), MODES[mode], 0.1, shape, first=True)
+    for t in range(2):
+        ch = wl.uniform_positions(hs.rng, shape, (41, 150)[t])
+        parity.compare_step(g, o, hs.advance(ch), MODES[mode], 0.1, shape)
+        if mode != "dense":
+            np.testing.assert_array_equal(g.last_selection(2, 320)["idx"], np.nonzero(ch.reshape(-1))[0])
+    g.close()
+
+
+def test_tensor_path_agrees_with_cuda_core_path(dare):
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=1, seq=200, prompt=100)
+    w, x0, x1, ch = wl.two_step_case(shape, 30, seed=8)
+    a = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    b = dare.Layer(shape, w, kernel_path=dare.PATH_SIMT)
+    for x in (x0, x1):
+        ya = a.step(parity.to_device(x, shape), 3, 0.1)
+        yb = b.step(parity.to_device(x, shape), 3, 0.1)
+        parity.assert_close("tensor vs cuda-core", ya.float().cpu().numpy(), yb.float().cpu().numpy(), 2e-2)
+    np.testing.assert_array_equal(a.last_selection(1, 200)["idx"], b.last_selection(1, 200)["idx"])
+    a.close(); b.close()
+
+
+def test_window_steps_tensor_path(dare):
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=2, seq=288, prompt=128)
+    w = wl.make_weights(shape, 6)
+    hs = wl.HiddenStream(shape, 6)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    p = shape.prompt
+    for t in range(3):
+        ch = wl.uniform_positions(hs.rng, shape, 30)
+        x = hs.advance(ch)
+        parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), (3, 1, 2)[t], 0.1, shape, pos_begin=p)
+    g.close()
+
+
+@pytest.fixture(scope="module")
+def config2():
+    shape = wl.LLADA_LAYER
+    w = wl.make_weights(shape)
+    hs = wl.HiddenStream(shape)
+    x0 = hs.first()
+    o = parity.oracle_layer(shape, w)
+    y0 = o.step(x0, 0, 0.1)
+    return shape, w, hs, x0, o, y0
+
+
+@pytest.mark.parametrize("n_changed", [26, 67, 154, 256, 512])
+def test_config2_llada_layer_full_size(dare, config2, n_changed):
+    """Config 2: d=4096, 32 heads x 128, seq 512, bf16; changed fraction 5/13/30/50/100 %, all three reuse modes."""
+    shape, w, hs0, x0, o0, y0 = config2
+    hs = copy.deepcopy(hs0)
+    ch = wl.uniform_positions(hs.rng, shape, n_changed)
+    x1 = hs.advance(ch)
+    g = dare.Layer(shape, w)
+    assert g.cfg.kernel_path == dare.PATH_AUTO
+    for mode in ("both", "kv", "o"):
+        g.reset()
+        yg = g.step(parity.to_device(x0, shape), MODES[mode], 0.1)
+        parity.assert_close("y step0", yg.float().cpu().numpy(), y0, parity.TOL_BF16)
+        o = copy.deepcopy(o0)
+        parity.compare_step(g, o, x1, MODES[mode], 0.1, shape)
+        np.testing.assert_array_equal(g.last_selection(1, 512)["idx"], np.nonzero(ch.reshape(-1))[0])
+    g.close()
