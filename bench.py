@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the DARE layer step (per-layer latency and token-positions per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--mode both|kv|o|dense]
+                    [--changed 0.13] [--layers 8]
+
+One "step" = one `dare_layer_step` = the whole hot path (norm, Q projection + drift score, threshold +
+compaction, gathered K/V projection + cache scatter, row-sparse attention, output projection) over one batch.
+Workload at N = 1: the LLaDA-8B-shaped attention layer, batch 1, seq 512, bf16, 13 % of the tokens changed per
+step (87 % reuse), mode "both".  Steps rotate over `--layers` layer instances (8 x 134 MB of weights, far more than
+the 126 MB L2) and alternate between two hidden-state buffers so that every timed step refreshes the same
+planned token set.
+
+Prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle on the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+MODES = {"dense": 0, "kv": 1, "o": 2, "both": 3}
+TAU = 0.1
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_inputs(shape, changed_frac, seed, torch, device):
+    """Two hidden-state buffers A, B: B redraws `changed_frac` of the rows of A (uniform positions) and perturbs the
+    rest by N(0, (1e-3)^2) before bf16 rounding; stepping A -> B -> A ... refreshes the same set every time."""
+    import numpy as np
+    from paper_2605_08134_b200 import workloads as wl
+    hs = wl.HiddenStream(shape, seed)
+    xa = hs.first()
+    n = int(round(changed_frac * shape.seq))
+    changed = wl.uniform_positions(hs.rng, shape, n)
+    xb = hs.advance(changed)
+    to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device).to(torch.bfloat16)
+    return xa, xb, changed, to(xa), to(xb)
+
+
+def make_layers(shape, n_layers, seed, torch, device, dare):
+    layers = []
+    gen = torch.Generator(device=device)
+    for l in range(n_layers):
+        gen.manual_seed(seed * 1000 + l)
+        w = {k: (torch.randn((shape.d_model, shape.d_model), generator=gen, device=device, dtype=torch.float32) * 0.02)
+             .to(torch.bfloat16) for k in ("w_q", "w_k", "w_v", "w_o")}
+        w["rms_gain"] = torch.ones(shape.d_model, device=device, dtype=torch.float32)
+        layers.append(dare.Layer(shape, w, device=device))
+    return layers
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    shape = wl.LLADA_LAYER
+    mode = MODES[args.mode]
+    peaks = load_peaks()
+    # every rank runs its own replica (sequences are independent: batch sharding, no data-path collective)
+    xa_np, xb_np, changed, xa, xb = make_inputs(shape, args.changed, shape.seed + 1000 * rank, torch, device)
+    n_planned = int(changed.sum())
+    layers = make_layers(shape, args.layers, shape.seed + 17 * rank, torch, device, dare)
+    y = torch.empty_like(xa)
+    stream = torch.cuda.current_stream(device)
+    T = shape.tokens
+
+    def one_pass(steps, m, start_parity=0, host=None):
+        launches = 0
+        for i in range(steps):
+            lay = layers[i % len(layers)]
+            # the parity of a layer's own step count decides which buffer it sees next
+            k = lay._bench_steps
+            src = (xa, xb)[k & 1] if host is None else host[k & 1]
+            if host is None:
+                lay.step(src, m, TAU, y)
+            else:
+                lay.step_host(src, m, TAU, host[2])
+            lay._bench_steps = k + 1
+            launches += lay.launch_count()
+        return launches
+
+    def prime(m):
+        for lay in layers:
+            lay.reset()
+            lay._bench_steps = 0
+        one_pass(len(layers), m)          # first step of every layer is dense and fills its caches
+        torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(steps, m, host=None):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        launches = one_pass(steps, m, host=host)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        dev_ms = ev0.elapsed_time(ev1)
+        ms = wall * 1e3 if host is not None else dev_ms
+        if dist is not None:
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        barrier()
+        return ms, launches
+
+    # ---- reuse path: warm-up, then exactly K timed steps with the clocks sampled
+    prime(mode)
+    one_pass(max(args.warmup, 3), mode)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    total_ms, launches = timed(args.steps, mode)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    # selection really is the planned one
+    sel = layers[0].last_selection(shape.batch, shape.seq)
+    expect = T if mode == 0 else n_planned
+    assert sel["count"] == expect, (sel["count"], expect)
+    if mode != 0:
+        assert np.array_equal(sel["idx"], np.nonzero(changed.reshape(-1))[0])
+    assert all(l.status() == 0 for l in layers)
+
+    # ---- dense path of the same library, same protocol
+    prime(0)
+    one_pass(max(args.warmup, 3), 0)
+    dense_ms, _ = timed(args.steps, 0)
+    dense_ms_per_step = dense_ms / args.steps
+
+    # ---- per-kernel times: a second pass of K steps with an event before every kernel
+    prime(mode)
+    one_pass(max(args.warmup, 3), mode)
+    for lay in layers:
+        lay.set_profiling(True)
+    acc = {}
+    barrier()
+    for i in range(args.steps):
+        lay = layers[i % len(layers)]
+        k = lay._bench_steps
+        lay.step((xa, xb)[k & 1], mode, TAU, y)
+        lay._bench_steps = k + 1
+        for name, ms in lay.kernel_times():
+            acc.setdefault(name, []).append(ms)
+    for lay in layers:
+        lay.set_profiling(False)
+    kernels = {k: 1e3 * sum(v) / len(v) for k, v in acc.items()}          # microseconds per launch
+
+    # ---- end to end through the host-buffer entry point (pinned host x and y, copies inside the timed region)
+    prime(mode)
+    xh = [torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).pin_memory() for a in (xa_np, xb_np)]
+    yh = torch.empty_like(xh[0]).pin_memory()
+    one_pass(max(args.warmup, 3), mode, host=(xh[0], xh[1], yh))
+    e2e_ms, _ = timed(args.steps, mode, host=(xh[0], xh[1], yh))
+    e2e_ms_per_step = e2e_ms / args.steps
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (algorithmic work of the DARE step itself, never the dense work avoided)
+    d, n = shape.d_model, (n_planned if mode != 0 else T)
+    n_kv = n if (mode & 1) else T
+    n_o = n if (mode & 2) else T
+    work = {
+        "q_gemm": ("tensor", 2.0 * T * d * d),
+        "out_gemm": ("tensor", 2.0 * T * d * d),
+        "kv_gemm": ("hbm", 2.0 * d * d * 2 + 3.0 * n_kv * d * 2) if n_kv <= 215 else ("tensor", 4.0 * n_kv * d * d),
+        "attention": ("tensor", 4.0 * n_o * shape.seq * d),
+        "rmsnorm": ("hbm", 2.0 * T * d * 2),
+    }
+    rows = []
+    for name, us in kernels.items():
+        if name in work and us > 0:
+            bound, amount = work[name]
+            if bound == "hbm":
+                ach, peak, unit = amount / (us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
+            else:
+                ach, peak, unit = amount / (us * 1e-6) / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+            rows.append({"kernel": name, "us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": peak,
+                         "unit": unit, "frac": round(ach / peak, 4)})
+        else:
+            rows.append({"kernel": name, "us": round(us, 2)})
+    dom = max((r for r in rows if "bound" in r), key=lambda r: r["us"])
+    roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": None,
+                "peak_source": f"of {peaks['source']} (sustained figure: the kernel is timed inside the step)",
+                "timing": "CUDA events recorded by the library around each kernel, second pass of K steps"}
+
+    # ---- CPU baseline: the oracle as it stands, bounded sample
+    cpu = None if args.no_cpu_baseline else cpu_baseline(shape, xa_np, xb_np, layers[0], mode, budget_s=12.0)
+
+    tokens_per_s = world * T / (ms_per_step * 1e-3)
+    out = {
+        "metric": "tokens_per_s_through_one_dare_layer", "value": round(tokens_per_s, 1), "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
+        "us_per_layer": round(ms_per_step * 1e3, 2),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": shape.name, "d_model": d, "n_heads": shape.n_heads, "head_dim": shape.head_dim,
+                   "batch": shape.batch, "seq_len": shape.seq, "mode": args.mode, "changed_fraction": args.changed,
+                   "refreshed_tokens": n, "threshold": TAU, "layers_rotated": args.layers,
+                   "l2": "inputs larger than L2: weights of %d layer instances (%.0f MB) rotate"
+                         % (args.layers, args.layers * 4 * d * d * 2 / 1e6),
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "dense": {"ms_per_step": round(dense_ms_per_step, 5), "value": round(world * T / (dense_ms_per_step * 1e-3), 1),
+                  "speedup_of_reuse_path": round(dense_ms_per_step / ms_per_step, 3)},
+        "e2e": {"value": round(world * T / (e2e_ms_per_step * 1e-3), 1), "unit": "tokens/s",
+                "ms_per_step": round(e2e_ms_per_step, 5),
+                "h2d_bytes_per_step": T * d * 2, "d2h_bytes_per_step": T * d * 2},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": roofline,
+        "kernels": rows,
+        "cpu_baseline": cpu,
+        "paper_context": "paper reports up to 1.20x per-layer latency reduction (DARE-O, RTX A6000, bf16); not a target",
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(shape, xa_np, xb_np, layer0, mode, budget_s):
+    """Times the fp64 oracle on the host cores: one dense step to fill its caches, then reuse steps on the same
+    A/B buffers until about `budget_s` seconds have gone by."""
+    import numpy as np
+    from oracle import dare_oracle as orc
+    w = {k: layer0._w[k].float().cpu().numpy() for k in ("w_q", "w_k", "w_v", "w_o", "rms_gain")}
+    o = orc.OracleLayer(shape.d_model, shape.n_heads, shape.head_dim, shape.batch, shape.seq, shape.rope_theta,
+                        shape.rms_eps, w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"])
+    o.step(xa_np, mode, TAU)
+    bufs = (xb_np, xa_np)
+    t0 = time.perf_counter()
+    steps = 0
+    while True:
+        o.step(bufs[steps & 1], mode, TAU)
+        steps += 1
+        if time.perf_counter() - t0 > budget_s or steps >= 200:
+            break
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    return {"value": round(steps * shape.tokens / dt, 1), "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+            "sample": f"{steps} reuse steps of the full workload after one dense step, {dt:.1f} s, numpy fp64"}
+
+
+def run_reference(args):
+    """Reference arm: the fp64 oracle on the host cores, same workload, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import dare_oracle as orc
+    from paper_2605_08134_b200 import workloads as wl
+    shape = wl.LLADA_LAYER
+    mode = MODES[args.mode]
+    w = wl.make_weights(shape)
+    hs = wl.HiddenStream(shape, shape.seed)
+    xa = hs.first()
+    changed = wl.uniform_positions(hs.rng, shape, int(round(args.changed * shape.seq)))
+    xb = hs.advance(changed)
+    o = orc.OracleLayer(shape.d_model, shape.n_heads, shape.head_dim, shape.batch, shape.seq, shape.rope_theta,
+                        shape.rms_eps, w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"])
+    o.step(xa, mode, TAU)
+    bufs = (xb, xa)
+    warm = max(args.warmup, 1)
+    steps = min(args.steps, 40)             # bounded sample: each oracle step is a fraction of a second
+    for i in range(warm):
+        o.step(bufs[i & 1], mode, TAU)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        o.step(bufs[(warm + i) & 1], mode, TAU)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    value = round(steps * shape.tokens / dt, 1)
+    sample = f"{steps} reuse steps of the full workload after one dense step (numpy fp64 oracle)"
+    print(json.dumps({
+        "impl": "reference", "metric": "tokens_per_s_through_one_dare_layer", "value": value, "unit": "tokens/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": warm,
+        "ms_per_step": round(dt / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "mode": args.mode, "changed_fraction": args.changed, "threshold": TAU},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": int(cores), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="both", choices=list(MODES))
+    ap.add_argument("--changed", type=float, default=0.13)
+    ap.add_argument("--layers", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -157,6 +157,15 @@ size_t dare_layer_state_bytes(const dare_layer_t* layer);
 dare_status_t dare_layer_export_state(dare_layer_t* layer, void* dst_host, size_t bytes, void* cuda_stream);
 dare_status_t dare_layer_import_state(dare_layer_t* layer, const void* src_host, size_t bytes, void* cuda_stream);
 
+/* Optional per-kernel timing for benchmarks: when enabled, every step records a CUDA event before each of its
+ * kernels (on the step's stream).  `dare_layer_last_kernel_times` waits for the last step to finish and returns,
+ * for each kernel in launch order, its slot id and the time to the next mark in milliseconds.  DARE_ERR_STATE if
+ * profiling is off or no step has run since it was enabled. */
+dare_status_t dare_layer_set_profiling(dare_layer_t* layer, int enable);
+dare_status_t dare_layer_last_kernel_times(dare_layer_t* layer, int32_t* slot_host, float* ms_host, int capacity,
+                                           int* n_out);
+const char* dare_kernel_slot_name(int slot);
+
 /* Number of kernels the last dare_layer_step enqueued (for launch accounting in benchmarks). */
 int dare_layer_last_launch_count(const dare_layer_t* layer);
 

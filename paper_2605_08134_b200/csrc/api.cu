@@ -100,26 +100,36 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   const bool kv_sparse = has_prev && (mode & DARE_MODE_KV);
   const bool o_sparse = has_prev && (mode & DARE_MODE_O);
   int launches = 0;
+  prof_begin(L);
   // Alg. 1/2 line 1
+  prof_mark(L, SLOT_NORM, st);
   launch_rmsnorm<T>(x, L->w.rms_gain, (T*)B.xn, T_, d, L->cfg.rms_eps, st); ++launches;
   // line 2: dense Q projection
+  prof_mark(L, SLOT_Q_GEMM, st);
   launch_gemm_simt<T>((const T*)B.xn, nullptr, nullptr, (const T*)L->w.w_q, B.tmp, T_, d, d, d, st); ++launches;
   // line 3 + stored-query update + rotary embedding
+  prof_mark(L, SLOT_Q_POST, st);
   launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
+  prof_mark(L, SLOT_SELECT, st);
   launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, B.status,
                 st); ++launches;
   // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
   const int* kv_idx = kv_sparse ? B.idx : nullptr;
   const int* kv_cnt = kv_sparse ? B.count : nullptr;
+  prof_mark(L, SLOT_KV_GEMM, st);
   launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_k, B.tmp, T_, d, d, 2 * d, st); ++launches;
   launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_v, B.tmp + d, T_, d, d, 2 * d, st); ++launches;
+  prof_mark(L, SLOT_KV_POST, st);
   launch_kv_post_simt<T>(B.tmp, 2 * d, kv_idx, kv_cnt, B.rope_cs, (T*)B.kc, (T*)B.vc, g, st); ++launches;
   // attention: Alg. 1 line 10 (all rows) or Alg. 2 lines 6, 8-10 (refresh set rows, others keep the cache)
+  prof_mark(L, SLOT_ATTN, st);
   launch_attention_simt<T>((const T*)B.q, (const T*)B.kc, (const T*)B.vc, o_sparse ? B.idx : nullptr,
                            o_sparse ? B.count : nullptr, (T*)B.oc, g, st); ++launches;
   // last line: output projection of every row
+  prof_mark(L, SLOT_OUT_GEMM, st);
   launch_out_proj_simt<T>((const T*)B.oc, (const T*)L->w.w_o, B.tmp, y, g, st); ++launches;
+  prof_end(L, st);
   L->last_launches = launches;
   CUDA_TRY(cudaGetLastError());
   return DARE_OK;
@@ -217,6 +227,9 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->kv_len = 0;
   L->last_launches = 0;
   L->tc = nullptr;
+  L->prof_on = false;
+  L->prof_n = 0;
+  L->prof_ev_ready = false;
   memset(&L->last_geom, 0, sizeof(L->last_geom));
   carve(cfg, use_tc, (char*)workspace, &L->buf);
   L->workspace = workspace;
@@ -224,6 +237,14 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   cudaError_t e = cudaMemset(L->buf.status, 0, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(L->buf.count, 0, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(L->buf.delta, 0, (size_t)cfg->max_batch * cfg->max_seq * sizeof(int));
+  {
+    // caches start finite: tiles that reach past the valid extent are masked, but must not carry NaN bit patterns
+    const size_t cache_bytes = (size_t)cfg->max_batch * cfg->max_seq * cfg->d_model * (cfg->dtype == DARE_BF16 ? 2 : 4);
+    if (e == cudaSuccess) e = cudaMemset(L->buf.kc, 0, cache_bytes);
+    if (e == cudaSuccess) e = cudaMemset(L->buf.vc, 0, cache_bytes);
+    if (e == cudaSuccess) e = cudaMemset(L->buf.oc, 0, cache_bytes);
+    if (e == cudaSuccess && L->buf.xg) e = cudaMemset(L->buf.xg, 0, cache_bytes + (size_t)128 * cfg->d_model * 2);
+  }
   if (e == cudaSuccess) {
     launch_rope_table(L->buf.rope_cs, cfg->max_seq, cfg->head_dim, (double)cfg->rope_theta, 0);
     e = cudaGetLastError();
@@ -274,6 +295,8 @@ dare_status_t dare_layer_destroy(dare_layer_t* L) {
   dare_status_t s = check_handle(L);
   if (s != DARE_OK) return s;
   if (L->use_tc) tc_destroy(L);
+  if (L->prof_ev_ready)
+    for (int i = 0; i <= kMaxMarks; ++i) cudaEventDestroy(L->prof_ev[i]);
   L->magic = 0;
   delete L;
   return DARE_OK;
@@ -408,6 +431,52 @@ dare_status_t dare_layer_import_state(dare_layer_t* L, const void* src_host, siz
   L->batch = h.batch;
   L->kv_len = h.kv_len;
   return DARE_OK;
+}
+
+dare_status_t dare_layer_set_profiling(dare_layer_t* L, int enable) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (enable && !L->prof_ev_ready) {
+    for (int i = 0; i <= kMaxMarks; ++i) CUDA_TRY(cudaEventCreate(&L->prof_ev[i]));
+    L->prof_ev_ready = true;
+  }
+  L->prof_on = enable != 0;
+  L->prof_n = 0;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_last_kernel_times(dare_layer_t* L, int32_t* slot_host, float* ms_host, int capacity,
+                                           int* n_out) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!n_out) return DARE_ERR_INVALID_ARG;
+  *n_out = 0;
+  if (!L->prof_on || L->prof_n == 0) return DARE_ERR_STATE;
+  CUDA_TRY(cudaEventSynchronize(L->prof_ev[L->prof_n]));
+  const int n = L->prof_n < capacity ? L->prof_n : capacity;
+  for (int i = 0; i < n; ++i) {
+    float ms = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&ms, L->prof_ev[i], L->prof_ev[i + 1]));
+    if (slot_host) slot_host[i] = L->prof_slot[i];
+    if (ms_host) ms_host[i] = ms;
+  }
+  *n_out = n;
+  return DARE_OK;
+}
+
+const char* dare_kernel_slot_name(int slot) {
+  switch (slot) {
+    case SLOT_NORM: return "rmsnorm";
+    case SLOT_Q_GEMM: return "q_gemm";
+    case SLOT_Q_POST: return "q_post";
+    case SLOT_SELECT: return "select_compact";
+    case SLOT_GATHER: return "gather_rows";
+    case SLOT_KV_GEMM: return "kv_gemm";
+    case SLOT_KV_POST: return "kv_post";
+    case SLOT_ATTN: return "attention";
+    case SLOT_OUT_GEMM: return "out_gemm";
+  }
+  return "?";
 }
 
 int dare_layer_last_launch_count(const dare_layer_t* L) {

@@ -1,0 +1,273 @@
+// Bidirectional (no mask) softmax attention on tcgen05 tensor cores, head_dim = 128, bf16 operands, fp32 softmax.
+//   dense      : every query row of the step window                       (Alg. 1 line 10)
+//   row-sparse : only the query rows of the refresh set, gathered by index (Alg. 2 lines 6, 8; Eq. 4)
+// The result rows are written straight into the attention-output cache at their cache rows; rows that are not
+// computed keep their cached value (Alg. 2 lines 9-10).
+//
+// One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 64:
+//   warp 0       TMA producer: K block and V block of the cache (two 64-column boxes each, 128-byte swizzle),
+//                double buffered
+//   warp 1       one thread issues S = Q K^T (M128 N64 K16 x 8) and O_blk = P V (M128 N128 K16 x 4, V as an MN-major
+//                operand) into tensor memory
+//   warps 2-9    softmax: thread <-> (query row, half): both halves read the row of S from tensor memory and agree on
+//                the running maximum; each exponentiates 32 of the 64 keys, writes them as bf16 into the swizzled
+//                P tile in shared memory, and rescales/accumulates its 64 of the 128 output columns in registers.
+#include "layer.h"
+#include "tc.h"
+#include "tc_ptx.cuh"
+
+namespace dare {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int BQ = 128;    // query rows per CTA
+constexpr int BKV = 64;    // keys per block
+constexpr int HD = 128;
+
+struct AttnSmem {
+  static constexpr int Q_BYTES = BQ * HD * 2;          // two 64-column chunks of [128 x 128 B]
+  static constexpr int K_BYTES = BKV * HD * 2;         // two chunks of [64 x 128 B]
+  static constexpr int V_BYTES = BKV * HD * 2;
+  static constexpr int P_BYTES = BQ * BKV * 2;         // [128 x 128 B]
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = Q_OFF + Q_BYTES;        // 2 buffers
+  static constexpr int V_OFF = K_OFF + 2 * K_BYTES;    // 2 buffers
+  static constexpr int P_OFF = V_OFF + 2 * V_BYTES;
+  static constexpr int L_OFF = P_OFF + P_BYTES;        // float[2][128] partial row sums
+  static constexpr int BAR_OFF = L_OFF + 2 * BQ * 4;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;
+};
+
+constexpr int kThreads = 320;
+constexpr int kSoftmaxThreads = 256;
+constexpr uint32_t kTmemCols = 256;     // S: columns [0, 64), O_blk: columns [64, 192)
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+               const AttnParams p) {
+  using S = AttnSmem;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::BAR_OFF);
+  uint64_t* k_full = bars;          // [2]
+  uint64_t* v_full = bars + 2;      // [2]
+  uint64_t* kv_empty = bars + 4;    // [2]
+  uint64_t* s_full = bars + 6;
+  uint64_t* p_full = bars + 7;
+  uint64_t* o_full = bars + 8;
+  uint64_t* o_free = bars + 9;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  float* l_part = reinterpret_cast<float*>(smem + S::L_OFF);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.y;
+  const StepGeom& g = p.g;
+  const int tps = (g.seq_act + BQ - 1) / BQ;
+  const int b = blockIdx.x / tps, tile = blockIdx.x - b * tps;
+
+  // ---- rows of this tile (uniform over the CTA)
+  int row0, rows_valid;
+  if (p.idx != nullptr) {
+    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
+    row0 = lo + tile * BQ;
+    if (row0 >= hi) return;
+    rows_valid = min(BQ, hi - row0);
+  } else {
+    row0 = b * g.seq_act + tile * BQ;
+    rows_valid = min(BQ, g.seq_act - tile * BQ);
+  }
+  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  const int kv_row0 = b * g.max_seq;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
+    mbar_init(s_full, 1);
+    mbar_init(p_full, kSoftmaxThreads);
+    mbar_init(o_full, 1);
+    mbar_init(o_free, kSoftmaxThreads);
+    fence_mbar_init();
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
+  {
+    uint8_t* qs = smem + S::Q_OFF;
+    for (int u = threadIdx.x; u < BQ * 16; u += kThreads) {
+      const int r = u >> 4, unit = u & 15;           // 16 units of 8 bf16 per row
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (r < rows_valid) {
+        const int t = p.idx ? p.idx[row0 + r] : row0 + r;
+        v = *reinterpret_cast<const uint4*>(p.q + (size_t)t * g.d + h * HD + unit * 8);
+      }
+      const int chunk = unit >> 3, uc = unit & 7;
+      *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + r * 128 + ((uc ^ (r & 7)) << 4)) = v;
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + BKV;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < n_blocks; ++i) {
+        const int buf = i & 1;
+        mbar_wait(&kv_empty[buf], ((i >> 1) & 1) ^ 1, p.status);
+        uint8_t* kd = smem + S::K_OFF + buf * S::K_BYTES;
+        uint8_t* vd = smem + S::V_OFF + buf * S::V_BYTES;
+        const int row = kv_row0 + i * BKV;
+        mbar_arrive_expect_tx(&k_full[buf], S::K_BYTES);
+        tma_load_2d(kd, &tm_k, h * HD, row, &k_full[buf]);
+        tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[buf]);
+        mbar_arrive_expect_tx(&v_full[buf], S::V_BYTES);
+        tma_load_2d(vd, &tm_v, h * HD, row, &v_full[buf]);
+        tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[buf]);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
+      constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
+      const uint32_t q_addr = smem_u32(smem + S::Q_OFF);
+      const uint32_t p_addr = smem_u32(smem + S::P_OFF);
+      auto issue_qk = [&](int i) {
+        const int buf = i & 1;
+        mbar_wait(&k_full[buf], (i >> 1) & 1, p.status);
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(smem + S::K_OFF + buf * S::K_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint64_t a = smem_desc_k_sw128(q_addr + (kk >> 2) * (BQ * 128) + (kk & 3) * 32);
+          const uint64_t bd = smem_desc_k_sw128(k_addr + (kk >> 2) * (BKV * 128) + (kk & 3) * 32);
+          umma_ss(tmem_s, a, bd, idesc_qk, kk != 0 ? 1u : 0u);
+        }
+        umma_commit(s_full);
+      };
+      issue_qk(0);
+      for (int i = 0; i < n_blocks; ++i) {
+        const int buf = i & 1;
+        mbar_wait(p_full, i & 1, p.status);                 // P(i) is in shared memory, S(i) has been read
+        mbar_wait(&v_full[buf], (i >> 1) & 1, p.status);
+        if (i > 0) mbar_wait(o_free, (i - 1) & 1, p.status);  // O_blk(i-1) has been read out of tensor memory
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(smem + S::V_OFF + buf * S::V_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < BKV / 16; ++ks) {
+          const uint64_t a = smem_desc_k_sw128(p_addr + ks * 32);
+          const uint64_t bd = smem_desc_mn_sw128(v_addr + ks * (16 * 128), BKV * 128);
+          umma_ss(tmem_o, a, bd, idesc_pv, ks != 0 ? 1u : 0u);
+        }
+        umma_commit(o_full);
+        umma_commit(&kv_empty[buf]);
+        if (i + 1 < n_blocks) issue_qk(i + 1);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- softmax and output accumulation
+    const int sw = warp - 2;                    // 0..7
+    const int half = sw >> 2;                   // which 32 keys of a block / which 64 output columns
+    const int quarter = warp & 3;               // TMEM lane quarter of this warp
+    const int r = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float c = rsqrtf((float)HD) * 1.4426950408889634f;   // softmax scale folded into the exp2 argument
+    float m = -INFINITY, l = 0.f;
+    float acc[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+    uint8_t* ps = smem + S::P_OFF;
+
+    for (int i = 0; i < n_blocks; ++i) {
+      mbar_wait(s_full, i & 1, p.status);
+      tc_fence_after();
+      float s_mine[32], s_other[32];
+      tmem_ld_32x32(tmem_s + lane_addr + half * 32, s_mine);
+      tmem_ld_32x32(tmem_s + lane_addr + (half ^ 1) * 32, s_other);
+      const int key0 = i * BKV;
+      float mx = m;
+      if (key0 + BKV > g.kv_len) {              // ragged last block: keys past kv_len do not exist
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if (key0 + half * 32 + j >= g.kv_len) s_mine[j] = -INFINITY;
+          if (key0 + (half ^ 1) * 32 + j >= g.kv_len) s_other[j] = -INFINITY;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fmaxf(s_mine[j], s_other[j]));
+      const float alpha = exp2f((m - mx) * c);
+      m = mx;
+      const float mc = mx * c;
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        s_mine[j] = exp2f(fmaf(s_mine[j], c, -mc));
+        sum += s_mine[j];
+      }
+      l = l * alpha + sum;
+      // P row segment: 32 bf16 = 4 sixteen-byte units at the swizzled positions of row r
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const int unit = half * 4 + v;
+        *reinterpret_cast<uint4*>(ps + r * 128 + ((unit ^ (r & 7)) << 4)) = pack8_bf16(s_mine + 8 * v);
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(p_full);
+
+      mbar_wait(o_full, i & 1, p.status);
+      tc_fence_after();
+#pragma unroll
+      for (int cgrp = 0; cgrp < 2; ++cgrp) {
+        float o[32];
+        tmem_ld_32x32(tmem_o + lane_addr + half * 64 + cgrp * 32, o);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha, o[j]);
+      }
+      tc_fence_before();
+      mbar_arrive(o_free);
+    }
+    // ---- combine the two halves' row sums, normalise, store
+    l_part[half * BQ + r] = l;
+    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+    const float inv = 1.f / (l_part[r] + l_part[BQ + r]);
+    if (r < rows_valid) {
+      const int t = p.idx ? p.idx[row0 + r] : row0 + r;
+      __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + half * 64;
+#pragma unroll
+      for (int i = 0; i < 64; ++i) acc[i] *= inv;
+#pragma unroll
+      for (int v = 0; v < 8; ++v) reinterpret_cast<uint4*>(dst)[v] = pack8_bf16(acc + 8 * v);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
+                                cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem::TOTAL);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int tps = (p.g.seq_act + BQ - 1) / BQ;
+  dim3 grid(p.g.batch * tps, p.g.n_heads);
+  if (grid.x == 0) return cudaSuccess;
+  attn_tc_kernel<<<grid, kThreads, AttnSmem::TOTAL, st>>>(tm_k, tm_v, p);
+  return cudaGetLastError();
+}
+
+}  // namespace dare

@@ -28,6 +28,11 @@ struct Buffers {
 
 struct TcState;
 
+// Kernel slots for the optional per-kernel timing.
+enum { SLOT_NORM = 0, SLOT_Q_GEMM, SLOT_Q_POST, SLOT_SELECT, SLOT_GATHER, SLOT_KV_GEMM, SLOT_KV_POST, SLOT_ATTN,
+       SLOT_OUT_GEMM, SLOT_COUNT };
+constexpr int kMaxMarks = 16;
+
 }  // namespace dare
 
 struct dare_layer {
@@ -44,9 +49,26 @@ struct dare_layer {
   int last_launches;
   dare::StepGeom last_geom;
   dare::TcState* tc;
+  // optional per-kernel timing (events recorded between the kernels of a step)
+  bool prof_on;
+  int prof_n;                                  // marks recorded by the last step
+  int prof_slot[dare::kMaxMarks];
+  cudaEvent_t prof_ev[dare::kMaxMarks + 1];
+  bool prof_ev_ready;
 };
 
 namespace dare {
+// Records an event before the kernel that occupies `slot` (no-op unless profiling is on).
+inline void prof_mark(dare_layer* L, int slot, cudaStream_t st) {
+  if (!L->prof_on || L->prof_n >= kMaxMarks) return;
+  L->prof_slot[L->prof_n] = slot;
+  cudaEventRecord(L->prof_ev[L->prof_n], st);
+  ++L->prof_n;
+}
+inline void prof_begin(dare_layer* L) { L->prof_n = 0; }
+inline void prof_end(dare_layer* L, cudaStream_t st) {
+  if (L->prof_on) cudaEventRecord(L->prof_ev[L->prof_n], st);
+}
 dare_status_t tc_create(dare_layer* L);
 void tc_destroy(dare_layer* L);
 dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode, float tau, void* y, cudaStream_t st);

@@ -10,6 +10,7 @@ struct TcState {
   CUtensorMap a_xn, a_xg, a_oc;            // A operands, box 64 x 128
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 64 (two boxes per 128-column tile)
   CUtensorMap w_k32, w_v32;                // weights, box 64 x 32 (two boxes per 64-column tile)
+  CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 64
 };
 
 namespace {
@@ -59,7 +60,8 @@ dare_status_t tc_create(dare_layer* L) {
             make_map(&s->a_oc, L->buf.oc, Tm, d, 128) && make_map(&s->w_q, L->w.w_q, d, d, 64) &&
             make_map(&s->w_k, L->w.w_k, d, d, 64) && make_map(&s->w_v, L->w.w_v, d, d, 64) &&
             make_map(&s->w_o, L->w.w_o, d, d, 64) && make_map(&s->w_k32, L->w.w_k, d, d, 32) &&
-            make_map(&s->w_v32, L->w.w_v, d, d, 32);
+            make_map(&s->w_v32, L->w.w_v, d, d, 32) && make_map(&s->kc64, L->buf.kc, Tm, d, 64) &&
+            make_map(&s->vc64, L->buf.vc, Tm, d, 64);
   if (!ok) { delete s; return DARE_ERR_CUDA; }
   L->tc = s;
   return DARE_OK;
@@ -90,44 +92,59 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.out_is_cache = 0; base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
 
+  prof_begin(L);
   // Alg. 1/2 line 1
+  prof_mark(L, SLOT_NORM, st);
   launch_rmsnorm<bf16>((const bf16*)x, L->w.rms_gain, (bf16*)B.xn, T_, d, L->cfg.rms_eps, st); ++launches;
   // line 2 + line 3 + stored-query update + rotary embedding, one kernel
   {
     GemmParams p = base;
     p.out0 = (bf16*)B.q;
+    prof_mark(L, SLOT_Q_GEMM, st);
     e = launch_gemm_tc(128, EPI_Q, S.a_xn, S.w_q, S.w_q, p, d / 128, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // lines 4-5 + Sec. 4
+  prof_mark(L, SLOT_SELECT, st);
   launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, B.status,
                 st); ++launches;
   // K/V projection with rotary embedding and cache scatter
   if (kv_sparse) {
+    prof_mark(L, SLOT_GATHER, st);
     launch_gather_rows<bf16>((const bf16*)B.xn, B.idx, B.count, (bf16*)B.xg, T_, d, st); ++launches;
     GemmParams p = base;
     p.idx = B.idx; p.count = B.count; p.n_split = d / 64;
     p.out0 = (bf16*)B.kc; p.out1 = (bf16*)B.vc; p.out_is_cache = 1;
+    prof_mark(L, SLOT_KV_GEMM, st);
     e = launch_gemm_tc(64, EPI_KV, S.a_xg, S.w_k32, S.w_v32, p, 2 * d / 64, (T_ + 127) / 128, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   } else {
     GemmParams p = base;
     p.n_split = d / 128;
     p.out0 = (bf16*)B.kc; p.out1 = (bf16*)B.vc; p.out_is_cache = 1;
+    prof_mark(L, SLOT_KV_GEMM, st);
     e = launch_gemm_tc(128, EPI_KV, S.a_xn, S.w_k, S.w_v, p, 2 * d / 128, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // attention (row-sparse over the refresh set when O reuse is on)
-  launch_attention_simt<bf16>((const bf16*)B.q, (const bf16*)B.kc, (const bf16*)B.vc, o_sparse ? B.idx : nullptr,
-                              o_sparse ? B.count : nullptr, (bf16*)B.oc, g, st); ++launches;
+  prof_mark(L, SLOT_ATTN, st);
+  {
+    AttnParams p;
+    p.q = (const bf16*)B.q; p.oc = (bf16*)B.oc; p.idx = o_sparse ? B.idx : nullptr;
+    p.batch_off = o_sparse ? B.batch_off : nullptr; p.g = g; p.status = B.status;
+    e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
+    if (e != cudaSuccess) return DARE_ERR_CUDA;
+  }
   // output projection of every row of the window, read from the O cache
   {
     GemmParams p = base;
     p.a_seq_stride = g.max_seq; p.a_row0 = g.pos_begin; p.hd_map = 128;
     p.out0 = (bf16*)y;
+    prof_mark(L, SLOT_OUT_GEMM, st);
     e = launch_gemm_tc(128, EPI_OUT, S.a_oc, S.w_o, S.w_o, p, d / 128, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
+  prof_end(L, st);
   L->last_launches = launches;
   if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
   return DARE_OK;

@@ -32,6 +32,18 @@ struct GemmParams {
   int* status;
 };
 
+struct AttnParams {
+  const __nv_bfloat16* q;   // [T, d] rotated queries of the step (flat token rows)
+  __nv_bfloat16* oc;        // attention-output cache
+  const int* idx;           // refresh set (row-sparse) or nullptr (all rows)
+  const int* batch_off;     // [batch+1] slice of idx per sequence (row-sparse only)
+  StepGeom g;
+  int* status;
+};
+
+cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
+                                cudaStream_t st);
+
 cudaError_t launch_gemm_tc(int bn, int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                            const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st);
 

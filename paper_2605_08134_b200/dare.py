@@ -58,6 +58,9 @@ def _load():
         "dare_layer_export_state": (C.c_int, [vp, vp, sz, vp]),
         "dare_layer_import_state": (C.c_int, [vp, vp, sz, vp]),
         "dare_layer_last_launch_count": (C.c_int, [vp]),
+        "dare_layer_set_profiling": (C.c_int, [vp, i32]),
+        "dare_layer_last_kernel_times": (C.c_int, [vp, vp, vp, i32, C.POINTER(C.c_int)]),
+        "dare_kernel_slot_name": (C.c_char_p, [C.c_int]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -137,6 +140,21 @@ def dare_layer_import_state(handle, src_ptr, nbytes, stream=0) -> int:
 
 def dare_layer_last_launch_count(handle) -> int:
     return _lib.dare_layer_last_launch_count(handle)
+
+
+def dare_layer_set_profiling(handle, enable: int) -> int:
+    return _lib.dare_layer_set_profiling(handle, enable)
+
+
+def dare_layer_last_kernel_times(handle, slot_ptr, ms_ptr, capacity):
+    """-> (status, n)"""
+    n = C.c_int(0)
+    st = _lib.dare_layer_last_kernel_times(handle, slot_ptr, ms_ptr, capacity, C.byref(n))
+    return st, n.value
+
+
+def dare_kernel_slot_name(slot: int) -> str:
+    return _lib.dare_kernel_slot_name(slot).decode()
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -234,6 +252,21 @@ class Layer:
             raise DareError(st, "dare_layer_read_caches")
         k, v, o = (h.float().numpy() for h in host)
         return {"k": k, "v": v, "o": o, "q_prev": qp}
+
+    def set_profiling(self, enable: bool):
+        st = dare_layer_set_profiling(self.handle, 1 if enable else 0)
+        if st != OK:
+            raise DareError(st, "dare_layer_set_profiling")
+
+    def kernel_times(self):
+        """-> list of (kernel name, milliseconds) of the last step, in launch order (profiling must be on)."""
+        import numpy as np
+        slots = np.zeros(16, np.int32)
+        ms = np.zeros(16, np.float32)
+        st, n = dare_layer_last_kernel_times(self.handle, slots.ctypes.data, ms.ctypes.data, 16)
+        if st != OK:
+            raise DareError(st, "dare_layer_last_kernel_times")
+        return [(dare_kernel_slot_name(int(slots[i])), float(ms[i])) for i in range(n)]
 
     def launch_count(self) -> int:
         return dare_layer_last_launch_count(self.handle)
