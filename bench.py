@@ -97,7 +97,7 @@ def make_inputs(shape, changed_frac, seed, torch, device):
     hs = wl.HiddenStream(shape, seed)
     xa = hs.first()
     n = int(round(changed_frac * shape.seq))
-    changed = wl.uniform_positions(hs.rng, shape, n)
+    changed = wl.uniform_positions(hs.rng, shape, n)      # n positions in every sequence
     xb = hs.advance(changed)
     to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device).to(torch.bfloat16)
     return xa, xb, changed, to(xa), to(xb)
@@ -135,6 +135,11 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
 
     shape = wl.LLADA_LAYER
+    if args.d_model or args.seq or args.batch:      # exploration only: the reported workload is the default one
+        dm = args.d_model or shape.d_model
+        sq = args.seq or shape.seq
+        shape = wl.scaled(shape, name=f"custom_d{dm}_b{args.batch or shape.batch}_s{sq}", d_model=dm,
+                          n_heads=dm // shape.head_dim, seq=sq, prompt=sq // 2, batch=args.batch or shape.batch)
     mode = MODES[args.mode]
     peaks = load_peaks()
     # every rank runs its own replica (sequences are independent: batch sharding, no data-path collective)
@@ -254,7 +259,7 @@ def run_ours(args):
         "q_gemm": ("tensor", 2.0 * T * d * d),
         "out_gemm": ("tensor", 2.0 * T * d * d),
         "kv_gemm": ("hbm", 2.0 * d * d * 2 + 3.0 * n_kv * d * 2) if n_kv <= 215 else ("tensor", 4.0 * n_kv * d * d),
-        "attention": ("tensor", 4.0 * n_o * shape.seq * d),
+        "attention": ("tensor", 4.0 * n_o * shape.seq * d),   # n_o counts rows of all sequences
         "rmsnorm": ("hbm", 2.0 * T * d * 2),
     }
     rows = []
@@ -390,6 +395,9 @@ def main():
     ap.add_argument("--changed", type=float, default=0.13)
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--d-model", type=int, default=0, help="exploration: other layer width (multiple of 128)")
+    ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
+    ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -166,6 +166,15 @@ dare_status_t dare_layer_last_kernel_times(dare_layer_t* layer, int32_t* slot_ho
                                            int* n_out);
 const char* dare_kernel_slot_name(int slot);
 
+/* Diagnostics: when enabled, block (0,0) of each tensor-core kernel of a step writes %globaltimer values (ns) at its
+ * phase boundaries into 64 slots of the workspace: slots [8k, 8k+8) belong to kernel k of the step in the order
+ * Q projection, K/V projection, attention, output projection; within a kernel: start, set-up done, first operand
+ * tile landed, main loop done, epilogue done, ~(earliest block start), latest block end, blocks that ran.  After the
+ * 64 slots come 1024 records (SM id, start, end) of the blocks of the Q projection, by linear block index.
+ * `out_host` (may be NULL, else room for 64 + 3*1024 values) receives the buffer of the last step (the call
+ * synchronises the stream); `enable` switches recording for later steps. */
+dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint64_t* out_host, void* cuda_stream);
+
 /* Number of kernels the last dare_layer_step enqueued (for launch accounting in benchmarks). */
 int dare_layer_last_launch_count(const dare_layer_t* layer);
 

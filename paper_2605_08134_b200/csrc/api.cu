@@ -66,6 +66,7 @@ size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) 
   B.batch_off = (int*)take(((size_t)c->max_batch + 1) * sizeof(int));
   B.count = (int*)take(sizeof(int));
   B.status = (int*)take(sizeof(int));
+  B.debug = (unsigned long long*)take((64 + 3 * 1024) * sizeof(unsigned long long));
   B.x_stage = take(Tm * d * e);
   B.y_stage = take(Tm * d * e);
   if (use_tc) {
@@ -109,7 +110,8 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   launch_gemm_simt<T>((const T*)B.xn, nullptr, nullptr, (const T*)L->w.w_q, B.tmp, T_, d, d, d, st); ++launches;
   // line 3 + stored-query update + rotary embedding
   prof_mark(L, SLOT_Q_POST, st);
-  launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
+  launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g,
+                        L->cfg.max_batch * L->cfg.max_seq, st); ++launches;
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
   prof_mark(L, SLOT_SELECT, st);
   launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, B.status,
@@ -230,6 +232,7 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->prof_on = false;
   L->prof_n = 0;
   L->prof_ev_ready = false;
+  L->debug_on = false;
   memset(&L->last_geom, 0, sizeof(L->last_geom));
   carve(cfg, use_tc, (char*)workspace, &L->buf);
   L->workspace = workspace;
@@ -358,10 +361,20 @@ dare_status_t dare_layer_read_caches(dare_layer_t* L, void* k_host, void* v_host
     if (dst[i])
       CUDA_TRY(cudaMemcpy2DAsync(dst[i], (size_t)L->kv_len * row, src[i], (size_t)L->cfg.max_seq * row,
                                  (size_t)L->kv_len * row, L->batch, cudaMemcpyDeviceToHost, st));
-  if (q_prev_host)
-    CUDA_TRY(cudaMemcpy2DAsync(q_prev_host, (size_t)L->kv_len * hd * 4, L->buf.q_prev, (size_t)L->cfg.max_seq * hd * 4,
-                               (size_t)L->kv_len * hd * 4, L->batch, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
+  if (q_prev_host) {
+    // the device keeps the stored query transposed ([head_dim][cache rows]); hand it out token-major
+    const size_t Tm = (size_t)L->cfg.max_batch * L->cfg.max_seq;
+    float* tmp = new (std::nothrow) float[Tm * hd];
+    if (!tmp) return DARE_ERR_INVALID_ARG;
+    cudaError_t e = cudaMemcpy(tmp, L->buf.q_prev, Tm * hd * sizeof(float), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { delete[] tmp; cudaGetLastError(); return DARE_ERR_CUDA; }
+    for (int b = 0; b < L->batch; ++b)
+      for (int i = 0; i < L->kv_len; ++i)
+        for (size_t j = 0; j < hd; ++j)
+          q_prev_host[((size_t)b * L->kv_len + i) * hd + j] = tmp[j * Tm + (size_t)b * L->cfg.max_seq + i];
+    delete[] tmp;
+  }
   return DARE_OK;
 }
 
@@ -461,6 +474,18 @@ dare_status_t dare_layer_last_kernel_times(dare_layer_t* L, int32_t* slot_host, 
     if (ms_host) ms_host[i] = ms;
   }
   *n_out = n;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_debug_timestamps(dare_layer_t* L, int enable, uint64_t* out_host, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (out_host) {
+    CUDA_TRY(cudaMemcpyAsync(out_host, L->buf.debug, (64 + 3 * 1024) * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+  }
+  L->debug_on = enable != 0;
   return DARE_OK;
 }
 

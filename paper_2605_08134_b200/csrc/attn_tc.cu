@@ -65,6 +65,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.y;
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
   const StepGeom& g = p.g;
   const int tps = (g.seq_act + BQ - 1) / BQ;
   const int b = blockIdx.x / tps, tile = blockIdx.x - b * tps;
@@ -117,6 +119,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + BKV;
+  if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -191,6 +194,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     for (int i = 0; i < n_blocks; ++i) {
       mbar_wait(s_full, i & 1, p.status);
       tc_fence_after();
+      if (dbg && i == 0 && threadIdx.x == 64) p.debug[2] = globaltimer_ns();
       float s_mine[32], s_other[32];
       tmem_ld_32x32(tmem_s + lane_addr + half * 32, s_mine);
       tmem_ld_32x32(tmem_s + lane_addr + (half ^ 1) * 32, s_other);
@@ -237,6 +241,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       tc_fence_before();
       mbar_arrive(o_free);
     }
+    if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
     // ---- combine the two halves' row sums, normalise, store
     l_part[half * BQ + r] = l;
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
@@ -252,6 +257,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
+  if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 

@@ -4,7 +4,8 @@
 namespace dare {
 
 // ------------------------------------------------------------------------------------------------ rotary table
-// cs[pos][j] = (cos, sin)(pos * theta^(-2j/head_dim)), evaluated in fp64 and stored as fp32.
+// cs[j][pos] = (cos, sin)(pos * theta^(-2j/head_dim)), evaluated in fp64 and stored as fp32.  Pair index major, so
+// that the threads of a tile (consecutive positions) read consecutive addresses.
 __global__ void rope_table_kernel(float2* cs, int max_seq, int half, double theta, int head_dim) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= max_seq * half) return;
@@ -12,7 +13,7 @@ __global__ void rope_table_kernel(float2* cs, int max_seq, int half, double thet
   double inv_freq = pow(theta, -2.0 * (double)j / (double)head_dim);
   double s, c;
   sincos((double)pos * inv_freq, &s, &c);
-  cs[i] = make_float2((float)c, (float)s);
+  cs[(size_t)j * max_seq + pos] = make_float2((float)c, (float)s);
 }
 
 void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaStream_t st) {

@@ -51,7 +51,7 @@ void launch_gemm_simt(const T* a, const int* a_idx, const int* count, const T* w
 // store Q in the layer dtype.
 template <typename T>
 void launch_q_post_simt(const float* qf, int ldq, const float* rope_cs, float* q_prev, float* scores, bool has_prev,
-                        T* q, const StepGeom& g, cudaStream_t st);
+                        T* q, const StepGeom& g, int q_rows, cudaStream_t st);
 // K/V post-pass: rows r < *count (or all when idx == nullptr): rotary embedding on K, store K and V to cache rows.
 template <typename T>
 void launch_kv_post_simt(const float* kvf, int ld, const int* idx, const int* count, const float* rope_cs, T* kc,

@@ -25,7 +25,7 @@ struct GemmSmem {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 128) ? 6 : 8;
+  static constexpr int STAGES = (BN == 256) ? 4 : ((BN == 128) ? 6 : 8);
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
 };
@@ -45,6 +45,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = blockIdx.x, mt = blockIdx.y;
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
+  const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+  if (EPI == EPI_Q && p.debug != nullptr && threadIdx.x == 0 && lin < 1024) {
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    p.debug[64 + 3 * lin] = smid;
+    p.debug[64 + 3 * lin + 1] = globaltimer_ns();
+  }
 
   // ---- which rows does this tile cover? (uniform over the CTA; a tile past the refresh set leaves at once)
   int a_row, t0, rows_valid;
@@ -84,6 +93,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int KB = p.K / 64;
+  // Each CTA walks the reduction dimension from its own starting block, so that the CTAs sharing an operand tile
+  // do not all ask the L2 for the same lines at the same moment.
+  const int k_rot = (int)((nt * p.rot_n + mt * p.rot_m) % KB);
+  if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -93,9 +106,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint8_t* a_dst = smem + s * S::STAGE_BYTES;
         uint8_t* b_dst = a_dst + S::A_BYTES;
         mbar_arrive_expect_tx(&full_bar[s], S::STAGE_BYTES);
-        tma_load_2d(a_dst, &tm_a, kb * 64, a_row, &full_bar[s]);
-        tma_load_2d(b_dst, tm_b, kb * 64, col_lo, &full_bar[s]);
-        tma_load_2d(b_dst + S::B_BYTES / 2, tm_b, kb * 64, col_hi, &full_bar[s]);
+        int kx = kb + k_rot;
+        if (kx >= KB) kx -= KB;
+        tma_load_2d(a_dst, &tm_a, kx * 64, a_row, &full_bar[s]);
+        if (p.b_single) {                       // both column halves are adjacent rows of W: one box
+          tma_load_2d(b_dst, tm_b, kx * 64, col_lo, &full_bar[s]);
+        } else {
+          tma_load_2d(b_dst, tm_b, kx * 64, col_lo, &full_bar[s]);
+          tma_load_2d(b_dst + S::B_BYTES / 2, tm_b, kx * 64, col_hi, &full_bar[s]);
+        }
       }
     }
     __syncwarp();
@@ -106,9 +125,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int s = kb % STAGES;
         mbar_wait(&full_bar[s], (kb / STAGES) & 1, p.status);
         tc_fence_after();
+        if (dbg && kb == 0) p.debug[2] = globaltimer_ns();
         const uint32_t a_addr = smem_u32(smem + s * S::STAGE_BYTES);
         const uint64_t a_desc = smem_desc_k_sw128(a_addr);
         const uint64_t b_desc = smem_desc_k_sw128(a_addr + S::A_BYTES);
+        for (int rep = 0; rep < p.mma_rep; ++rep)
 #pragma unroll
         for (int k = 0; k < 4; ++k)  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
           umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
@@ -121,6 +142,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // ---- epilogue: thread <-> output row
     mbar_wait(accum_bar, 0, p.status);
     tc_fence_after();
+    if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
     const int quarter = warp & 3;               // TMEM lanes this warp may touch: 32*quarter .. +31
     const int r = quarter * 32 + lane;
     const bool valid = r < rows_valid;
@@ -133,74 +155,92 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     constexpr int HALF_W = BN / 2;
     const bool is_b1 = nt >= p.n_split;
 
+    constexpr int ROW_BYTES = BN * 2;            // one staged output row (bf16)
+    constexpr int UNITS = ROW_BYTES / 16;        // 16-byte units per staged row
+    // The operand ring is idle once the accumulator is complete: its first 128 x ROW_BYTES bytes stage the tile so
+    // that the global stores below are whole contiguous row segments.
+    uint8_t* stg = smem;
+    const size_t tm_rows = (size_t)p.q_prev_rows;  // row count of the transposed stored-query array
+    const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
+    const bool score_tile = (EPI == EPI_Q) && head == p.g.score_head;
+
     float dot = 0.f, n1 = 0.f, n2 = 0.f;
 #pragma unroll 1
     for (int c = 0; c < NCH; ++c) {
       float lo[32], hi[32];
       tmem_ld_32x32(t_lane + c * 32, lo);
       tmem_ld_32x32(t_lane + HALF_W + c * 32, hi);
-      if (!valid) continue;
       const int j0 = jb * HALF_W + c * 32;       // index of lo[0] inside the head (rotary pair index)
-      if (EPI == EPI_Q) {
-        if (head == p.g.score_head) {
-          float* qp = p.q_prev + crow * p.g.head_dim;
+      if (valid) {
+        if (score_tile) {
+          // stored query, transposed [head_dim][cache rows]: consecutive rows of a tile are consecutive addresses
+          float* qa = p.q_prev + (size_t)j0 * tm_rows + crow;
+          float* qb = p.q_prev + (size_t)(p.g.head_dim / 2 + j0) * tm_rows + crow;
           if (p.has_prev) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              const float4 a = *reinterpret_cast<const float4*>(qp + j0 + i);
-              const float4 b = *reinterpret_cast<const float4*>(qp + p.g.head_dim / 2 + j0 + i);
-              dot = fmaf(lo[i], a.x, dot); dot = fmaf(lo[i + 1], a.y, dot);
-              dot = fmaf(lo[i + 2], a.z, dot); dot = fmaf(lo[i + 3], a.w, dot);
-              dot = fmaf(hi[i], b.x, dot); dot = fmaf(hi[i + 1], b.y, dot);
-              dot = fmaf(hi[i + 2], b.z, dot); dot = fmaf(hi[i + 3], b.w, dot);
-              n2 = fmaf(a.x, a.x, n2); n2 = fmaf(a.y, a.y, n2); n2 = fmaf(a.z, a.z, n2); n2 = fmaf(a.w, a.w, n2);
-              n2 = fmaf(b.x, b.x, n2); n2 = fmaf(b.y, b.y, n2); n2 = fmaf(b.z, b.z, n2); n2 = fmaf(b.w, b.w, n2);
+            for (int i = 0; i < 32; ++i) {
+              const float a = qa[(size_t)i * tm_rows], b = qb[(size_t)i * tm_rows];
+              dot = fmaf(lo[i], a, dot); dot = fmaf(hi[i], b, dot);
+              n2 = fmaf(a, a, n2); n2 = fmaf(b, b, n2);
+              n1 = fmaf(lo[i], lo[i], n1); n1 = fmaf(hi[i], hi[i], n1);
             }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) { n1 = fmaf(lo[i], lo[i], n1); n1 = fmaf(hi[i], hi[i], n1); }
           }
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            *reinterpret_cast<float4*>(qp + j0 + i) = make_float4(lo[i], lo[i + 1], lo[i + 2], lo[i + 3]);
-            *reinterpret_cast<float4*>(qp + p.g.head_dim / 2 + j0 + i) =
-                make_float4(hi[i], hi[i + 1], hi[i + 2], hi[i + 3]);
+          for (int i = 0; i < 32; ++i) { qa[(size_t)i * tm_rows] = lo[i]; qb[(size_t)i * tm_rows] = hi[i]; }
+        }
+        if (rotate) {
+          // rotary table, transposed [pair index][position]
+          const float2* cs = p.rope + (size_t)j0 * p.g.max_seq + pos;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float2 cv = cs[(size_t)i * p.g.max_seq];
+            const float a0 = lo[i], b0 = hi[i];
+            lo[i] = a0 * cv.x - b0 * cv.y;
+            hi[i] = a0 * cv.y + b0 * cv.x;
           }
         }
       }
-      const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
-      if (rotate) {
-        const float2* cs = p.rope + (size_t)pos * (p.g.head_dim / 2) + j0;
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float4 c2 = *reinterpret_cast<const float4*>(cs + i);   // (cos, sin) of two consecutive pairs
-          const float a0 = lo[i], b0 = hi[i], a1 = lo[i + 1], b1 = hi[i + 1];
-          lo[i] = a0 * c2.x - b0 * c2.y;  hi[i] = a0 * c2.y + b0 * c2.x;
-          lo[i + 1] = a1 * c2.z - b1 * c2.w;  hi[i + 1] = a1 * c2.w + b1 * c2.z;
-        }
+      for (int v = 0; v < 4; ++v) {
+        const int u_lo = c * 4 + v, u_hi = UNITS / 2 + c * 4 + v;
+        *reinterpret_cast<uint4*>(stg + r * ROW_BYTES + ((u_lo ^ (r & (UNITS - 1))) << 4)) = pack8_bf16(lo + 8 * v);
+        *reinterpret_cast<uint4*>(stg + r * ROW_BYTES + ((u_hi ^ (r & (UNITS - 1))) << 4)) = pack8_bf16(hi + 8 * v);
       }
-      __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
-      const size_t orow = p.out_is_cache ? crow : (size_t)t;
-      __nv_bfloat16* dst = out + orow * p.ld_out;
-      uint4* d_lo = reinterpret_cast<uint4*>(dst + col_lo + c * 32);
-      uint4* d_hi = reinterpret_cast<uint4*>(dst + col_hi + c * 32);
-#pragma unroll
-      for (int v = 0; v < 4; ++v) { d_lo[v] = pack8_bf16(lo + 8 * v); d_hi[v] = pack8_bf16(hi + 8 * v); }
     }
-    if (EPI == EPI_Q) {
-      if (valid && head == p.g.score_head) {
-        float s;
-        if (p.has_prev) {
-          const float den = sqrtf(n1) * sqrtf(n2);
-          s = 1.f - (den > 0.f ? dot / den : 0.f);
-        } else {
-          s = __int_as_float(0x7f800000);
-        }
-        p.scores[t] = s;
+    if (score_tile && valid) {
+      float sc;
+      if (p.has_prev) {
+        const float den = sqrtf(n1) * sqrtf(n2);
+        sc = 1.f - (den > 0.f ? dot / den : 0.f);
+      } else {
+        sc = __int_as_float(0x7f800000);
+      }
+      p.scores[t] = sc;
+    }
+    __syncwarp();
+    if (dbg && threadIdx.x == 64) p.debug[4] = globaltimer_ns();
+    // ---- write-out: each warp stores its own 32 rows, UNITS lanes per row
+    {
+      __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
+      const long long my_orow = valid ? (long long)(p.out_is_cache ? crow : (size_t)t) : -1;
+      constexpr int ROWS_PER_IT = 32 / UNITS;
+      const int unit = lane % UNITS;
+      const int col = unit < UNITS / 2 ? col_lo + unit * 8 : col_hi + (unit - UNITS / 2) * 8;
+#pragma unroll
+      for (int rr = 0; rr < 32; rr += ROWS_PER_IT) {
+        const int row_l = rr + lane / UNITS;
+        const long long orow = __shfl_sync(0xffffffffu, my_orow, row_l);
+        const int R = quarter * 32 + row_l;
+        const uint4 v = *reinterpret_cast<const uint4*>(stg + R * ROW_BYTES + ((unit ^ (R & (UNITS - 1))) << 4));
+        if (orow >= 0) *reinterpret_cast<uint4*>(out + (size_t)orow * p.ld_out + col) = v;
       }
     }
   }
+  if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
   tc_fence_before();
   __syncthreads();
+  if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
+  if (EPI == EPI_Q && p.debug != nullptr && threadIdx.x == 0 && lin < 1024) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
   if (warp == 1) tmem_dealloc(tmem_base, BN < 32 ? 32 : BN);
 }
 
@@ -227,6 +267,7 @@ cudaError_t launch_gemm_tc(int bn, int epi, const CUtensorMap& a, const CUtensor
     if (epi == EPI_KV) return launch_one<128, EPI_KV>(a, b0, b1, p, n_tiles, m_tiles, st);
     return launch_one<128, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
   }
+  if (bn == 256 && epi == EPI_OUT) return launch_one<256, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
   if (bn == 64) {
     if (epi == EPI_KV) return launch_one<64, EPI_KV>(a, b0, b1, p, n_tiles, m_tiles, st);
     if (epi == EPI_OUT) return launch_one<64, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);

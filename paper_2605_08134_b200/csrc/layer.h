@@ -7,19 +7,20 @@ namespace dare {
 
 // Device buffers carved from the caller's workspace.
 struct Buffers {
-  float* rope_cs;   // [max_seq, head_dim/2] (cos, sin)
+  float* rope_cs;   // [head_dim/2, max_seq] (cos, sin), pair index major
   void* xn;         // [T, d]  normalised hidden states (layer dtype)
   void* q;          // [T, d]  rotated queries (layer dtype)
   void* kc;         // [max_batch*max_seq, d] K cache (rotated)
   void* vc;         // [max_batch*max_seq, d] V cache
   void* oc;         // [max_batch*max_seq, d] attention-output cache (before W_O)
-  float* q_prev;    // [max_batch*max_seq, head_dim] un-rotated scoring-head query of the previous step, fp32
+  float* q_prev;    // [head_dim, max_batch*max_seq] un-rotated scoring-head query of the previous step, fp32
   float* scores;    // [T]
   int* idx;         // [T] refresh set, ascending
   int* delta;       // [max_batch*max_seq] staleness counters
   int* batch_off;   // [max_batch+1]
   int* count;       // [1]
   int* status;      // [1] device status word
+  unsigned long long* debug;  // [64] kernel phase timestamps (diagnostics, written by block (0,0) when enabled)
   void* x_stage;    // [T, d] staging for the host-buffer entry point
   void* y_stage;
   void* xg;         // tensor-core path: gathered x_norm rows
@@ -55,6 +56,7 @@ struct dare_layer {
   int prof_slot[dare::kMaxMarks];
   cudaEvent_t prof_ev[dare::kMaxMarks + 1];
   bool prof_ev_ready;
+  bool debug_on;
 };
 
 namespace dare {

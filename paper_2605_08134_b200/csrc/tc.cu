@@ -1,5 +1,6 @@
 // Host side of the tensor-core path: TMA tensor maps and the per-step kernel sequence.
 #include <new>
+#include <stdlib.h>
 
 #include "layer.h"
 #include "tc.h"
@@ -10,6 +11,7 @@ struct TcState {
   CUtensorMap a_xn, a_xg, a_oc;            // A operands, box 64 x 128
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 64 (two boxes per 128-column tile)
   CUtensorMap w_k32, w_v32;                // weights, box 64 x 32 (two boxes per 64-column tile)
+  CUtensorMap w_o128;                      // experiment: box 64 x 128
   CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 64
 };
 
@@ -61,7 +63,7 @@ dare_status_t tc_create(dare_layer* L) {
             make_map(&s->w_k, L->w.w_k, d, d, 64) && make_map(&s->w_v, L->w.w_v, d, d, 64) &&
             make_map(&s->w_o, L->w.w_o, d, d, 64) && make_map(&s->w_k32, L->w.w_k, d, d, 32) &&
             make_map(&s->w_v32, L->w.w_v, d, d, 32) && make_map(&s->kc64, L->buf.kc, Tm, d, 64) &&
-            make_map(&s->vc64, L->buf.vc, Tm, d, 64);
+            make_map(&s->vc64, L->buf.vc, Tm, d, 64) && make_map(&s->w_o128, L->w.w_o, d, d, 128);
   if (!ok) { delete s; return DARE_ERR_CUDA; }
   L->tc = s;
   return DARE_OK;
@@ -86,11 +88,21 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   cudaError_t e;
 
   GemmParams base;
+  static const int rot_n = getenv("DARE_ROT_N") ? atoi(getenv("DARE_ROT_N")) : 0;
+  static const int rot_m = getenv("DARE_ROT_M") ? atoi(getenv("DARE_ROT_M")) : 0;
+  base.rot_n = rot_n; base.rot_m = rot_m; base.b_single = 0;
+  static const int mma_rep = getenv("DARE_MMA_REP") ? atoi(getenv("DARE_MMA_REP")) : 1;
+  base.mma_rep = mma_rep;
+  static const int single = getenv("DARE_B_SINGLE") ? atoi(getenv("DARE_B_SINGLE")) : 0;
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
   base.hd_map = g.head_dim; base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
   base.out_is_cache = 0; base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
+  base.q_prev_rows = L->cfg.max_batch * L->cfg.max_seq;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
+  base.debug = nullptr;
+  unsigned long long* dbg = L->debug_on ? B.debug : nullptr;
+  if (dbg) cudaMemsetAsync(dbg, 0, (64 + 3 * 1024) * sizeof(unsigned long long), st);
 
   prof_begin(L);
   // Alg. 1/2 line 1
@@ -100,6 +112,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   {
     GemmParams p = base;
     p.out0 = (bf16*)B.q;
+    p.debug = dbg;
     prof_mark(L, SLOT_Q_GEMM, st);
     e = launch_gemm_tc(128, EPI_Q, S.a_xn, S.w_q, S.w_q, p, d / 128, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
@@ -115,6 +128,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     GemmParams p = base;
     p.idx = B.idx; p.count = B.count; p.n_split = d / 64;
     p.out0 = (bf16*)B.kc; p.out1 = (bf16*)B.vc; p.out_is_cache = 1;
+    p.debug = dbg ? dbg + 8 : nullptr;
     prof_mark(L, SLOT_KV_GEMM, st);
     e = launch_gemm_tc(64, EPI_KV, S.a_xg, S.w_k32, S.w_v32, p, 2 * d / 64, (T_ + 127) / 128, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
@@ -122,6 +136,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     GemmParams p = base;
     p.n_split = d / 128;
     p.out0 = (bf16*)B.kc; p.out1 = (bf16*)B.vc; p.out_is_cache = 1;
+    p.debug = dbg ? dbg + 8 : nullptr;
     prof_mark(L, SLOT_KV_GEMM, st);
     e = launch_gemm_tc(128, EPI_KV, S.a_xn, S.w_k, S.w_v, p, 2 * d / 128, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
@@ -132,16 +147,20 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     AttnParams p;
     p.q = (const bf16*)B.q; p.oc = (bf16*)B.oc; p.idx = o_sparse ? B.idx : nullptr;
     p.batch_off = o_sparse ? B.batch_off : nullptr; p.g = g; p.status = B.status;
+    p.debug = dbg ? dbg + 16 : nullptr;
     e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // output projection of every row of the window, read from the O cache
   {
     GemmParams p = base;
-    p.a_seq_stride = g.max_seq; p.a_row0 = g.pos_begin; p.hd_map = 128;
+    static const int out_bn = getenv("DARE_OUT_BN") ? atoi(getenv("DARE_OUT_BN")) : 128;
+    p.a_seq_stride = g.max_seq; p.a_row0 = g.pos_begin; p.hd_map = out_bn;
     p.out0 = (bf16*)y;
+    p.debug = dbg ? dbg + 24 : nullptr;
     prof_mark(L, SLOT_OUT_GEMM, st);
-    e = launch_gemm_tc(128, EPI_OUT, S.a_oc, S.w_o, S.w_o, p, d / 128, m_tiles_dense, st); ++launches;
+    p.b_single = (single && out_bn == 128) ? 1 : 0;
+    e = launch_gemm_tc(out_bn, EPI_OUT, S.a_oc, (out_bn == 256 || p.b_single) ? S.w_o128 : S.w_o, S.w_o, p, d / out_bn, m_tiles_dense, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   prof_end(L, st);

@@ -11,6 +11,9 @@ enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2 };
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
+  int mma_rep;           // timing experiment only: issue every MMA this many times (1 = normal)
+  int b_single;          // the W tile is one TMA box of BN rows (column halves adjacent) instead of two of BN/2
+  int rot_n, rot_m;      // per-tile rotation of the starting reduction block (in blocks per n-tile / m-tile)
   int m_total;           // dense: tokens of the step; gathered: capacity of the row list
   int seq_act;           // dense row mapping: rows per sequence ...
   int tiles_per_seq;     // ... and 128-row tiles per sequence
@@ -25,11 +28,13 @@ struct GemmParams {
   __nv_bfloat16* out1;
   int ld_out;
   int out_is_cache;      // output rows addressed by cache row (1) or by flat token index (0)
-  const float2* rope;
-  float* q_prev;
+  const float2* rope;    // rotary table, transposed: [head_dim/2][max_seq]
+  float* q_prev;         // stored scoring-head query, transposed: [head_dim][q_prev_rows]
+  int q_prev_rows;       // = max_batch * max_seq
   float* scores;
   int has_prev;
   int* status;
+  unsigned long long* debug;   // 8 timestamp slots of this kernel or nullptr
 };
 
 struct AttnParams {
@@ -39,6 +44,7 @@ struct AttnParams {
   const int* batch_off;     // [batch+1] slice of idx per sequence (row-sparse only)
   StepGeom g;
   int* status;
+  unsigned long long* debug;
 };
 
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,

@@ -61,6 +61,7 @@ def _load():
         "dare_layer_set_profiling": (C.c_int, [vp, i32]),
         "dare_layer_last_kernel_times": (C.c_int, [vp, vp, vp, i32, C.POINTER(C.c_int)]),
         "dare_kernel_slot_name": (C.c_char_p, [C.c_int]),
+        "dare_layer_debug_timestamps": (C.c_int, [vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -151,6 +152,10 @@ def dare_layer_last_kernel_times(handle, slot_ptr, ms_ptr, capacity):
     n = C.c_int(0)
     st = _lib.dare_layer_last_kernel_times(handle, slot_ptr, ms_ptr, capacity, C.byref(n))
     return st, n.value
+
+
+def dare_layer_debug_timestamps(handle, enable, out_ptr, stream=0) -> int:
+    return _lib.dare_layer_debug_timestamps(handle, enable, out_ptr, stream)
 
 
 def dare_kernel_slot_name(slot: int) -> str:
@@ -267,6 +272,16 @@ class Layer:
         if st != OK:
             raise DareError(st, "dare_layer_last_kernel_times")
         return [(dare_kernel_slot_name(int(slots[i])), float(ms[i])) for i in range(n)]
+
+    def debug_timestamps(self, enable=True):
+        """-> uint64[8, 8] phase timestamps (ns) of the tensor-core kernels of the last step; see include/dare.h."""
+        import numpy as np
+        out = np.zeros(64 + 3 * 1024, np.uint64)
+        st = dare_layer_debug_timestamps(self.handle, 1 if enable else 0, out.ctypes.data, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_debug_timestamps")
+        self.debug_blocks = out[64:].reshape(1024, 3)
+        return out[:64].reshape(8, 8)
 
     def launch_count(self) -> int:
         return dare_layer_last_launch_count(self.handle)
