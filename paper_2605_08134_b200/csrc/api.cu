@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include "layer.h"
+#include "tc.h"
 
 using namespace dare;
 
@@ -110,12 +111,11 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   launch_gemm_simt<T>((const T*)B.xn, nullptr, nullptr, (const T*)L->w.w_q, B.tmp, T_, d, d, d, st); ++launches;
   // line 3 + stored-query update + rotary embedding
   prof_mark(L, SLOT_Q_POST, st);
-  launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g,
-                        L->cfg.max_batch * L->cfg.max_seq, st); ++launches;
+  launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
   prof_mark(L, SLOT_SELECT, st);
-  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, B.status,
-                st); ++launches;
+  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, nullptr,
+                nullptr, 0, st); ++launches;
   // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
   const int* kv_idx = kv_sparse ? B.idx : nullptr;
   const int* kv_cnt = kv_sparse ? B.count : nullptr;
@@ -361,20 +361,10 @@ dare_status_t dare_layer_read_caches(dare_layer_t* L, void* k_host, void* v_host
     if (dst[i])
       CUDA_TRY(cudaMemcpy2DAsync(dst[i], (size_t)L->kv_len * row, src[i], (size_t)L->cfg.max_seq * row,
                                  (size_t)L->kv_len * row, L->batch, cudaMemcpyDeviceToHost, st));
+  if (q_prev_host)
+    CUDA_TRY(cudaMemcpy2DAsync(q_prev_host, (size_t)L->kv_len * hd * 4, L->buf.q_prev, (size_t)L->cfg.max_seq * hd * 4,
+                               (size_t)L->kv_len * hd * 4, L->batch, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
-  if (q_prev_host) {
-    // the device keeps the stored query transposed ([head_dim][cache rows]); hand it out token-major
-    const size_t Tm = (size_t)L->cfg.max_batch * L->cfg.max_seq;
-    float* tmp = new (std::nothrow) float[Tm * hd];
-    if (!tmp) return DARE_ERR_INVALID_ARG;
-    cudaError_t e = cudaMemcpy(tmp, L->buf.q_prev, Tm * hd * sizeof(float), cudaMemcpyDeviceToHost);
-    if (e != cudaSuccess) { delete[] tmp; cudaGetLastError(); return DARE_ERR_CUDA; }
-    for (int b = 0; b < L->batch; ++b)
-      for (int i = 0; i < L->kv_len; ++i)
-        for (size_t j = 0; j < hd; ++j)
-          q_prev_host[((size_t)b * L->kv_len + i) * hd + j] = tmp[j * Tm + (size_t)b * L->cfg.max_seq + i];
-    delete[] tmp;
-  }
   return DARE_OK;
 }
 

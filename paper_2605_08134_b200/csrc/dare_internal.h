@@ -36,8 +36,10 @@ void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaS
 template <typename T>
 void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st);
 // Threshold + ballot/prefix-sum compaction + staleness update.  `scores == nullptr` or `select_all` selects all.
+// With gather_dst != nullptr the rows src[idx[r]] (row_bytes each, multiple of 16) are also copied to dst[r].
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, int* status, cudaStream_t st);
+                   int* batch_off, int* delta, const void* gather_src, void* gather_dst, int row_bytes,
+                   cudaStream_t st);
 template <typename T>
 void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
 
@@ -51,7 +53,7 @@ void launch_gemm_simt(const T* a, const int* a_idx, const int* count, const T* w
 // store Q in the layer dtype.
 template <typename T>
 void launch_q_post_simt(const float* qf, int ldq, const float* rope_cs, float* q_prev, float* scores, bool has_prev,
-                        T* q, const StepGeom& g, int q_rows, cudaStream_t st);
+                        T* q, const StepGeom& g, cudaStream_t st);
 // K/V post-pass: rows r < *count (or all when idx == nullptr): rotary embedding on K, store K and V to cache rows.
 template <typename T>
 void launch_kv_post_simt(const float* kvf, int ld, const int* idx, const int* count, const float* rope_cs, T* kc,

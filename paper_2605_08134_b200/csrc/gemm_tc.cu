@@ -1,16 +1,23 @@
 // bf16 projection GEMMs on the 5th-generation tensor cores: C[m, n] = sum_k A[m, k] * W[n, k]  (W = [out, in],
-// Alg. 1 lines 2, 7, 11).  One 128 x BN output tile per CTA:
-//   warp 0    TMA producer: A and W tiles (64 k-elements = 128 bytes per row, 128-byte swizzle) into a ring of stages
-//   warp 1    allocates tensor memory, one thread issues tcgen05.mma (M = 128, N = BN, K = 16) into fp32 accumulators
-//             and commits each stage back to the producer
-//   warps 2-5 epilogue: each thread owns one output row (one TMEM lane), reads it with tcgen05.ld and applies the
-//             fused tail of that projection:
-//               Q    drift score of the scoring head against the stored query (Sec. 3.1), store of the new query,
-//                    rotary embedding, bf16 store
-//               K/V  rotary embedding of K, scatter of both rows into the caches at the refresh-set rows (Eq. 3)
-//               OUT  plain bf16 store of y
-// Column mapping of a tile: BN/2 columns starting at `lo` and BN/2 columns starting at `lo + head_dim/2` of one head,
-// so that both elements of every rotary pair sit in the same thread.
+// Alg. 1 lines 2, 7, 11).  One CTA = one 128 x 256 output tile over one slice of the reduction dimension:
+//   warp 0    TMA producer: a 128-row A tile and a 256-row W tile per 64 k-elements (128 bytes per row, 128-byte
+//             swizzle) into a ring of 4 stages
+//   warp 1    allocates tensor memory; one thread issues tcgen05.mma (M = 128, N = 256, K = 16: a single-CTA MMA
+//             costs about the same time whatever its N, so only the widest N runs the tensor pipe at full rate)
+//             into a 128 x 256 fp32 accumulator and commits each stage back to the producer
+//   warps 2-5 epilogue: each thread owns one output row (one TMEM lane)
+// Split-K: when a launch has too few tiles to fill the GPU, the two CTAs of a thread-block cluster share a tile, each
+// over half of the reduction.  Every CTA first moves its fp32 accumulator from tensor memory into its own shared
+// memory (the operand ring is idle by then).  The halves are then combined by a reduce-scatter over distributed
+// shared memory: CTA k owns 64 rows of the tile and receives the partner's partial of those rows by one bulk copy
+// per warp (32 KB, completion counted on an mbarrier of the receiver).  Each CTA finishes the rows it owns with all
+// of its warps: one warp per row, lane <-> column pairs, so that table reads and output stores are contiguous.
+// The fused epilogue work is thereby spread over both CTAs as well.
+// Fused epilogues:
+//   Q    drift score of the scoring head against the stored query (Sec. 3.1), store of the new query, rotary
+//        embedding, bf16 store
+//   K/V  rotary embedding of K, scatter of both rows into the caches at the refresh-set rows (Eq. 3)
+//   OUT  plain bf16 store of y
 #include "layer.h"
 #include "tc.h"
 #include "tc_ptx.cuh"
@@ -19,259 +26,334 @@ namespace dare {
 
 using namespace ptx;
 
+namespace {
+constexpr int BM = 128, BK = 64;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int HD = 128;                              // head width the rotary/score epilogues assume
 template <int BN>
-struct GemmSmem {
-  static constexpr int BM = 128, BK = 64;
-  static constexpr int A_BYTES = BM * BK * 2;
+struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 256) ? 4 : ((BN == 128) ? 6 : 8);
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-  static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
+  static constexpr int SMEM_TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
+  static constexpr int PROW_BYTES = BN * 4;
+  static constexpr int RECV_OFFSET = BM * PROW_BYTES;
 };
+// After the main loop the ring is reused: [0, 128 KB) this CTA's fp32 partial tile, [row][256 columns], 1 KB per row,
+// the 16-byte units of a row XOR-swizzled with the row index (bank-conflict-free for row-per-thread writes and for
+// row-per-warp reads); [128 KB, 192 KB) the partner's partial of the 64 rows this CTA owns (split-K only).
+}  // namespace
 
-template <int BN, int EPI>
+template <int EPI, int BN>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
-  using S = GemmSmem<BN>;
-  constexpr int STAGES = S::STAGES;
+  constexpr int STAGES = Cfg<BN>::STAGES, STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
+  constexpr int PROW_BYTES = Cfg<BN>::PROW_BYTES, RECV_OFFSET = Cfg<BN>::RECV_OFFSET;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S::BAR_OFFSET);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg<BN>::BAR_OFFSET);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* accum_bar = empty_bar + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_bar + 1);
+  uint64_t* recv_bar = accum_bar + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(recv_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = blockIdx.x, mt = blockIdx.y;
-  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  const int splits = gridDim.z;                 // = cluster size along z
+  const int z = (int)cluster_ctarank();
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  const int lin = blockIdx.y * gridDim.x + blockIdx.x;
-  if (EPI == EPI_Q && p.debug != nullptr && threadIdx.x == 0 && lin < 1024) {
-    unsigned smid;
-    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    p.debug[64 + 3 * lin] = smid;
-    p.debug[64 + 3 * lin + 1] = globaltimer_ns();
-  }
+  const int lin = (z * gridDim.y + mt) * gridDim.x + nt;
+  const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
+  if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
-  // ---- which rows does this tile cover? (uniform over the CTA; a tile past the refresh set leaves at once)
+  // ---- which rows does this tile cover? (uniform over the cluster; a tile past the refresh set leaves at once)
   int a_row, t0, rows_valid;
+  int pos0 = 0;          // dense tiles: position and cache row of the tile's first row
+  size_t crow0 = 0;
   if (p.count != nullptr) {
     const int n = min(*p.count, p.m_total);
-    t0 = mt * 128;
+    t0 = mt * BM;
     if (t0 >= n) return;
-    rows_valid = min(128, n - t0);
+    rows_valid = min(BM, n - t0);
     a_row = t0;
   } else {
     const int b = mt / p.tiles_per_seq, tis = mt - b * p.tiles_per_seq;
-    t0 = b * p.seq_act + tis * 128;
-    rows_valid = min(128, p.seq_act - tis * 128);
-    a_row = b * p.a_seq_stride + p.a_row0 + tis * 128;
+    t0 = b * p.seq_act + tis * BM;
+    rows_valid = min(BM, p.seq_act - tis * BM);
+    a_row = b * p.a_seq_stride + p.a_row0 + tis * BM;
+    pos0 = p.g.pos_begin + tis * BM;
+    crow0 = (size_t)b * p.g.max_seq + pos0;
   }
-  // ---- which columns?
-  const int tph = p.hd_map / BN;                 // tiles per head
-  const int nt_local = nt < p.n_split ? nt : nt - p.n_split;
-  const int head = nt_local / tph, jb = nt_local - head * tph;
-  const int col_lo = head * p.hd_map + jb * (BN / 2);
-  const int col_hi = col_lo + p.hd_map / 2;
-  const CUtensorMap* tm_b = nt < p.n_split ? &tm_b0 : &tm_b1;
+  // ---- which columns?  Tiles [0, n_split) belong to W0/out0, the rest to W1/out1.
+  const bool is_b1 = nt >= p.n_split;
+  const int n0 = (is_b1 ? nt - p.n_split : nt) * BN;
+  const CUtensorMap* tm_b = is_b1 ? &tm_b1 : &tm_b0;
+  // ---- which slice of the reduction?
+  const int KB = p.K / BK;
+  const int kb_begin = (int)(((long long)KB * z) / splits), kb_end = (int)(((long long)KB * (z + 1)) / splits);
+  const int nkb = kb_end - kb_begin;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(accum_bar, 1);
+    mbar_init(recv_bar, 1);
     fence_mbar_init();
+    if (splits > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)(BM / 2) * PROW_BYTES);   // the partner's 64 rows
     prefetch_tmap(&tm_a);
     prefetch_tmap(tm_b);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN < 32 ? 32 : BN);
+    tmem_alloc(tmem_slot, BN);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int KB = p.K / 64;
-  // Each CTA walks the reduction dimension from its own starting block, so that the CTAs sharing an operand tile
-  // do not all ask the L2 for the same lines at the same moment.
-  const int k_rot = (int)((nt * p.rot_n + mt * p.rot_m) % KB);
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
+
+  // epilogue geometry
+  const int rows_per_cta = BM / splits;           // rows of the tile this CTA finishes
+  const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
+  const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
+  const int head0 = n0 / HD;
 
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < KB; ++kb) {
-        const int s = kb % STAGES;
-        mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, p.status);
-        uint8_t* a_dst = smem + s * S::STAGE_BYTES;
-        uint8_t* b_dst = a_dst + S::A_BYTES;
-        mbar_arrive_expect_tx(&full_bar[s], S::STAGE_BYTES);
-        int kx = kb + k_rot;
-        if (kx >= KB) kx -= KB;
-        tma_load_2d(a_dst, &tm_a, kx * 64, a_row, &full_bar[s]);
-        if (p.b_single) {                       // both column halves are adjacent rows of W: one box
-          tma_load_2d(b_dst, tm_b, kx * 64, col_lo, &full_bar[s]);
-        } else {
-          tma_load_2d(b_dst, tm_b, kx * 64, col_lo, &full_bar[s]);
-          tma_load_2d(b_dst + S::B_BYTES / 2, tm_b, kx * 64, col_hi, &full_bar[s]);
-        }
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % STAGES;
+        mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
+        uint8_t* a_dst = smem + s * STAGE_BYTES;
+        mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+        tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
+        tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, BN);
-      for (int kb = 0; kb < KB; ++kb) {
-        const int s = kb % STAGES;
-        mbar_wait(&full_bar[s], (kb / STAGES) & 1, p.status);
+      constexpr uint32_t idesc = idesc_bf16(BM, BN);
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % STAGES;
+        mbar_wait(&full_bar[s], (i / STAGES) & 1, p.status);
         tc_fence_after();
-        if (dbg && kb == 0) p.debug[2] = globaltimer_ns();
-        const uint32_t a_addr = smem_u32(smem + s * S::STAGE_BYTES);
+        if (dbg && i == 0) p.debug[2] = globaltimer_ns();
+        const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
         const uint64_t a_desc = smem_desc_k_sw128(a_addr);
-        const uint64_t b_desc = smem_desc_k_sw128(a_addr + S::A_BYTES);
-        for (int rep = 0; rep < p.mma_rep; ++rep)
+        const uint64_t b_desc = smem_desc_k_sw128(a_addr + A_BYTES);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
-          umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+        for (int k = 0; k < BK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
+          umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
         umma_commit(&empty_bar[s]);
       }
       umma_commit(accum_bar);
     }
     __syncwarp();
   } else {
-    // ---- epilogue: thread <-> output row
+    // While the main loop runs, pull the table rows the finishing pass of this CTA will read into the L2
+    // (dense tiles; 512 bytes = 4 lines per row and table).
+    if (p.idx == nullptr) {
+      const bool score_tile = (EPI == EPI_Q) && p.has_prev && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+      for (int i = threadIdx.x - 64; i < rows_per_cta * 4; i += 128) {
+        const int r = z * rows_per_cta + (i >> 2);
+        if (r >= rows_valid) break;
+        if (rotate) prefetch_l2(p.rope + (size_t)(pos0 + r) * (HD / 2) + (i & 3) * 16);
+        if (score_tile) prefetch_l2(p.q_prev + (crow0 + r) * HD + (i & 3) * 32);
+      }
+    }
     mbar_wait(accum_bar, 0, p.status);
     tc_fence_after();
     if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
-    const int quarter = warp & 3;               // TMEM lanes this warp may touch: 32*quarter .. +31
+    if (rec && threadIdx.x == 64) p.debug[64 + 3 * lin + 1] = globaltimer_ns();
+  }
+
+  // ---- every CTA of the cluster has finished its main loop: the rings are free to receive partial rows
+  tc_fence_before();
+  if (splits > 1) cluster_sync_all(); else __syncthreads();
+  tc_fence_after();
+  if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[32] = globaltimer_ns();
+  if (warp >= 2) {
+    // this warp's 32 rows of the partial accumulator: tensor memory -> own shared memory, thread <-> row
     const int r = quarter * 32 + lane;
-    const bool valid = r < rows_valid;
+    const uint32_t dst = smem_u32(smem + (size_t)r * PROW_BYTES);
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    int t = 0;                                  // token (flat active index) of this row
-    if (valid) t = p.idx ? p.idx[t0 + r] : t0 + r;
-    const int pos = p.g.position(t);
-    const size_t crow = (size_t)p.g.cache_row(t);
-    constexpr int NCH = BN / 64;                // chunks of 32 column pairs
-    constexpr int HALF_W = BN / 2;
-    const bool is_b1 = nt >= p.n_split;
-
-    constexpr int ROW_BYTES = BN * 2;            // one staged output row (bf16)
-    constexpr int UNITS = ROW_BYTES / 16;        // 16-byte units per staged row
-    // The operand ring is idle once the accumulator is complete: its first 128 x ROW_BYTES bytes stage the tile so
-    // that the global stores below are whole contiguous row segments.
-    uint8_t* stg = smem;
-    const size_t tm_rows = (size_t)p.q_prev_rows;  // row count of the transposed stored-query array
-    const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
-    const bool score_tile = (EPI == EPI_Q) && head == p.g.score_head;
-
-    float dot = 0.f, n1 = 0.f, n2 = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < NCH; ++c) {
-      float lo[32], hi[32];
-      tmem_ld_32x32(t_lane + c * 32, lo);
-      tmem_ld_32x32(t_lane + HALF_W + c * 32, hi);
-      const int j0 = jb * HALF_W + c * 32;       // index of lo[0] inside the head (rotary pair index)
-      if (valid) {
-        if (score_tile) {
-          // stored query, transposed [head_dim][cache rows]: consecutive rows of a tile are consecutive addresses
-          float* qa = p.q_prev + (size_t)j0 * tm_rows + crow;
-          float* qb = p.q_prev + (size_t)(p.g.head_dim / 2 + j0) * tm_rows + crow;
-          if (p.has_prev) {
+    for (int ch = 0; ch < BN / 32; ++ch) {
+      float v[32];
+      tmem_ld_32x32(t_lane + ch * 32, v);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float a = qa[(size_t)i * tm_rows], b = qb[(size_t)i * tm_rows];
-              dot = fmaf(lo[i], a, dot); dot = fmaf(hi[i], b, dot);
-              n2 = fmaf(a, a, n2); n2 = fmaf(b, b, n2);
-              n1 = fmaf(lo[i], lo[i], n1); n1 = fmaf(hi[i], hi[i], n1);
+      for (int g4 = 0; g4 < 8; ++g4)
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(((ch * 8 + g4) ^ (r & 7)) << 4)),
+                     "f"(v[4 * g4]), "f"(v[4 * g4 + 1]), "f"(v[4 * g4 + 2]), "f"(v[4 * g4 + 3]) : "memory");
+    }
+    if (splits > 1) {
+      const int owner = r / rows_per_cta;
+      if (owner != z) {                            // hand the 32 rows to their owner: one 32 KB bulk copy
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int rl0 = quarter * 32 - owner * rows_per_cta;
+          const uint32_t src = smem_u32(smem + (size_t)(quarter * 32) * PROW_BYTES);
+          const uint32_t rdst = map_to_cta(smem_u32(smem + RECV_OFFSET + (size_t)rl0 * PROW_BYTES), (uint32_t)owner);
+          const uint32_t rbar = map_to_cta(smem_u32(recv_bar), (uint32_t)owner);
+          bulk_copy_to_cta(rdst, src, 32 * PROW_BYTES, rbar);
+        }
+      }
+    }
+  }
+  if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[33] = globaltimer_ns();
+  __syncthreads();
+  if (splits > 1) mbar_wait(recv_bar, 0, p.status);     // the partner's rows have landed
+  if (dbg && threadIdx.x == 64) p.debug[4] = globaltimer_ns();
+
+  // ---- finish the owned rows: one warp per row, lane <-> pairs (2*lane, 2*lane+1) of each head of the tile.
+  // Rows are taken four at a time so that their table reads are in flight together.
+  {
+    __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
+    const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+    constexpr int RB = 4;
+#pragma unroll 1
+    for (int rl0 = warp; rl0 < rows_per_cta; rl0 += 6 * RB) {
+      int tok[RB];
+      size_t crow[RB];
+      bool ok[RB];
+      float4 cs[RB];
+      float2 qa[RB], qb[RB];
+#pragma unroll
+      for (int k = 0; k < RB; ++k) {
+        const int rl = rl0 + 6 * k;
+        const int r = z * rows_per_cta + rl;
+        ok[k] = rl < rows_per_cta && r < rows_valid;
+        tok[k] = 0; crow[k] = 0;
+        cs[k] = make_float4(1.f, 0.f, 1.f, 0.f);
+        qa[k] = qb[k] = make_float2(0.f, 0.f);
+        if (ok[k]) {
+          int pos;
+          if (p.idx) {
+            tok[k] = p.idx[t0 + r];
+            pos = p.g.position(tok[k]);
+            crow[k] = (size_t)p.g.cache_row(tok[k]);
+          } else {
+            tok[k] = t0 + r;
+            pos = pos0 + r;
+            crow[k] = crow0 + r;
+          }
+          if (rotate) cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)pos * (HD / 2) + 2 * lane);
+          if (score_tile && p.has_prev) {
+            qa[k] = *reinterpret_cast<const float2*>(p.q_prev + crow[k] * HD + 2 * lane);
+            qb[k] = *reinterpret_cast<const float2*>(p.q_prev + crow[k] * HD + HD / 2 + 2 * lane);
+          }
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < RB; ++k) {
+        if (!ok[k]) continue;
+        const int rl = rl0 + 6 * k;
+        const size_t orow = p.out_is_cache ? crow[k] : (size_t)tok[k];
+#pragma unroll
+        for (int hh = 0; hh < BN / HD; ++hh) {
+          float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
+          const int c_lo = hh * HD + 2 * lane, c_hi = c_lo + HD / 2;
+          const uint32_t off_lo = (uint32_t)((((c_lo >> 2) ^ (rl & 7)) << 4) | ((c_lo & 3) << 2));
+          const uint32_t off_hi = (uint32_t)((((c_hi >> 2) ^ (rl & 7)) << 4) | ((c_hi & 3) << 2));
+          {
+            const uint8_t* row = smem + (size_t)(z * rows_per_cta + rl) * PROW_BYTES;      // this CTA's partial
+            lo = *reinterpret_cast<const float2*>(row + off_lo);
+            hi = *reinterpret_cast<const float2*>(row + off_hi);
+          }
+          if (splits > 1) {
+            const uint8_t* row = smem + RECV_OFFSET + (size_t)rl * PROW_BYTES;             // the partner's partial
+            const float2 a = *reinterpret_cast<const float2*>(row + off_lo);
+            const float2 b = *reinterpret_cast<const float2*>(row + off_hi);
+            lo.x += a.x; lo.y += a.y; hi.x += b.x; hi.y += b.y;
+          }
+          if (EPI == EPI_Q && head0 + hh == p.g.score_head) {
+            // Sec. 3.1: 1 - cos(current, stored) on the un-rotated query of the scoring head; then store the current
+            float* qp = p.q_prev + crow[k] * HD;
+            float dot = 0.f, n1 = 0.f, n2 = 0.f;
+            if (p.has_prev) {
+              const float2 a = qa[k], b = qb[k];
+              dot = lo.x * a.x + lo.y * a.y + hi.x * b.x + hi.y * b.y;
+              n1 = lo.x * lo.x + lo.y * lo.y + hi.x * hi.x + hi.y * hi.y;
+              n2 = a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y;
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+                dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                n1 += __shfl_xor_sync(0xffffffffu, n1, o);
+                n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+              }
+            }
+            *reinterpret_cast<float2*>(qp + 2 * lane) = lo;
+            *reinterpret_cast<float2*>(qp + HD / 2 + 2 * lane) = hi;
+            if (lane == 0) {
+              float sc = __int_as_float(0x7f800000);   // +inf: nothing to compare with
+              if (p.has_prev) {
+                const float den = sqrtf(n1) * sqrtf(n2);
+                sc = 1.f - (den > 0.f ? dot / den : 0.f);
+              }
+              p.scores[tok[k]] = sc;
             }
           }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) { qa[(size_t)i * tm_rows] = lo[i]; qb[(size_t)i * tm_rows] = hi[i]; }
-        }
-        if (rotate) {
-          // rotary table, transposed [pair index][position]
-          const float2* cs = p.rope + (size_t)j0 * p.g.max_seq + pos;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float2 cv = cs[(size_t)i * p.g.max_seq];
-            const float a0 = lo[i], b0 = hi[i];
-            lo[i] = a0 * cv.x - b0 * cv.y;
-            hi[i] = a0 * cv.y + b0 * cv.x;
+          if (rotate) {
+            const float a0 = lo.x, b0 = hi.x, a1 = lo.y, b1 = hi.y;
+            lo.x = a0 * cs[k].x - b0 * cs[k].y; hi.x = a0 * cs[k].y + b0 * cs[k].x;
+            lo.y = a1 * cs[k].z - b1 * cs[k].w; hi.y = a1 * cs[k].w + b1 * cs[k].z;
           }
+          __nv_bfloat16* dst = out + orow * p.ld_out + n0;
+          *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = __floats2bfloat162_rn(lo.x, lo.y);
+          *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = __floats2bfloat162_rn(hi.x, hi.y);
         }
-      }
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const int u_lo = c * 4 + v, u_hi = UNITS / 2 + c * 4 + v;
-        *reinterpret_cast<uint4*>(stg + r * ROW_BYTES + ((u_lo ^ (r & (UNITS - 1))) << 4)) = pack8_bf16(lo + 8 * v);
-        *reinterpret_cast<uint4*>(stg + r * ROW_BYTES + ((u_hi ^ (r & (UNITS - 1))) << 4)) = pack8_bf16(hi + 8 * v);
-      }
-    }
-    if (score_tile && valid) {
-      float sc;
-      if (p.has_prev) {
-        const float den = sqrtf(n1) * sqrtf(n2);
-        sc = 1.f - (den > 0.f ? dot / den : 0.f);
-      } else {
-        sc = __int_as_float(0x7f800000);
-      }
-      p.scores[t] = sc;
-    }
-    __syncwarp();
-    if (dbg && threadIdx.x == 64) p.debug[4] = globaltimer_ns();
-    // ---- write-out: each warp stores its own 32 rows, UNITS lanes per row
-    {
-      __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
-      const long long my_orow = valid ? (long long)(p.out_is_cache ? crow : (size_t)t) : -1;
-      constexpr int ROWS_PER_IT = 32 / UNITS;
-      const int unit = lane % UNITS;
-      const int col = unit < UNITS / 2 ? col_lo + unit * 8 : col_hi + (unit - UNITS / 2) * 8;
-#pragma unroll
-      for (int rr = 0; rr < 32; rr += ROWS_PER_IT) {
-        const int row_l = rr + lane / UNITS;
-        const long long orow = __shfl_sync(0xffffffffu, my_orow, row_l);
-        const int R = quarter * 32 + row_l;
-        const uint4 v = *reinterpret_cast<const uint4*>(stg + R * ROW_BYTES + ((unit ^ (R & (UNITS - 1))) << 4));
-        if (orow >= 0) *reinterpret_cast<uint4*>(out + (size_t)orow * p.ld_out + col) = v;
       }
     }
   }
   if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
   tc_fence_before();
-  __syncthreads();
+  // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
+  if (splits > 1) cluster_sync_all(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
-  if (EPI == EPI_Q && p.debug != nullptr && threadIdx.x == 0 && lin < 1024) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
-  if (warp == 1) tmem_dealloc(tmem_base, BN < 32 ? 32 : BN);
+  if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
+  if (warp == 1) tmem_dealloc(tmem_base, BN);
 }
 
-template <int BN, int EPI>
+template <int EPI, int BN>
 static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
-                              int n_tiles, int m_tiles, cudaStream_t st) {
+                              int n_tiles, int m_tiles, int splits, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = gemm_tc_kernel<BN, EPI>;
+  auto kern = gemm_tc_kernel<EPI, BN>;
+  constexpr int SMEM_TOTAL = Cfg<BN>::SMEM_TOTAL;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmSmem<BN>::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid(n_tiles, m_tiles);
-  kern<<<grid, 192, GemmSmem<BN>::TOTAL, st>>>(a, b0, b1, p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_tiles, m_tiles, splits);
+  cfg.blockDim = dim3(192);
+  cfg.dynamicSmemBytes = SMEM_TOTAL;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = splits;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a, b0, b1, p);
 }
 
-cudaError_t launch_gemm_tc(int bn, int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st) {
+cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
-  if (bn == 128) {
-    if (epi == EPI_Q) return launch_one<128, EPI_Q>(a, b0, b1, p, n_tiles, m_tiles, st);
-    if (epi == EPI_KV) return launch_one<128, EPI_KV>(a, b0, b1, p, n_tiles, m_tiles, st);
-    return launch_one<128, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
+  if (bn == 256) {
+    if (epi == EPI_Q) return launch_one<EPI_Q, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_KV) return launch_one<EPI_KV, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    return launch_one<EPI_OUT, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
   }
-  if (bn == 256 && epi == EPI_OUT) return launch_one<256, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
-  if (bn == 64) {
-    if (epi == EPI_KV) return launch_one<64, EPI_KV>(a, b0, b1, p, n_tiles, m_tiles, st);
-    if (epi == EPI_OUT) return launch_one<64, EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
-  }
+  if (bn == 128 && epi == EPI_KV) return launch_one<EPI_KV, 128>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
   return cudaErrorInvalidValue;
 }
 

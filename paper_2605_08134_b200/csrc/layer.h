@@ -7,13 +7,13 @@ namespace dare {
 
 // Device buffers carved from the caller's workspace.
 struct Buffers {
-  float* rope_cs;   // [head_dim/2, max_seq] (cos, sin), pair index major
+  float* rope_cs;   // [max_seq, head_dim/2] (cos, sin)
   void* xn;         // [T, d]  normalised hidden states (layer dtype)
   void* q;          // [T, d]  rotated queries (layer dtype)
   void* kc;         // [max_batch*max_seq, d] K cache (rotated)
   void* vc;         // [max_batch*max_seq, d] V cache
   void* oc;         // [max_batch*max_seq, d] attention-output cache (before W_O)
-  float* q_prev;    // [head_dim, max_batch*max_seq] un-rotated scoring-head query of the previous step, fp32
+  float* q_prev;    // [max_batch*max_seq, head_dim] un-rotated scoring-head query of the previous step, fp32
   float* scores;    // [T]
   int* idx;         // [T] refresh set, ascending
   int* delta;       // [max_batch*max_seq] staleness counters

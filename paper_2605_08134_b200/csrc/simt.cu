@@ -112,22 +112,22 @@ template <typename T>
 __global__ void __launch_bounds__(128) q_post_kernel(const float* __restrict__ qf, int ldq,
                                                      const float2* __restrict__ rope_cs, float* __restrict__ q_prev,
                                                      float* __restrict__ scores, int has_prev, T* __restrict__ q,
-                                                     StepGeom g, int q_rows) {
+                                                     StepGeom g) {
   __shared__ float red[3][4];
   const int t = blockIdx.x;
   const int hd = g.head_dim, half = hd >> 1;
   const float* row = qf + (size_t)t * ldq;
   const int cr = g.cache_row(t);
-  float* qp = q_prev + cr;                         // transposed store: element j of this token at qp[j * q_rows]
+  float* qp = q_prev + (size_t)cr * hd;
   const float* q0 = row + g.score_head * hd;
   float dot = 0.f, n1 = 0.f, n2 = 0.f;
   for (int j = threadIdx.x; j < hd; j += blockDim.x) {
     const float a = q0[j];
     if (has_prev) {
-      const float b = qp[(size_t)j * q_rows];
+      const float b = qp[j];
       dot = fmaf(a, b, dot); n1 = fmaf(a, a, n1); n2 = fmaf(b, b, n2);
     }
-    qp[(size_t)j * q_rows] = a;
+    qp[j] = a;
   }
   if (has_prev) {
 #pragma unroll
@@ -150,12 +150,12 @@ __global__ void __launch_bounds__(128) q_post_kernel(const float* __restrict__ q
     scores[t] = __int_as_float(0x7f800000);  // +inf: nothing to compare with
   }
   const int pos = g.position(t);
-  const float2* cs = rope_cs + pos;                // transposed table [pair index][position]
+  const float2* cs = rope_cs + (size_t)pos * half;
   T* out = q + (size_t)t * g.d;
   for (int p = threadIdx.x; p < g.d / 2; p += blockDim.x) {
     const int h = p / half, j = p - h * half;
     const float a = row[h * hd + j], b = row[h * hd + j + half];
-    const float2 c = cs[(size_t)j * g.max_seq];
+    const float2 c = cs[j];
     out[h * hd + j] = from_f<T>(a * c.x - b * c.y);
     out[h * hd + j + half] = from_f<T>(a * c.y + b * c.x);
   }
@@ -163,15 +163,15 @@ __global__ void __launch_bounds__(128) q_post_kernel(const float* __restrict__ q
 
 template <typename T>
 void launch_q_post_simt(const float* qf, int ldq, const float* rope_cs, float* q_prev, float* scores, bool has_prev,
-                        T* q, const StepGeom& g, int q_rows, cudaStream_t st) {
+                        T* q, const StepGeom& g, cudaStream_t st) {
   if (g.tokens() <= 0) return;
   q_post_kernel<T><<<g.tokens(), 128, 0, st>>>(qf, ldq, reinterpret_cast<const float2*>(rope_cs), q_prev, scores,
-                                               has_prev ? 1 : 0, q, g, q_rows);
+                                               has_prev ? 1 : 0, q, g);
 }
 template void launch_q_post_simt<float>(const float*, int, const float*, float*, float*, bool, float*, const StepGeom&,
-                                        int, cudaStream_t);
+                                        cudaStream_t);
 template void launch_q_post_simt<__nv_bfloat16>(const float*, int, const float*, float*, float*, bool, __nv_bfloat16*,
-                                                const StepGeom&, int, cudaStream_t);
+                                                const StepGeom&, cudaStream_t);
 
 // ------------------------------------------------------------------------------------------------ K/V post-pass
 // Eq. 3 / Alg. 1 lines 8-9: the refreshed rows replace their cache rows; every other cache row is left untouched.
@@ -187,13 +187,13 @@ __global__ void __launch_bounds__(128) kv_post_kernel(const float* __restrict__ 
   const size_t cr = (size_t)g.cache_row(t);
   const float* krow = kvf + (size_t)r * ld;
   const float* vrow = krow + d;
-  const float2* cs = rope_cs + g.position(t);
+  const float2* cs = rope_cs + (size_t)g.position(t) * half;
   T* ko = kc + cr * d;
   T* vo = vc + cr * d;
   for (int p = threadIdx.x; p < d / 2; p += blockDim.x) {
     const int h = p / half, j = p - h * half;
     const float a = krow[h * hd + j], b = krow[h * hd + j + half];
-    const float2 c = cs[(size_t)j * g.max_seq];
+    const float2 c = cs[j];
     ko[h * hd + j] = from_f<T>(a * c.x - b * c.y);
     ko[h * hd + j + half] = from_f<T>(a * c.y + b * c.x);
   }

@@ -11,9 +11,6 @@ enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2 };
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
-  int mma_rep;           // timing experiment only: issue every MMA this many times (1 = normal)
-  int b_single;          // the W tile is one TMA box of BN rows (column halves adjacent) instead of two of BN/2
-  int rot_n, rot_m;      // per-tile rotation of the starting reduction block (in blocks per n-tile / m-tile)
   int m_total;           // dense: tokens of the step; gathered: capacity of the row list
   int seq_act;           // dense row mapping: rows per sequence ...
   int tiles_per_seq;     // ... and 128-row tiles per sequence
@@ -22,15 +19,13 @@ struct GemmParams {
   const int* idx;        // gathered: token of each A row (ascending refresh set), else nullptr
   const int* count;      // gathered: device count of rows, else nullptr
   StepGeom g;
-  int hd_map;            // head width used for the column mapping of a tile
-  int n_split;           // tiles [0, n_split) use B0/out0, the rest B1/out1
+  int n_split;           // n-tiles [0, n_split) use W0/out0, the rest W1/out1
   __nv_bfloat16* out0;
   __nv_bfloat16* out1;
   int ld_out;
   int out_is_cache;      // output rows addressed by cache row (1) or by flat token index (0)
-  const float2* rope;    // rotary table, transposed: [head_dim/2][max_seq]
-  float* q_prev;         // stored scoring-head query, transposed: [head_dim][q_prev_rows]
-  int q_prev_rows;       // = max_batch * max_seq
+  const float2* rope;    // rotary table [max_seq][head_dim/2]
+  float* q_prev;         // stored scoring-head query [cache rows][head_dim], fp32
   float* scores;
   int has_prev;
   int* status;
@@ -50,7 +45,11 @@ struct AttnParams {
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st);
 
-cudaError_t launch_gemm_tc(int bn, int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st);
+// grid = (n_tiles of bn columns, m_tiles of 128 rows, splits of the reduction dimension = cluster size: 1 or 2);
+// bn = 256 (full tensor rate) or 128 (more CTAs for the weight-streaming K/V projection of a small refresh set).
+// The W tensor maps must have a box of bn rows.
+cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st);
+
 
 }  // namespace dare
