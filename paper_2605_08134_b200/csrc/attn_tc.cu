@@ -67,23 +67,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int h = blockIdx.y;
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
+  pdl_launch_dependents();
   const StepGeom& g = p.g;
   const int tps = (g.seq_act + BQ - 1) / BQ;
   const int b = blockIdx.x / tps, tile = blockIdx.x - b * tps;
-
-  // ---- rows of this tile (uniform over the CTA)
-  int row0, rows_valid;
-  if (p.idx != nullptr) {
-    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
-    row0 = lo + tile * BQ;
-    if (row0 >= hi) return;
-    rows_valid = min(BQ, hi - row0);
-  } else {
-    row0 = b * g.seq_act + tile * BQ;
-    rows_valid = min(BQ, g.seq_act - tile * BQ);
-  }
-  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
-  const int kv_row0 = b * g.max_seq;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
@@ -99,10 +86,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
+  // The set-up above overlapped the tail of the previous kernel in the stream; its results are needed from here on.
+  pdl_wait();
+  // ---- rows of this tile (uniform over the CTA)
+  int row0 = 0, rows_valid = 0;
+  bool active = true;
+  if (p.idx != nullptr) {
+    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
+    row0 = lo + tile * BQ;
+    active = row0 < hi;
+    rows_valid = min(BQ, hi - row0);
+  } else {
+    row0 = b * g.seq_act + tile * BQ;
+    rows_valid = min(BQ, g.seq_act - tile * BQ);
+  }
+  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  const int kv_row0 = b * g.max_seq;
   // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
   {
     uint8_t* qs = smem + S::Q_OFF;
-    for (int u = threadIdx.x; u < BQ * 16; u += kThreads) {
+    for (int u = threadIdx.x; active && u < BQ * 16; u += kThreads) {
       const int r = u >> 4, unit = u & 15;           // 16 units of 8 bf16 per row
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (r < rows_valid) {
@@ -121,6 +124,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + BKV;
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
+  if (active) {
   if (warp == 0) {
     if (lane == 0) {
       for (int i = 0; i < n_blocks; ++i) {
@@ -255,6 +259,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int v = 0; v < 8; ++v) reinterpret_cast<uint4*>(dst)[v] = pack8_bf16(acc + 8 * v);
     }
   }
+  }  // active
   tc_fence_before();
   __syncthreads();
   if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
@@ -272,8 +277,7 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
   const int tps = (p.g.seq_act + BQ - 1) / BQ;
   dim3 grid(p.g.batch * tps, p.g.n_heads);
   if (grid.x == 0) return cudaSuccess;
-  attn_tc_kernel<<<grid, kThreads, AttnSmem::TOTAL, st>>>(tm_k, tm_v, p);
-  return cudaGetLastError();
+  return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), AttnSmem::TOTAL, st, 1, tm_k, tm_v, p);
 }
 
 }  // namespace dare

@@ -1,5 +1,6 @@
 // Memory-bound kernels shared by both kernel paths: rotary table, RMSNorm, threshold + compaction, row gather.
 #include "dare_internal.h"
+#include "tc_ptx.cuh"
 
 namespace dare {
 
@@ -75,6 +76,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
                                                       T* __restrict__ xn, int d, float eps) {
   constexpr int N = Vec16<T>::N;
   __shared__ float red[32];
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();
   const size_t row = blockIdx.x;
   const T* xr = x + row * d;
   T* yr = xn + row * d;
@@ -133,7 +136,7 @@ void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float
   int nvec = d / Vec16<T>::N;
   int threads = nvec >= 512 ? 256 : (nvec >= 128 ? 128 : ((nvec + 31) / 32) * 32);
   if (threads > 256) threads = 256;
-  rmsnorm_kernel<T, 2><<<rows, threads, 0, st>>>(x, gain, xn, d, eps);
+  launch_pdl(rmsnorm_kernel<T, 2>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps);
 }
 template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t);
 template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, __nv_bfloat16*, int, int, float,
@@ -155,6 +158,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
   extern __shared__ int my_rows[];          // tokens whose rows this CTA copies (gather only)
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
+  ptx::pdl_launch_dependents();
+  ptx::pdl_wait();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool publish = blockIdx.x == 0;
@@ -225,9 +230,9 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
     grid = T < 64 ? (T > 0 ? T : 1) : 64;
     smem = ((size_t)(T + grid - 1) / grid + 1) * sizeof(int);
   }
-  select_kernel<<<grid, 1024, smem, st>>>(scores, tau, (select_all || scores == nullptr) ? 1 : 0, g, idx, count,
-                                          batch_off, delta, reinterpret_cast<const uint4*>(gather_src),
-                                          reinterpret_cast<uint4*>(gather_dst), row_bytes / 16);
+  launch_pdl(select_kernel, dim3(grid), dim3(1024), smem, st, 1, scores, tau, (select_all || scores == nullptr) ? 1 : 0,
+             g, idx, count, batch_off, delta, reinterpret_cast<const uint4*>(gather_src),
+             reinterpret_cast<uint4*>(gather_dst), row_bytes / 16);
 }
 
 // ------------------------------------------------------------------------------------------------ row gather

@@ -65,28 +65,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int z = (int)cluster_ctarank();
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
+  pdl_launch_dependents();
   const int lin = (z * gridDim.y + mt) * gridDim.x + nt;
   const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
-  // ---- which rows does this tile cover? (uniform over the cluster; a tile past the refresh set leaves at once)
-  int a_row, t0, rows_valid;
-  int pos0 = 0;          // dense tiles: position and cache row of the tile's first row
-  size_t crow0 = 0;
-  if (p.count != nullptr) {
-    const int n = min(*p.count, p.m_total);
-    t0 = mt * BM;
-    if (t0 >= n) return;
-    rows_valid = min(BM, n - t0);
-    a_row = t0;
-  } else {
-    const int b = mt / p.tiles_per_seq, tis = mt - b * p.tiles_per_seq;
-    t0 = b * p.seq_act + tis * BM;
-    rows_valid = min(BM, p.seq_act - tis * BM);
-    a_row = b * p.a_seq_stride + p.a_row0 + tis * BM;
-    pos0 = p.g.pos_begin + tis * BM;
-    crow0 = (size_t)b * p.g.max_seq + pos0;
-  }
   // ---- which columns?  Tiles [0, n_split) belong to W0/out0, the rest to W1/out1.
   const bool is_b1 = nt >= p.n_split;
   const int n0 = (is_b1 ? nt - p.n_split : nt) * BN;
@@ -113,7 +96,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above overlapped the tail of the previous kernel in the stream; its results are needed from here on.
+  pdl_wait();
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
+
+  // ---- which rows does this tile cover? (uniform over the cluster; a tile past the refresh set has nothing to do)
+  int a_row = 0, t0 = 0, rows_valid = 0;
+  int pos0 = 0;          // dense tiles: position and cache row of the tile's first row
+  size_t crow0 = 0;
+  bool active = true;
+  if (p.count != nullptr) {
+    const int n = min(*p.count, p.m_total);
+    t0 = mt * BM;
+    active = t0 < n;
+    rows_valid = min(BM, n - t0);
+    a_row = t0;
+  } else {
+    const int b = mt / p.tiles_per_seq, tis = mt - b * p.tiles_per_seq;
+    t0 = b * p.seq_act + tis * BM;
+    rows_valid = min(BM, p.seq_act - tis * BM);
+    a_row = b * p.a_seq_stride + p.a_row0 + tis * BM;
+    pos0 = p.g.pos_begin + tis * BM;
+    crow0 = (size_t)b * p.g.max_seq + pos0;
+  }
 
   // epilogue geometry
   const int rows_per_cta = BM / splits;           // rows of the tile this CTA finishes
@@ -121,6 +126,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
 
+  if (active) {
   if (warp == 0) {
     if (lane == 0) {
       for (int i = 0; i < nkb; ++i) {
@@ -310,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
   }
   if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
+  }  // active
   tc_fence_before();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
   if (splits > 1) cluster_sync_all(); else __syncthreads();
@@ -329,19 +336,7 @@ static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_tiles, m_tiles, splits);
-  cfg.blockDim = dim3(192);
-  cfg.dynamicSmemBytes = SMEM_TOTAL;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = splits;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, a, b0, b1, p);
+  return launch_pdl(kern, dim3(n_tiles, m_tiles, splits), dim3(192), SMEM_TOTAL, st, splits, a, b0, b1, p);
 }
 
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,

@@ -161,6 +161,15 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const float (&v)[3
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// ---- programmatic dependent launch ----
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor in the stream is
+// still running.  pdl_wait() blocks until the predecessor has completed and its writes are visible; everything
+// before it (barrier set-up, tensor-memory allocation, descriptor prefetch) overlaps the predecessor's tail.
+// Every CTA calls pdl_wait() before it touches global data or exits, which keeps completion transitive along the
+// stream.  pdl_launch_dependents() lets the successor start its own set-up.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- thread-block clusters: distributed shared memory ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
