@@ -4,13 +4,13 @@
 // The result rows are written straight into the attention-output cache at their cache rows; rows that are not
 // computed keep their cached value (Alg. 2 lines 9-10).
 //
-// One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 64:
+// One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 128:
 //   warp 0       TMA producer: K block and V block of the cache (two 64-column boxes each, 128-byte swizzle),
 //                double buffered
-//   warp 1       one thread issues S = Q K^T (M128 N64 K16 x 8) and O_blk = P V (M128 N128 K16 x 4, V as an MN-major
+//   warp 1       one thread issues S = Q K^T (M128 N128 K16 x 8) and O_blk = P V (M128 N128 K16 x 8, V as an MN-major
 //                operand) into tensor memory
 //   warps 2-9    softmax: thread <-> (query row, half): both halves read the row of S from tensor memory and agree on
-//                the running maximum; each exponentiates 32 of the 64 keys, writes them as bf16 into the swizzled
+//                the running maximum; each exponentiates 64 of the 128 keys, writes them as bf16 into the swizzled
 //                P tile in shared memory, and rescales/accumulates its 64 of the 128 output columns in registers.
 #include "layer.h"
 #include "tc.h"
@@ -23,14 +23,14 @@ using namespace ptx;
 namespace {
 
 constexpr int BQ = 128;    // query rows per CTA
-constexpr int BKV = 64;    // keys per block
+constexpr int BKV = 128;   // keys per block
 constexpr int HD = 128;
 
 struct AttnSmem {
   static constexpr int Q_BYTES = BQ * HD * 2;          // two 64-column chunks of [128 x 128 B]
   static constexpr int K_BYTES = BKV * HD * 2;         // two chunks of [64 x 128 B]
   static constexpr int V_BYTES = BKV * HD * 2;
-  static constexpr int P_BYTES = BQ * BKV * 2;         // [128 x 128 B]
+  static constexpr int P_BYTES = BQ * BKV * 2;         // two 64-key chunks of [128 x 128 B]
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_OFF + Q_BYTES;        // 2 buffers
   static constexpr int V_OFF = K_OFF + 2 * K_BYTES;    // 2 buffers
@@ -42,7 +42,7 @@ struct AttnSmem {
 
 constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 256;
-constexpr uint32_t kTmemCols = 256;     // S: columns [0, 64), O_blk: columns [64, 192)
+constexpr uint32_t kTmemCols = 256;     // S: columns [0, 128), O_blk: columns [128, 256)
 
 }  // namespace
 
@@ -67,11 +67,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int h = blockIdx.y;
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  pdl_launch_dependents();
   const StepGeom& g = p.g;
   const int tps = (g.seq_act + BQ - 1) / BQ;
   const int b = blockIdx.x / tps, tile = blockIdx.x - b * tps;
 
+  // Row tiles past the first one of a sequence are usually empty in the row-sparse case: they look at the refresh
+  // set before spending anything on set-up.
+  if (p.idx != nullptr && tile > 0) {
+    pdl_wait();
+    if (p.batch_off[b] + tile * BQ >= p.batch_off[b + 1]) return;
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
     mbar_init(s_full, 1);
@@ -88,6 +93,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   // The set-up above overlapped the tail of the previous kernel in the stream; its results are needed from here on.
   pdl_wait();
+  pdl_launch_dependents();
   // ---- rows of this tile (uniform over the CTA)
   int row0 = 0, rows_valid = 0;
   bool active = true;
@@ -171,7 +177,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint32_t v_addr = smem_u32(smem + S::V_OFF + buf * S::V_BYTES);
 #pragma unroll
         for (int ks = 0; ks < BKV / 16; ++ks) {
-          const uint64_t a = smem_desc_k_sw128(p_addr + ks * 32);
+          const uint64_t a = smem_desc_k_sw128(p_addr + (ks >> 2) * (BQ * 128) + (ks & 3) * 32);
           const uint64_t bd = smem_desc_mn_sw128(v_addr + ks * (16 * 128), BKV * 128);
           umma_ss(tmem_o, a, bd, idesc_pv, ks != 0 ? 1u : 0u);
         }
@@ -199,36 +205,49 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_wait(s_full, i & 1, p.status);
       tc_fence_after();
       if (dbg && i == 0 && threadIdx.x == 64) p.debug[2] = globaltimer_ns();
-      float s_mine[32], s_other[32];
-      tmem_ld_32x32(tmem_s + lane_addr + half * 32, s_mine);
-      tmem_ld_32x32(tmem_s + lane_addr + (half ^ 1) * 32, s_other);
       const int key0 = i * BKV;
+      const bool ragged = key0 + BKV > g.kv_len;      // last block: keys past kv_len do not exist
       float mx = m;
-      if (key0 + BKV > g.kv_len) {              // ragged last block: keys past kv_len do not exist
+      // the other half's 64 scores only matter for the row maximum
+#pragma unroll
+      for (int cgrp = 0; cgrp < 2; ++cgrp) {
+        float so[32];
+        tmem_ld_32x32(tmem_s + lane_addr + (half ^ 1) * 64 + cgrp * 32, so);
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          if (key0 + half * 32 + j >= g.kv_len) s_mine[j] = -INFINITY;
-          if (key0 + (half ^ 1) * 32 + j >= g.kv_len) s_other[j] = -INFINITY;
+          const float v = (ragged && key0 + (half ^ 1) * 64 + cgrp * 32 + j >= g.kv_len) ? -INFINITY : so[j];
+          mx = fmaxf(mx, v);
         }
       }
+      float s_mine[64];
+      {
+        float t0_[32], t1_[32];
+        tmem_ld_32x32(tmem_s + lane_addr + half * 64, t0_);
+        tmem_ld_32x32(tmem_s + lane_addr + half * 64 + 32, t1_);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fmaxf(s_mine[j], s_other[j]));
+        for (int j = 0; j < 32; ++j) { s_mine[j] = t0_[j]; s_mine[32 + j] = t1_[j]; }
+      }
+      if (ragged) {
+#pragma unroll
+        for (int j = 0; j < 64; ++j)
+          if (key0 + half * 64 + j >= g.kv_len) s_mine[j] = -INFINITY;
+      }
+#pragma unroll
+      for (int j = 0; j < 64; ++j) mx = fmaxf(mx, s_mine[j]);
       const float alpha = exp2f((m - mx) * c);
       m = mx;
       const float mc = mx * c;
       float sum = 0.f;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+      for (int j = 0; j < 64; ++j) {
         s_mine[j] = exp2f(fmaf(s_mine[j], c, -mc));
         sum += s_mine[j];
       }
       l = l * alpha + sum;
-      // P row segment: 32 bf16 = 4 sixteen-byte units at the swizzled positions of row r
+      // P row segment: this half's 64 keys are one 128-byte row of 64-key chunk `half`, 8 swizzled 16-byte units
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const int unit = half * 4 + v;
-        *reinterpret_cast<uint4*>(ps + r * 128 + ((unit ^ (r & 7)) << 4)) = pack8_bf16(s_mine + 8 * v);
-      }
+      for (int v = 0; v < 8; ++v)
+        *reinterpret_cast<uint4*>(ps + half * (BQ * 128) + r * 128 + ((v ^ (r & 7)) << 4)) = pack8_bf16(s_mine + 8 * v);
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(p_full);

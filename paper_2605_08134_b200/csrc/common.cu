@@ -76,8 +76,11 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
                                                       T* __restrict__ xn, int d, float eps) {
   constexpr int N = Vec16<T>::N;
   __shared__ float red[32];
+  // This kernel reads only the step's input and writes x_norm, which no kernel still running can be reading (the
+  // launch is released by the previous kernel only after that kernel has seen all of its own predecessors finish).
+  // So it works right away, under the previous kernel's tail, and waits for that kernel only before it exits,
+  // which keeps "kernel N done => kernels < N done" true along the stream.
   ptx::pdl_launch_dependents();
-  ptx::pdl_wait();
   const size_t row = blockIdx.x;
   const T* xr = x + row * d;
   T* yr = xn + row * d;
@@ -128,6 +131,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     for (int e = 0; e < N; ++e) t[e] = t[e] * r * gain[vi * N + e];
     Vec16<T>::store(yr + vi * N, t);
   }
+  ptx::pdl_wait();
 }
 
 template <typename T>
@@ -158,8 +162,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
   extern __shared__ int my_rows[];          // tokens whose rows this CTA copies (gather only)
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
-  ptx::pdl_launch_dependents();
   ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool publish = blockIdx.x == 0;

@@ -45,6 +45,45 @@ struct Cfg {
 // row-per-warp reads); [128 KB, 192 KB) the partner's partial of the 64 rows this CTA owns (split-K only).
 }  // namespace
 
+// Finishing pass, per warp: RB rows at a time (rows rl0, rl0 + 6, ...); their table reads are issued together.
+constexpr int RB = 6;
+struct RowBatch {
+  int tok[RB];
+  size_t crow[RB];
+  bool ok[RB];
+  float4 cs[RB];          // (cos, sin) of the two rotary pairs this lane owns
+  float2 qa[RB], qb[RB];  // stored query of the scoring head: elements 2*lane.. and 64 + 2*lane..
+};
+
+template <int EPI>
+__device__ __forceinline__ void load_row_batch(RowBatch& rb, const GemmParams& p, int rl0, int z, int rows_per_cta,
+                                               int rows_valid, int t0, int pos0, size_t crow0, bool rotate,
+                                               bool score_tile, int lane) {
+#pragma unroll
+  for (int k = 0; k < RB; ++k) {
+    const int rl = rl0 + 6 * k;
+    const int r = z * rows_per_cta + rl;
+    rb.ok[k] = rl < rows_per_cta && r < rows_valid;
+    const int rc = rb.ok[k] ? r : 0;              // rows that do not exist read row 0's tables and are dropped later
+    int pos;
+    if (p.idx) {
+      rb.tok[k] = p.idx[t0 + rc];
+      pos = p.g.position(rb.tok[k]);
+      rb.crow[k] = (size_t)p.g.cache_row(rb.tok[k]);
+    } else {
+      rb.tok[k] = t0 + rc;
+      pos = pos0 + rc;
+      rb.crow[k] = crow0 + rc;
+    }
+    // no instruction consumes these loads before the finishing pass, so they stay in flight across the exchange
+    if (rotate) rb.cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)pos * (HD / 2) + 2 * lane);
+    if (EPI == EPI_Q && score_tile && p.has_prev) {
+      rb.qa[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + 2 * lane);
+      rb.qb[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + HD / 2 + 2 * lane);
+    }
+  }
+}
+
 template <int EPI, int BN>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
@@ -65,7 +104,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int z = (int)cluster_ctarank();
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  pdl_launch_dependents();
   const int lin = (z * gridDim.y + mt) * gridDim.x + nt;
   const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
@@ -79,6 +117,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int kb_begin = (int)(((long long)KB * z) / splits), kb_end = (int)(((long long)KB * (z + 1)) / splits);
   const int nkb = kb_end - kb_begin;
 
+  // Row tiles past the first one of a gathered launch are usually empty (the refresh set is small): they look at
+  // the count before spending anything on set-up.  The others set up first and wait for the previous kernel later.
+  const bool likely = p.count == nullptr || mt == 0;
+  if (!likely) {
+    pdl_wait();
+    if (mt * BM >= min(*p.count, p.m_total)) return;     // uniform over the cluster
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(accum_bar, 1);
@@ -96,8 +141,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // Everything above overlapped the tail of the previous kernel in the stream; its results are needed from here on.
+  // The weights do not depend on the previous kernel in the stream: the producer starts their first tiles now, so
+  // that they stream in while that kernel drains.  Everything it produced is needed only after pdl_wait().
+  const int n_early = likely ? (nkb < STAGES ? nkb : STAGES) : 0;
+  if (warp == 0 && lane == 0) {
+    for (int i = 0; i < n_early; ++i) {
+      mbar_arrive_expect_tx(&full_bar[i], STAGE_BYTES);
+      tma_load_2d(smem + i * STAGE_BYTES + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[i]);
+    }
+  }
   pdl_wait();
+  pdl_launch_dependents();
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   // ---- which rows does this tile cover? (uniform over the cluster; a tile past the refresh set has nothing to do)
@@ -125,11 +179,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
+  const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+  RowBatch rb;
 
   if (active) {
   if (warp == 0) {
     if (lane == 0) {
-      for (int i = 0; i < nkb; ++i) {
+      for (int i = 0; i < n_early; ++i)          // the W halves of these stages are already on their way
+        tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
+      for (int i = n_early; i < nkb; ++i) {
         const int s = i % STAGES;
         mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
         uint8_t* a_dst = smem + s * STAGE_BYTES;
@@ -162,19 +220,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // While the main loop runs, pull the table rows the finishing pass of this CTA will read into the L2
     // (dense tiles; 512 bytes = 4 lines per row and table).
     if (p.idx == nullptr) {
-      const bool score_tile = (EPI == EPI_Q) && p.has_prev && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
       for (int i = threadIdx.x - 64; i < rows_per_cta * 4; i += 128) {
         const int r = z * rows_per_cta + (i >> 2);
         if (r >= rows_valid) break;
         if (rotate) prefetch_l2(p.rope + (size_t)(pos0 + r) * (HD / 2) + (i & 3) * 16);
-        if (score_tile) prefetch_l2(p.q_prev + (crow0 + r) * HD + (i & 3) * 32);
+        if (score_tile && p.has_prev) prefetch_l2(p.q_prev + (crow0 + r) * HD + (i & 3) * 32);
       }
     }
+    // the table reads of this warp's first rows of the finishing pass: in flight for the whole main loop
+    load_row_batch<EPI>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
     mbar_wait(accum_bar, 0, p.status);
     tc_fence_after();
     if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
     if (rec && threadIdx.x == 64) p.debug[64 + 3 * lin + 1] = globaltimer_ns();
   }
+
+  // The table reads of the first rows the producer and MMA warps will finish start now (those of the other warps
+  // started before the main loop) and land during the exchange below.
+  if (warp < 2) load_row_batch<EPI>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
 
   // ---- every CTA of the cluster has finished its main loop: the rings are free to receive partial rows
   tc_fence_before();
@@ -219,104 +282,103 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // Rows are taken four at a time so that their table reads are in flight together.
   {
     __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
-    const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
-    constexpr int RB = 4;
 #pragma unroll 1
     for (int rl0 = warp; rl0 < rows_per_cta; rl0 += 6 * RB) {
-      int tok[RB];
-      size_t crow[RB];
-      bool ok[RB];
-      float4 cs[RB];
-      float2 qa[RB], qb[RB];
+      if (rl0 != warp) load_row_batch<EPI>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[34 + (rl0 - warp) / (6 * RB) * 2] = globaltimer_ns();
+      // (1) combine the partial rows: lane <-> pairs (2*lane, 2*lane+1) of each head
+      float2 vlo[RB][BN / HD], vhi[RB][BN / HD];
 #pragma unroll
       for (int k = 0; k < RB; ++k) {
-        const int rl = rl0 + 6 * k;
-        const int r = z * rows_per_cta + rl;
-        ok[k] = rl < rows_per_cta && r < rows_valid;
-        tok[k] = 0; crow[k] = 0;
-        cs[k] = make_float4(1.f, 0.f, 1.f, 0.f);
-        qa[k] = qb[k] = make_float2(0.f, 0.f);
-        if (ok[k]) {
-          int pos;
-          if (p.idx) {
-            tok[k] = p.idx[t0 + r];
-            pos = p.g.position(tok[k]);
-            crow[k] = (size_t)p.g.cache_row(tok[k]);
-          } else {
-            tok[k] = t0 + r;
-            pos = pos0 + r;
-            crow[k] = crow0 + r;
-          }
-          if (rotate) cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)pos * (HD / 2) + 2 * lane);
-          if (score_tile && p.has_prev) {
-            qa[k] = *reinterpret_cast<const float2*>(p.q_prev + crow[k] * HD + 2 * lane);
-            qb[k] = *reinterpret_cast<const float2*>(p.q_prev + crow[k] * HD + HD / 2 + 2 * lane);
-          }
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < RB; ++k) {
-        if (!ok[k]) continue;
-        const int rl = rl0 + 6 * k;
-        const size_t orow = p.out_is_cache ? crow[k] : (size_t)tok[k];
+        const int rl = rb.ok[k] ? rl0 + 6 * k : warp;     // rows that do not exist re-read an existing one
 #pragma unroll
         for (int hh = 0; hh < BN / HD; ++hh) {
-          float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
           const int c_lo = hh * HD + 2 * lane, c_hi = c_lo + HD / 2;
           const uint32_t off_lo = (uint32_t)((((c_lo >> 2) ^ (rl & 7)) << 4) | ((c_lo & 3) << 2));
           const uint32_t off_hi = (uint32_t)((((c_hi >> 2) ^ (rl & 7)) << 4) | ((c_hi & 3) << 2));
-          {
-            const uint8_t* row = smem + (size_t)(z * rows_per_cta + rl) * PROW_BYTES;      // this CTA's partial
-            lo = *reinterpret_cast<const float2*>(row + off_lo);
-            hi = *reinterpret_cast<const float2*>(row + off_hi);
-          }
+          const uint8_t* mine = smem + (size_t)(z * rows_per_cta + rl) * PROW_BYTES;      // this CTA's partial
+          float2 lo = *reinterpret_cast<const float2*>(mine + off_lo);
+          float2 hi = *reinterpret_cast<const float2*>(mine + off_hi);
           if (splits > 1) {
-            const uint8_t* row = smem + RECV_OFFSET + (size_t)rl * PROW_BYTES;             // the partner's partial
-            const float2 a = *reinterpret_cast<const float2*>(row + off_lo);
-            const float2 b = *reinterpret_cast<const float2*>(row + off_hi);
+            const uint8_t* theirs = smem + RECV_OFFSET + (size_t)rl * PROW_BYTES;         // the partner's partial
+            const float2 a = *reinterpret_cast<const float2*>(theirs + off_lo);
+            const float2 b = *reinterpret_cast<const float2*>(theirs + off_hi);
             lo.x += a.x; lo.y += a.y; hi.x += b.x; hi.y += b.y;
           }
-          if (EPI == EPI_Q && head0 + hh == p.g.score_head) {
-            // Sec. 3.1: 1 - cos(current, stored) on the un-rotated query of the scoring head; then store the current
-            float* qp = p.q_prev + crow[k] * HD;
-            float dot = 0.f, n1 = 0.f, n2 = 0.f;
-            if (p.has_prev) {
-              const float2 a = qa[k], b = qb[k];
-              dot = lo.x * a.x + lo.y * a.y + hi.x * b.x + hi.y * b.y;
-              n1 = lo.x * lo.x + lo.y * lo.y + hi.x * hi.x + hi.y * hi.y;
-              n2 = a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y;
+          vlo[k][hh] = lo; vhi[k][hh] = hi;
+        }
+      }
+      // (2) Sec. 3.1 on the un-rotated query of the scoring head: 1 - cos(current, stored), all rows of the batch
+      //     reduced across the lanes together; lane k finishes row k.  Then the current query is stored.
+      if (EPI == EPI_Q && score_tile) {
+        float dot[RB], n1[RB], n2[RB];
 #pragma unroll
-              for (int o = 16; o > 0; o >>= 1) {
-                dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                n1 += __shfl_xor_sync(0xffffffffu, n1, o);
-                n2 += __shfl_xor_sync(0xffffffffu, n2, o);
-              }
-            }
+        for (int k = 0; k < RB; ++k) {
+          float2 lo = vlo[k][0], hi = vhi[k][0];
+#pragma unroll
+          for (int hh = 1; hh < BN / HD; ++hh)
+            if (head0 + hh == p.g.score_head) { lo = vlo[k][hh]; hi = vhi[k][hh]; }
+          const float2 a = rb.qa[k], b = rb.qb[k];
+          dot[k] = lo.x * a.x + lo.y * a.y + hi.x * b.x + hi.y * b.y;
+          n1[k] = lo.x * lo.x + lo.y * lo.y + hi.x * hi.x + hi.y * hi.y;
+          n2[k] = a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y;
+          if (rb.ok[k]) {
+            float* qp = p.q_prev + rb.crow[k] * HD;
             *reinterpret_cast<float2*>(qp + 2 * lane) = lo;
             *reinterpret_cast<float2*>(qp + HD / 2 + 2 * lane) = hi;
-            if (lane == 0) {
-              float sc = __int_as_float(0x7f800000);   // +inf: nothing to compare with
-              if (p.has_prev) {
-                const float den = sqrtf(n1) * sqrtf(n2);
-                sc = 1.f - (den > 0.f ? dot / den : 0.f);
-              }
-              p.scores[tok[k]] = sc;
-            }
           }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int k = 0; k < RB; ++k) {
+            dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], o);
+            n1[k] += __shfl_xor_sync(0xffffffffu, n1[k], o);
+            n2[k] += __shfl_xor_sync(0xffffffffu, n2[k], o);
+          }
+        }
+        float my_dot = 0.f, my_n1 = 0.f, my_n2 = 0.f;
+        int my_tok = -1;
+#pragma unroll
+        for (int k = 0; k < RB; ++k)
+          if (lane == k) { my_dot = dot[k]; my_n1 = n1[k]; my_n2 = n2[k]; my_tok = rb.ok[k] ? rb.tok[k] : -1; }
+        if (my_tok >= 0) {
+          float sc = __int_as_float(0x7f800000);   // +inf: nothing to compare with
+          if (p.has_prev) {
+            const float den = sqrtf(my_n1) * sqrtf(my_n2);
+            sc = 1.f - (den > 0.f ? my_dot / den : 0.f);
+          }
+          p.scores[my_tok] = sc;
+        }
+      }
+      // (3) rotary embedding and bf16 store
+#pragma unroll
+      for (int k = 0; k < RB; ++k) {
+        if (!rb.ok[k]) continue;
+        const size_t orow = p.out_is_cache ? rb.crow[k] : (size_t)rb.tok[k];
+        __nv_bfloat16* dst = out + orow * p.ld_out + n0;
+#pragma unroll
+        for (int hh = 0; hh < BN / HD; ++hh) {
+          float2 lo = vlo[k][hh], hi = vhi[k][hh];
+          const int c_lo = hh * HD + 2 * lane, c_hi = c_lo + HD / 2;
           if (rotate) {
             const float a0 = lo.x, b0 = hi.x, a1 = lo.y, b1 = hi.y;
-            lo.x = a0 * cs[k].x - b0 * cs[k].y; hi.x = a0 * cs[k].y + b0 * cs[k].x;
-            lo.y = a1 * cs[k].z - b1 * cs[k].w; hi.y = a1 * cs[k].w + b1 * cs[k].z;
+            lo.x = a0 * rb.cs[k].x - b0 * rb.cs[k].y; hi.x = a0 * rb.cs[k].y + b0 * rb.cs[k].x;
+            lo.y = a1 * rb.cs[k].z - b1 * rb.cs[k].w; hi.y = a1 * rb.cs[k].w + b1 * rb.cs[k].z;
           }
-          __nv_bfloat16* dst = out + orow * p.ld_out + n0;
           *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = __floats2bfloat162_rn(lo.x, lo.y);
           *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = __floats2bfloat162_rn(hi.x, hi.y);
         }
       }
+      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[35 + (rl0 - warp) / (6 * RB) * 2] = globaltimer_ns();
     }
   }
   if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
-  }  // active
+  } else if (warp == 0 && lane == 0) {
+    // a tile past the refresh set: complete the stages whose W halves were started early, then let them land
+    for (int i = 0; i < n_early; ++i) tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, 0, &full_bar[i]);
+    for (int i = 0; i < n_early; ++i) mbar_wait(&full_bar[i], 0, p.status);
+  }
   tc_fence_before();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
   if (splits > 1) cluster_sync_all(); else __syncthreads();

@@ -10,7 +10,7 @@ struct TcState {
   CUtensorMap a_xn, a_xg, a_oc;            // A operands, box 64 x 128 rows
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 256 rows
   CUtensorMap w_k128, w_v128;              // weights, box 64 x 128 rows
-  CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 64 rows
+  CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 128 rows (keys)
 };
 
 namespace {
@@ -68,8 +68,8 @@ dare_status_t tc_create(dare_layer* L) {
             make_map(&s->a_oc, L->buf.oc, Tm, d, 128) && make_map(&s->w_q, L->w.w_q, d, d, 256) &&
             make_map(&s->w_k, L->w.w_k, d, d, 256) && make_map(&s->w_v, L->w.w_v, d, d, 256) &&
             make_map(&s->w_o, L->w.w_o, d, d, 256) && make_map(&s->w_k128, L->w.w_k, d, d, 128) &&
-            make_map(&s->w_v128, L->w.w_v, d, d, 128) && make_map(&s->kc64, L->buf.kc, Tm, d, 64) &&
-            make_map(&s->vc64, L->buf.vc, Tm, d, 64);
+            make_map(&s->w_v128, L->w.w_v, d, d, 128) && make_map(&s->kc64, L->buf.kc, Tm, d, 128) &&
+            make_map(&s->vc64, L->buf.vc, Tm, d, 128);
   if (!ok) { delete s; return DARE_ERR_CUDA; }
   L->tc = s;
   return DARE_OK;

@@ -165,8 +165,9 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const float (&v)[3
 // A kernel launched with the programmatic-serialization attribute may start while its predecessor in the stream is
 // still running.  pdl_wait() blocks until the predecessor has completed and its writes are visible; everything
 // before it (barrier set-up, tensor-memory allocation, descriptor prefetch) overlaps the predecessor's tail.
-// Every CTA calls pdl_wait() before it touches global data or exits, which keeps completion transitive along the
-// stream.  pdl_launch_dependents() lets the successor start its own set-up.
+// Every CTA calls pdl_wait() before it touches data another kernel writes and before it exits, which keeps completion
+// transitive along the stream.  pdl_launch_dependents() lets the successor start its own set-up; the kernels call
+// it after their own pdl_wait(), so a successor only ever starts once everything two or more kernels back is done.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
