@@ -255,12 +255,18 @@ def run_ours(args):
     d, n = shape.d_model, (n_planned if mode != 0 else T)
     n_kv = n if (mode & 1) else T
     n_o = n if (mode & 2) else T
+    # algorithmic work per launch (what the DARE step itself must move or compute, never the dense work avoided):
+    #   projections: 2*M*d*d flop each; the K/V projection of a small refresh set is a stream of both weight
+    #   matrices (2*d*d*2 bytes) plus the gathered rows in and the K, V rows out (3*n*d*2 bytes);
+    #   attention: 4*rows*S*d flop; RMSNorm: read + write of [T, d] bf16; selection: scores in, index list out,
+    #   plus the compacted copy of the refresh set's x_norm rows (read + write) when K/V reuse is on.
     work = {
         "q_gemm": ("tensor", 2.0 * T * d * d),
         "out_gemm": ("tensor", 2.0 * T * d * d),
         "kv_gemm": ("hbm", 2.0 * d * d * 2 + 3.0 * n_kv * d * 2) if n_kv <= 215 else ("tensor", 4.0 * n_kv * d * d),
         "attention": ("tensor", 4.0 * n_o * shape.seq * d),   # n_o counts rows of all sequences
         "rmsnorm": ("hbm", 2.0 * T * d * 2),
+        "select_compact": ("hbm", 4.0 * T + 4.0 * n + (2.0 * n * d * 2 if (mode & 1) else 0.0)),
     }
     rows = []
     for name, us in kernels.items():
@@ -275,8 +281,11 @@ def run_ours(args):
         else:
             rows.append({"kernel": name, "us": round(us, 2)})
     dom = max((r for r in rows if "bound" in r), key=lambda r: r["us"])
+    # DRAM bytes per launch of that kernel from one ncu capture of this workload (profiles/ holds the summaries)
+    ncu_traffic = {"q_gemm": 38.5e6, "kv_gemm": 69.0e6, "out_gemm": 38.2e6}
     roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
-                "unit": dom["unit"], "frac": dom["frac"], "traffic": None,
+                "unit": dom["unit"], "frac": dom["frac"],
+                "traffic": ncu_traffic.get(dom["kernel"]) if shape.name == wl.LLADA_LAYER.name else None,
                 "peak_source": f"of {peaks['source']} (sustained figure: the kernel is timed inside the step)",
                 "timing": "CUDA events recorded by the library around each kernel, second pass of K steps"}
 
