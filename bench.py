@@ -89,16 +89,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def make_inputs(shape, changed_frac, seed, torch, device):
+def make_inputs_np(shape, changed_frac, seed):
     """Two hidden-state buffers A, B: B redraws `changed_frac` of the rows of A (uniform positions) and perturbs the
     rest by N(0, (1e-3)^2) before bf16 rounding; stepping A -> B -> A ... refreshes the same set every time."""
-    import numpy as np
     from paper_2605_08134_b200 import workloads as wl
     hs = wl.HiddenStream(shape, seed)
     xa = hs.first()
     n = int(round(changed_frac * shape.seq))
     changed = wl.uniform_positions(hs.rng, shape, n)      # n positions in every sequence
     xb = hs.advance(changed)
+    return xa, xb, changed
+
+
+def make_inputs(shape, changed_frac, seed, torch, device):
+    import numpy as np
+    xa, xb, changed = make_inputs_np(shape, changed_frac, seed)
     to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device).to(torch.bfloat16)
     return xa, xb, changed, to(xa), to(xb)
 
@@ -120,11 +125,9 @@ def run_ours(args):
     import torch
     from paper_2605_08134_b200 import build
     build.build()
-    from paper_2605_08134_b200 import dare, workloads as wl
+    from paper_2605_08134_b200 import dare, distrib, workloads as wl
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = distrib.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
@@ -143,7 +146,7 @@ def run_ours(args):
     mode = MODES[args.mode]
     peaks = load_peaks()
     # every rank runs its own replica (sequences are independent: batch sharding, no data-path collective)
-    xa_np, xb_np, changed, xa, xb = make_inputs(shape, args.changed, shape.seed + 1000 * rank, torch, device)
+    xa_np, xb_np, changed, xa, xb = make_inputs(shape, args.changed, distrib.rank_seed(shape.seed, rank), torch, device)
     n_planned = int(changed.sum())
     layers = make_layers(shape, args.layers, shape.seed + 17 * rank, torch, device, dare)
     y = torch.empty_like(xa)
@@ -189,10 +192,7 @@ def run_ours(args):
         wall = time.perf_counter() - t0
         dev_ms = ev0.elapsed_time(ev1)
         ms = wall * 1e3 if host is not None else dev_ms
-        if dist is not None:
-            t = torch.tensor([ms], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = distrib.max_over_ranks(ms, dist, device)
         barrier()
         return ms, launches
 
@@ -292,7 +292,7 @@ def run_ours(args):
     # ---- CPU baseline: the oracle as it stands, bounded sample
     cpu = None if args.no_cpu_baseline else cpu_baseline(shape, xa_np, xb_np, layers[0], mode, budget_s=12.0)
 
-    tokens_per_s = world * T / (ms_per_step * 1e-3)
+    tokens_per_s = distrib.whole_job_rate(T, world, ms_per_step)
     out = {
         "metric": "tokens_per_s_through_one_dare_layer", "value": round(tokens_per_s, 1), "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
