@@ -175,6 +175,22 @@ const char* dare_kernel_slot_name(int slot);
  * synchronises the stream); `enable` switches recording for later steps. */
 dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint64_t* out_host, void* cuda_stream);
 
+/* Stand-alone pieces of the path for token counts far beyond one layer step (e.g. a whole batch of sequences
+ * scored at once), organised for HBM bandwidth.  Device pointers, asynchronous on the stream.
+ *
+ * dare_drift_scores: Sec. 3.1, s_i = 1 - cos(q_now[i], q_prev[i]) for `rows` rows of `head_dim` float32 each
+ * (row-major, head_dim a multiple of 4); a zero-norm row scores 1.
+ *
+ * dare_select_compact: Eq. 2 and its complement over `n_tokens` float32 scores: idx receives the ascending list of
+ * tokens with !(s <= threshold) (room for n_tokens entries), *count their number.  `scratch` is
+ * dare_select_compact_scratch_bytes(n_tokens) bytes of device memory owned by the caller (per-tile counts and
+ * offsets); n_tokens <= 2^30; NaN threshold is rejected. */
+dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t rows, int head_dim, float* scores,
+                                void* cuda_stream);
+size_t dare_select_compact_scratch_bytes(int64_t n_tokens);
+dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float threshold, int32_t* idx, int32_t* count,
+                                  void* scratch, size_t scratch_bytes, void* cuda_stream);
+
 /* Number of kernels the last dare_layer_step enqueued (for launch accounting in benchmarks). */
 int dare_layer_last_launch_count(const dare_layer_t* layer);
 

@@ -494,6 +494,34 @@ const char* dare_kernel_slot_name(int slot) {
   return "?";
 }
 
+dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t rows, int head_dim, float* scores,
+                                void* cuda_stream) {
+  if (!q_now || !q_prev || !scores) return DARE_ERR_INVALID_ARG;
+  if (rows < 0 || head_dim <= 0 || head_dim % 4 != 0) return DARE_ERR_SHAPE;
+  if (!aligned16(q_now) || !aligned16(q_prev)) return DARE_ERR_ALIGN;
+  CUDA_TRY(launch_drift_scores(q_now, q_prev, rows, head_dim, scores, (cudaStream_t)cuda_stream));
+  return DARE_OK;
+}
+
+size_t dare_select_compact_scratch_bytes(int64_t n_tokens) {
+  if (n_tokens < 0 || n_tokens > (int64_t)1 << 30) return 0;
+  return align_up((size_t)select_large_tiles(n_tokens) * sizeof(int)) * 2 + kAlign;
+}
+
+dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float threshold, int32_t* idx, int32_t* count,
+                                  void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!scores || !idx || !count || !scratch) return DARE_ERR_INVALID_ARG;
+  if (isnan(threshold)) return DARE_ERR_INVALID_ARG;
+  if (n_tokens < 0 || n_tokens > (int64_t)1 << 30) return DARE_ERR_SHAPE;
+  if (!aligned16(scores) || !aligned16(scratch)) return DARE_ERR_ALIGN;
+  if (scratch_bytes < dare_select_compact_scratch_bytes(n_tokens)) return DARE_ERR_WORKSPACE;
+  const size_t half = align_up((size_t)select_large_tiles(n_tokens) * sizeof(int));
+  int* counts = (int*)scratch;
+  int* offsets = (int*)((char*)scratch + half);
+  CUDA_TRY(launch_select_large(scores, n_tokens, threshold, idx, count, counts, offsets, (cudaStream_t)cuda_stream));
+  return DARE_OK;
+}
+
 int dare_layer_last_launch_count(const dare_layer_t* L) {
   if (check_handle(L) != DARE_OK) return 0;
   return L->last_launches;

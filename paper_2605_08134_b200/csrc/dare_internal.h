@@ -70,6 +70,12 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
 template <typename T>
 void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
 
+// ---- stand-alone score / compaction for large token counts (select_large.cu)
+int select_large_tiles(long long n);
+cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, int hd, float* scores, cudaStream_t st);
+cudaError_t launch_select_large(const float* scores, long long n, float tau, int* idx, int* count, int* tile_counts,
+                                int* tile_offsets, cudaStream_t st);
+
 // ---- SIMT path (simt.cu) ----------------------------------------------------------------------------------
 // C[m, n] (fp32, ld = ldc) = sum_k A[arow(m), k] * W[n, k];  arow(m) = a_idx ? a_idx[m] : m;
 // rows m >= *count (when count != nullptr) are skipped.

@@ -62,6 +62,9 @@ def _load():
         "dare_layer_last_kernel_times": (C.c_int, [vp, vp, vp, i32, C.POINTER(C.c_int)]),
         "dare_kernel_slot_name": (C.c_char_p, [C.c_int]),
         "dare_layer_debug_timestamps": (C.c_int, [vp, i32, vp, vp]),
+        "dare_drift_scores": (C.c_int, [vp, vp, C.c_int64, i32, vp, vp]),
+        "dare_select_compact_scratch_bytes": (sz, [C.c_int64]),
+        "dare_select_compact": (C.c_int, [vp, C.c_int64, f32, vp, vp, vp, sz, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -156,6 +159,19 @@ def dare_layer_last_kernel_times(handle, slot_ptr, ms_ptr, capacity):
 
 def dare_layer_debug_timestamps(handle, enable, out_ptr, stream=0) -> int:
     return _lib.dare_layer_debug_timestamps(handle, enable, out_ptr, stream)
+
+
+def dare_drift_scores(q_now_ptr, q_prev_ptr, rows, head_dim, scores_ptr, stream=0) -> int:
+    return _lib.dare_drift_scores(q_now_ptr, q_prev_ptr, rows, head_dim, scores_ptr, stream)
+
+
+def dare_select_compact_scratch_bytes(n_tokens: int) -> int:
+    return _lib.dare_select_compact_scratch_bytes(n_tokens)
+
+
+def dare_select_compact(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, scratch_ptr, scratch_bytes, stream=0) -> int:
+    return _lib.dare_select_compact(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, scratch_ptr, scratch_bytes,
+                                    stream)
 
 
 def dare_kernel_slot_name(slot: int) -> str:

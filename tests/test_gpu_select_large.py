@@ -1,0 +1,81 @@
+"""Stand-alone drift score and multi-tile compaction at token counts far beyond one layer step, against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import dare_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dare():
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare as d
+    return d
+
+
+def _scores(n, seed):
+    """Bimodal scores like the method's: most tokens near zero, a fraction spread over (0.3, 1.5); some NaN, +-inf."""
+    rng = np.random.default_rng(seed)
+    s = np.abs(rng.standard_normal(n).astype(np.float32)) * np.float32(1e-5)
+    hot = rng.random(n) < 0.13
+    s[hot] = rng.uniform(0.3, 1.5, int(hot.sum())).astype(np.float32)
+    if n > 10:
+        s[3] = np.nan; s[7] = np.inf; s[9] = -np.inf
+    return s
+
+
+@pytest.mark.parametrize("n", [0, 1, 5, 4095, 4096, 4097, 100_003, 1 << 20, (1 << 22) + 12345])
+def test_select_compact_matches_the_predicate(dare, n):
+    import torch
+    s = _scores(n, n % 97)
+    sd = torch.from_numpy(s).cuda() if n else torch.zeros(4, device="cuda")
+    idx = torch.full((max(n, 1),), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    nb = dare.dare_select_compact_scratch_bytes(n)
+    assert nb >= 256
+    scratch = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    for tau in (0.1, -1.0, float("inf")):
+        st = dare.dare_select_compact(sd.data_ptr(), n, tau, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(), nb,
+                                      torch.cuda.current_stream().cuda_stream)
+        assert st == 0
+        torch.cuda.synchronize()
+        want = np.nonzero(orc.refresh_mask(s, tau))[0]
+        assert int(cnt.item()) == len(want)
+        np.testing.assert_array_equal(idx[:len(want)].cpu().numpy(), want)
+
+
+def test_select_compact_rejects_bad_arguments(dare):
+    import torch
+    sd = torch.zeros(1024, device="cuda")
+    idx = torch.zeros(1024, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    ok = (sd.data_ptr(), 1024, 0.1, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(), 4096)
+    assert dare.dare_select_compact(*ok) == 0
+    assert dare.dare_select_compact(0, *ok[1:]) == dare.ERR_INVALID_ARG
+    assert dare.dare_select_compact(ok[0], 1024, float("nan"), *ok[3:]) == dare.ERR_INVALID_ARG
+    assert dare.dare_select_compact(ok[0], -1, *ok[2:]) == dare.ERR_SHAPE
+    assert dare.dare_select_compact(*ok[:6], 16) == dare.ERR_WORKSPACE
+    assert dare.dare_select_compact(ok[0] + 4, *ok[1:]) == dare.ERR_ALIGN
+    assert dare.dare_select_compact_scratch_bytes(-5) == 0
+
+
+@pytest.mark.parametrize("rows,hd", [(1, 128), (1000, 64), (65537, 128)])
+def test_drift_scores_match_oracle(dare, rows, hd):
+    import torch
+    rng = np.random.default_rng(rows)
+    a = rng.standard_normal((rows, hd)).astype(np.float32)
+    b = (a + 0.3 * rng.standard_normal((rows, hd))).astype(np.float32)
+    b[0] = 0.0                                     # zero-norm row: score 1
+    if rows > 2:
+        b[1] = a[1]; b[2] = -a[2]
+    ad, bd = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    out = torch.empty(rows, device="cuda")
+    assert dare.dare_drift_scores(ad.data_ptr(), bd.data_ptr(), rows, hd, out.data_ptr()) == 0
+    torch.cuda.synchronize()
+    want = orc.drift_score(a, b)
+    np.testing.assert_allclose(out.cpu().numpy(), want, rtol=0, atol=2e-6)
+    assert out[0].item() == 1.0
+    assert dare.dare_drift_scores(ad.data_ptr(), bd.data_ptr(), rows, 6, out.data_ptr()) == dare.ERR_SHAPE
