@@ -191,6 +191,21 @@ size_t dare_select_compact_scratch_bytes(int64_t n_tokens);
 dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float threshold, int32_t* idx, int32_t* count,
                                   void* scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* dare_select_compact for callers that may not allocate (the paper has no counterpart: this is a service of the
+ * library, not a step of the method).  An inference server that gives all device memory to its own arena at start-up,
+ * or a latency-critical loop that cannot take the device-wide synchronisation of a cudaMalloc, has no scratch buffer
+ * to pass; here the per-tile counts and offsets live in a 32 KB array inside the library image (present on every GPU
+ * that loads the library until the process exits).  Same inputs, outputs and results as dare_select_compact.
+ *   - n_tokens <= dare_select_compact_static_max_tokens() (= 16,777,216); more returns DARE_ERR_SHAPE.
+ *   - The call allocates nothing and frees nothing, on the device or through any library.
+ *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress with that device
+ *     current): make that first call outside any stream capture.
+ *   - All calls on a device share the array; it keeps the previous call's contents (nothing needs clearing: a call
+ *     writes every entry before reading it).  Calls that overlap on the GPU, e.g. on two streams, race on it. */
+int64_t dare_select_compact_static_max_tokens(void);
+dare_status_t dare_select_compact_static(const float* scores, int64_t n_tokens, float threshold, int32_t* idx,
+                                         int32_t* count, void* cuda_stream);
+
 /* Number of kernels the last dare_layer_step enqueued (for launch accounting in benchmarks). */
 int dare_layer_last_launch_count(const dare_layer_t* layer);
 

@@ -6,6 +6,9 @@
 //     (2) exclusive scan of the tile counts (one CTA) -> scratch, total -> *count
 //     (3) per-tile ballot/popcount compaction written at the tile's offset: ascending index list
 // No CTA waits for another; the order of the list does not depend on scheduling.
+#include <math.h>
+#include <mutex>
+
 #include "dare_internal.h"
 
 namespace dare {
@@ -149,3 +152,59 @@ cudaError_t launch_select_large(const float* scores, long long n, float tau, int
 }
 
 }  // namespace dare
+
+// ------------------------------------------------------------------------------------------------------------------
+// Compaction without any caller-provided or allocated scratch.
+//
+// Some hosts of this library hand all of the device's memory to one arena at start-up and forbid every later
+// cudaMalloc (an inference server with a fixed memory plan), or sit in a latency-critical loop where the device-wide
+// synchronisation an allocation implies is not acceptable.  For them the per-tile counts and offsets of the three-pass
+// compaction live in a small array that is part of the library image: 2 x 4096 ints = 32 KB of device memory on every
+// GPU that loads the library, held until the process exits.  That bounds the call at 4096 tiles = 16,777,216 scores.
+//
+// In host code the name `g_select_scratch` is only a stand-in for the symbol; the address a kernel may use comes from
+// cudaGetSymbolAddress, asked once per device with that device current (the first call on a device does this; make
+// that first call outside any stream capture).  All calls on a device share the array: it still holds the previous
+// call's tile counts when the next one starts (every entry a call reads is written by that call first, so nothing
+// needs clearing), and two calls that overlap on the GPU (different streams) race on it.
+namespace dare {
+namespace {
+constexpr int kStaticTiles = 4096;
+static __device__ __align__(256) int g_select_scratch[2 * kStaticTiles];
+constexpr int kMaxDevices = 64;
+int* g_select_scratch_addr[kMaxDevices] = {};
+std::mutex g_select_scratch_mutex;
+
+cudaError_t static_scratch_for_current_device(int** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_select_scratch_mutex);
+  if (g_select_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_select_scratch);
+    if (e != cudaSuccess) return e;
+    g_select_scratch_addr[dev] = static_cast<int*>(p);
+  }
+  *out = g_select_scratch_addr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+}  // namespace dare
+
+extern "C" int64_t dare_select_compact_static_max_tokens(void) { return (int64_t)dare::kStaticTiles * dare::kTile; }
+
+extern "C" dare_status_t dare_select_compact_static(const float* scores, int64_t n_tokens, float threshold, int32_t* idx,
+                                                    int32_t* count, void* cuda_stream) {
+  if (!scores || !idx || !count) return DARE_ERR_INVALID_ARG;
+  if (isnan(threshold)) return DARE_ERR_INVALID_ARG;
+  if (n_tokens < 0 || n_tokens > dare_select_compact_static_max_tokens()) return DARE_ERR_SHAPE;   // beyond the array
+  if ((reinterpret_cast<uintptr_t>(scores) & 15u) != 0) return DARE_ERR_ALIGN;
+  int* scratch = nullptr;
+  if (dare::static_scratch_for_current_device(&scratch) != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
+  cudaError_t e = dare::launch_select_large(scores, n_tokens, threshold, idx, count, scratch,
+                                            scratch + dare::kStaticTiles, (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
+  return DARE_OK;
+}

@@ -65,6 +65,8 @@ def _load():
         "dare_drift_scores": (C.c_int, [vp, vp, C.c_int64, i32, vp, vp]),
         "dare_select_compact_scratch_bytes": (sz, [C.c_int64]),
         "dare_select_compact": (C.c_int, [vp, C.c_int64, f32, vp, vp, vp, sz, vp]),
+        "dare_select_compact_static_max_tokens": (C.c_int64, []),
+        "dare_select_compact_static": (C.c_int, [vp, C.c_int64, f32, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -172,6 +174,15 @@ def dare_select_compact_scratch_bytes(n_tokens: int) -> int:
 def dare_select_compact(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, scratch_ptr, scratch_bytes, stream=0) -> int:
     return _lib.dare_select_compact(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, scratch_ptr, scratch_bytes,
                                     stream)
+
+
+def dare_select_compact_static_max_tokens() -> int:
+    return _lib.dare_select_compact_static_max_tokens()
+
+
+def dare_select_compact_static(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, stream=0) -> int:
+    """dare_select_compact without a scratch argument: for callers that may not allocate device memory."""
+    return _lib.dare_select_compact_static(scores_ptr, n_tokens, threshold, idx_ptr, count_ptr, stream)
 
 
 def dare_kernel_slot_name(slot: int) -> str:
