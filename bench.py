@@ -394,6 +394,57 @@ def run_reference(args):
     }))
 
 
+def run_micro(args):
+    """Memory-bound pieces of the path at a token count large enough to show bandwidth (one JSON line):
+    the drift score (Sec. 3.1) and the threshold + compaction (Eq. 2) over 2^24 tokens, head_dim 128."""
+    import torch
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare
+    peaks = load_peaks()
+    dev = torch.device("cuda", 0)
+    st = torch.cuda.current_stream(dev).cuda_stream
+    out = {"metric": "memory_bound_kernels", "unit": "GB/s", "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
+           "kernels": []}
+
+    def time_it(fn, reps=20):
+        for _ in range(3):
+            fn()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(reps):
+            fn()
+        ev1.record()
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / reps * 1e-3
+
+    rows, hd = 1 << 22, 128
+    a = torch.randn((rows, hd), device=dev)
+    b = a + 0.01 * torch.randn((rows, hd), device=dev)
+    sc = torch.empty(rows, device=dev)
+    t = time_it(lambda: dare.dare_drift_scores(a.data_ptr(), b.data_ptr(), rows, hd, sc.data_ptr(), st))
+    algo = 2.0 * rows * hd * 4 + rows * 4
+    out["kernels"].append({"kernel": "drift_scores", "rows": rows, "head_dim": hd, "us": round(t * 1e6, 1),
+                           "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3)})
+    del a, b
+    n = 1 << 24
+    s = torch.rand(n, device=dev)
+    s = torch.where(s < 0.87, s * 1e-5, s)
+    idx = torch.empty(n, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    nb = dare.dare_select_compact_scratch_bytes(n)
+    scratch = torch.empty(nb, dtype=torch.uint8, device=dev)
+    t = time_it(lambda: dare.dare_select_compact(s.data_ptr(), n, 0.1, idx.data_ptr(), cnt.data_ptr(),
+                                                 scratch.data_ptr(), nb, st))
+    k = int(cnt.item())
+    algo = 4.0 * n + 4.0 * k            # scores in, index list out (the kernels read the scores twice)
+    out["kernels"].append({"kernel": "select_compact", "tokens": n, "refreshed": k, "us": round(t * 1e6, 1),
+                           "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3),
+                           "dram_bytes_moved": 8.0 * n + 4.0 * k})
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -407,8 +458,11 @@ def main():
     ap.add_argument("--d-model", type=int, default=0, help="exploration: other layer width (multiple of 128)")
     ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
     ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
+    ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.micro:
+        run_micro(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

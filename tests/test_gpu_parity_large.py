@@ -1,0 +1,101 @@
+"""Parity at the larger configurations on subsets the oracle can afford (sequences are independent, so a batch row
+checked alone against a batch-1 oracle is a full check of that row)."""
+import copy
+
+import numpy as np
+import pytest
+
+from paper_2605_08134_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dare():
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare as d
+    return d
+
+
+def _weights_gpu(shape, seed, torch):
+    """bf16 weights drawn on the GPU (N(0, 0.02^2)); returned as torch tensors and as float32 numpy for the oracle."""
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    w = {k: (torch.randn((shape.d_model, shape.d_model), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+         for k in ("w_q", "w_k", "w_v", "w_o")}
+    w["rms_gain"] = torch.ones(shape.d_model, device="cuda")
+    wn = {k: v.float().cpu().numpy() for k, v in w.items()}
+    return w, wn
+
+
+def test_config3_dare_o_batched_clustered_steps(dare):
+    """Config 3: batch 8, seq 1024, mode O, 113 clustered + 20 scattered positions changed per sequence and step.
+    All 8 sequences run on the GPU; sequences 0 and 5 are checked against batch-1 oracles for 4 consecutive steps;
+    index sets of all sequences are checked against the plan every step."""
+    import torch
+    shape = wl.LLADA_DARE_O
+    w_t, w_np = _weights_gpu(shape, 33, torch)
+    hs = wl.HiddenStream(shape)
+    g = dare.Layer(shape, w_t)
+    one = wl.scaled(shape, batch=1)
+    checked = (0, 5)
+    oracles = {b: parity.oracle_layer(one, w_np) for b in checked}
+    x = hs.first()
+    y = g.step(parity.to_device(x, shape), 2, 0.1)
+    yo = {b: oracles[b].step(x[b:b + 1], 2, 0.1) for b in checked}
+    for b in checked:
+        parity.assert_close(f"y step0 seq{b}", y[b:b + 1].float().cpu().numpy(), yo[b], parity.TOL_BF16)
+    for step in range(1, 5):
+        ch = wl.clustered_positions(hs.rng, shape, step, 113, 20)
+        x = hs.advance(ch)
+        y = g.step(parity.to_device(x, shape), 2, 0.1)
+        sel = g.last_selection(shape.batch, shape.seq)
+        np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
+        assert sel["count"] == 133 * shape.batch
+        np.testing.assert_array_equal(np.diff(sel["batch_off"]), np.full(shape.batch, 133))
+        caches = g.read_caches(shape.batch, shape.seq)
+        for b in checked:
+            o = oracles[b]
+            yo_b = o.step(x[b:b + 1], 2, 0.1)
+            parity.check_margin(o.last_scores, 0.1)
+            np.testing.assert_array_equal(sel["idx"][sel["batch_off"][b]:sel["batch_off"][b + 1]] - b * shape.seq, o.last_idx)
+            parity.assert_close(f"y step{step} seq{b}", y[b:b + 1].float().cpu().numpy(), yo_b, parity.TOL_BF16)
+            parity.assert_close(f"o_cache step{step} seq{b}", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
+            parity.assert_close(f"k_cache step{step} seq{b}", caches["k"][b:b + 1], o.k_cache, parity.TOL_BF16, max_factor=2.0)
+            np.testing.assert_array_equal(sel["delta"][b], o.delta[0])
+    assert g.status() == 0
+    g.close()
+
+
+@pytest.mark.parametrize("frac,pattern,mode", [(0.15, "uniform", 3), (0.5, "clustered", 1)])
+def test_config5_long_context_one_sequence(dare, frac, pattern, mode):
+    """Config 5: batch 4, seq 4096; all four sequences run on the GPU, sequence 2 is checked against a batch-1 oracle
+    (one dense step + one reuse step), index sets of all sequences against the plan."""
+    import torch
+    shape = wl.LLADA_LONG
+    w_t, w_np = _weights_gpu(shape, 55, torch)
+    hs = wl.HiddenStream(shape)
+    g = dare.Layer(shape, w_t)
+    one = wl.scaled(shape, batch=1)
+    b = 2
+    o = parity.oracle_layer(one, w_np)
+    x0 = hs.first()
+    y0 = g.step(parity.to_device(x0, shape), mode, 0.1)
+    parity.assert_close("y step0", y0[b:b + 1].float().cpu().numpy(), o.step(x0[b:b + 1], mode, 0.1), parity.TOL_BF16)
+    n = int(round(frac * shape.seq))
+    ch = wl.uniform_positions(hs.rng, shape, n) if pattern == "uniform" else wl.clustered_positions(hs.rng, shape, 9, n, 0)
+    x1 = hs.advance(ch)
+    y1 = g.step(parity.to_device(x1, shape), mode, 0.1)
+    sel = g.last_selection(shape.batch, shape.seq)
+    np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
+    yo = o.step(x1[b:b + 1], mode, 0.1)
+    parity.check_margin(o.last_scores, 0.1)
+    parity.assert_close("y step1", y1[b:b + 1].float().cpu().numpy(), yo, parity.TOL_BF16)
+    caches = g.read_caches(shape.batch, shape.seq)
+    parity.assert_close("k_cache", caches["k"][b:b + 1], o.k_cache, parity.TOL_BF16, max_factor=2.0)
+    parity.assert_close("v_cache", caches["v"][b:b + 1], o.v_cache, parity.TOL_BF16, max_factor=2.0)
+    parity.assert_close("o_cache", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
+    assert g.status() == 0
+    g.close()
