@@ -12,6 +12,11 @@
 //   warps 2-9    softmax: thread <-> (query row, half): both halves read the row of S from tensor memory and agree on
 //                the running maximum; each exponentiates 64 of the 128 keys, writes them as bf16 into the swizzled
 //                P tile in shared memory, and rescales/accumulates its 64 of the 128 output columns in registers.
+// Key split: when a launch has few (tile, head) pairs - the row-sparse case with one row tile per sequence - the
+// gridDim.z CTAs of a cluster share a pair, CTA z taking key blocks z, z + gridDim.z, ...  Each CTA leaves its
+// un-normalised accumulator, running maximum and row sum in shared memory; CTA k owns 128/gridDim.z of the rows and
+// receives the other CTAs' partials of those rows by bulk copies over distributed shared memory, then merges them
+// (the usual rescaling by exp(m_z - max_z m_z)) and writes the rows out.
 #include "layer.h"
 #include "tc.h"
 #include "tc_ptx.cuh"
@@ -38,6 +43,10 @@ struct AttnSmem {
   static constexpr int L_OFF = P_OFF + P_BYTES;        // float[2][128] partial row sums
   static constexpr int BAR_OFF = L_OFF + 2 * BQ * 4;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;
+  // after the key loop the operand buffers are idle; the merge of a key split reuses them:
+  static constexpr int DUMP_OFF = 0;                   // this CTA's accumulator [128 rows][128 cols] fp32, 64 KB
+  static constexpr int STAT_OFF = DUMP_OFF + BQ * HD * 4;   // running maximum [128], row sum [128]
+  static constexpr int RECV_OFF = STAT_OFF + 2 * BQ * 4;    // up to 3 senders x (rows x 512 B + rows x 8 B)
 };
 
 constexpr int kThreads = 320;
@@ -60,16 +69,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   uint64_t* p_full = bars + 7;
   uint64_t* o_full = bars + 8;
   uint64_t* o_free = bars + 9;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  uint64_t* recv_bar = bars + 10;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
   float* l_part = reinterpret_cast<float*>(smem + S::L_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y;
-  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  const int h = blockIdx.x;
+  const int ksplit = gridDim.z;                      // = cluster size along z
+  const int z = ksplit > 1 ? (int)cluster_ctarank() : 0;
+  const int rows_own = BQ / ksplit;                   // rows of the tile this CTA writes out
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
   const StepGeom& g = p.g;
-  const int tps = (g.seq_act + BQ - 1) / BQ;
-  const int b = blockIdx.x / tps, tile = blockIdx.x - b * tps;
+  // blockIdx.y = tile * batch + b: the first row tile of every sequence comes first in launch order, so that in the
+  // row-sparse case the CTAs that have work are scheduled before the (many) tiles past the refresh set
+  const int tile = blockIdx.y / g.batch, b = blockIdx.y - tile * g.batch;
 
   // Row tiles past the first one of a sequence are usually empty in the row-sparse case: they look at the refresh
   // set before spending anything on set-up.
@@ -83,7 +97,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     mbar_init(p_full, kSoftmaxThreads);
     mbar_init(o_full, 1);
     mbar_init(o_free, kSoftmaxThreads);
+    mbar_init(recv_bar, 1);
     fence_mbar_init();
+    if (ksplit > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)((ksplit - 1) * rows_own * (HD * 4 + 8)));
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
@@ -106,7 +122,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     row0 = b * g.seq_act + tile * BQ;
     rows_valid = min(BQ, g.seq_act - tile * BQ);
   }
-  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  const int n_blocks_all = (g.kv_len + BKV - 1) / BKV;
+  const int n_blocks = n_blocks_all > z ? (n_blocks_all - z + ksplit - 1) / ksplit : 0;   // blocks z, z + ksplit, ...
   const int kv_row0 = b * g.max_seq;
   // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
   {
@@ -138,7 +155,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         mbar_wait(&kv_empty[buf], ((i >> 1) & 1) ^ 1, p.status);
         uint8_t* kd = smem + S::K_OFF + buf * S::K_BYTES;
         uint8_t* vd = smem + S::V_OFF + buf * S::V_BYTES;
-        const int row = kv_row0 + i * BKV;
+        const int row = kv_row0 + (z + i * ksplit) * BKV;
         mbar_arrive_expect_tx(&k_full[buf], S::K_BYTES);
         tma_load_2d(kd, &tm_k, h * HD, row, &k_full[buf]);
         tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[buf]);
@@ -167,7 +184,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         umma_commit(s_full);
       };
-      issue_qk(0);
+      if (n_blocks > 0) issue_qk(0);
       for (int i = 0; i < n_blocks; ++i) {
         const int buf = i & 1;
         mbar_wait(p_full, i & 1, p.status);                 // P(i) is in shared memory, S(i) has been read
@@ -205,7 +222,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_wait(s_full, i & 1, p.status);
       tc_fence_after();
       if (dbg && i == 0 && threadIdx.x == 64) p.debug[2] = globaltimer_ns();
-      const int key0 = i * BKV;
+      const int key0 = (z + i * ksplit) * BKV;
       const bool ragged = key0 + BKV > g.kv_len;      // last block: keys past kv_len do not exist
       float mx = m;
       // the other half's 64 scores only matter for the row maximum
@@ -265,22 +282,100 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_arrive(o_free);
     }
     if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
-    // ---- combine the two halves' row sums, normalise, store
+    // ---- combine the two halves' row sums
     l_part[half * BQ + r] = l;
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
-    const float inv = 1.f / (l_part[r] + l_part[BQ + r]);
-    if (r < rows_valid) {
+    const float l_row = l_part[r] + l_part[BQ + r];
+    if (ksplit == 1) {
+      // normalise, store
+      const float inv = 1.f / l_row;
+      if (r < rows_valid) {
+        const int t = p.idx ? p.idx[row0 + r] : row0 + r;
+        __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + half * 64;
+#pragma unroll
+        for (int i = 0; i < 64; ++i) acc[i] *= inv;
+#pragma unroll
+        for (int v = 0; v < 8; ++v) reinterpret_cast<uint4*>(dst)[v] = pack8_bf16(acc + 8 * v);
+      }
+    } else {
+      // key split: leave the un-normalised row, its maximum and its sum in shared memory for the merge
+      asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");      // every l_part read is done
+      float* dump = reinterpret_cast<float*>(smem + S::DUMP_OFF) + (size_t)r * HD;
+#pragma unroll
+      for (int v = 0; v < 16; ++v) {
+        const int unit = half * 16 + v;                  // 32 sixteen-byte units per 512-byte row, XOR-swizzled
+        *reinterpret_cast<float4*>(dump + ((unit ^ (r & 7)) << 2)) =
+            make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+      }
+      if (half == 0) {
+        float* stat = reinterpret_cast<float*>(smem + S::STAT_OFF);
+        stat[r] = m;
+        stat[BQ + r] = l_row;
+      }
+      fence_proxy_async_smem();
+    }
+  }
+  if (ksplit > 1) {
+    // ---- merge of the key split (all warps)
+    __syncthreads();
+    tc_fence_before();
+    cluster_sync_all();                                  // every CTA of the cluster is past its key loop
+    tc_fence_after();
+    if (warp == 2 && lane < ksplit && lane != z) {
+      // hand the rows owned by CTA `lane` to it: the rows, their maxima, their sums
+      const int k = lane;
+      const int slot = z < k ? z : z - 1;
+      const uint32_t slot_bytes = (uint32_t)rows_own * (HD * 4 + 8);
+      const uint32_t dst = map_to_cta(smem_u32(smem + S::RECV_OFF) + slot * slot_bytes, (uint32_t)k);
+      const uint32_t bar = map_to_cta(smem_u32(recv_bar), (uint32_t)k);
+      bulk_copy_to_cta(dst, smem_u32(smem + S::DUMP_OFF + (size_t)k * rows_own * HD * 4), rows_own * HD * 4, bar);
+      bulk_copy_to_cta(dst + rows_own * HD * 4, smem_u32(smem + S::STAT_OFF + k * rows_own * 4), rows_own * 4, bar);
+      bulk_copy_to_cta(dst + rows_own * HD * 4 + rows_own * 4, smem_u32(smem + S::STAT_OFF + (BQ + k * rows_own) * 4),
+                       rows_own * 4, bar);
+    }
+    mbar_wait(recv_bar, 0, p.status);
+    const float c = rsqrtf((float)HD) * 1.4426950408889634f;
+    const float* dump = reinterpret_cast<const float*>(smem + S::DUMP_OFF);
+    const float* stat = reinterpret_cast<const float*>(smem + S::STAT_OFF);
+    const uint32_t slot_floats = (uint32_t)rows_own * (HD + 2);
+    const float* recv = reinterpret_cast<const float*>(smem + S::RECV_OFF);
+    for (int rl = warp; rl < rows_own; rl += kThreads / 32) {
+      const int r = z * rows_own + rl;
+      if (r >= rows_valid) break;
+      float mz[4], lz[4];
+      mz[0] = stat[r]; lz[0] = stat[BQ + r];
+      float mx = mz[0];
+      for (int s2 = 0; s2 < ksplit - 1; ++s2) {
+        const float* sl = recv + s2 * slot_floats;
+        mz[s2 + 1] = sl[rows_own * HD + rl];
+        lz[s2 + 1] = sl[rows_own * HD + rows_own + rl];
+        mx = fmaxf(mx, mz[s2 + 1]);
+      }
+      const int off = ((lane ^ (r & 7)) << 2);           // this lane's 4 columns inside the swizzled row
+      float w = exp2f((mz[0] - mx) * c);
+      float4 o = *reinterpret_cast<const float4*>(dump + (size_t)r * HD + off);
+      o.x *= w; o.y *= w; o.z *= w; o.w *= w;
+      float lsum = w * lz[0];
+      for (int s2 = 0; s2 < ksplit - 1; ++s2) {
+        w = exp2f((mz[s2 + 1] - mx) * c);
+        const float4 a = *reinterpret_cast<const float4*>(recv + s2 * slot_floats + (size_t)rl * HD + off);
+        o.x = fmaf(a.x, w, o.x); o.y = fmaf(a.y, w, o.y); o.z = fmaf(a.z, w, o.z); o.w = fmaf(a.w, w, o.w);
+        lsum = fmaf(w, lz[s2 + 1], lsum);
+      }
+      const float inv = 1.f / lsum;
       const int t = p.idx ? p.idx[row0 + r] : row0 + r;
-      __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + half * 64;
-#pragma unroll
-      for (int i = 0; i < 64; ++i) acc[i] *= inv;
-#pragma unroll
-      for (int v = 0; v < 8; ++v) reinterpret_cast<uint4*>(dst)[v] = pack8_bf16(acc + 8 * v);
+      __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + 4 * lane;
+      __nv_bfloat162 lo2 = __floats2bfloat162_rn(o.x * inv, o.y * inv), hi2 = __floats2bfloat162_rn(o.z * inv, o.w * inv);
+      uint2 packed;
+      packed.x = *reinterpret_cast<uint32_t*>(&lo2);
+      packed.y = *reinterpret_cast<uint32_t*>(&hi2);
+      *reinterpret_cast<uint2*>(dst) = packed;
     }
   }
   }  // active
   tc_fence_before();
-  __syncthreads();
+  // nobody leaves while a copy out of its shared memory may still be in flight (its receiver has seen it land)
+  if (ksplit > 1) cluster_sync_all(); else __syncthreads();
   if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
@@ -294,9 +389,16 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
     attr_set = true;
   }
   const int tps = (p.g.seq_act + BQ - 1) / BQ;
-  dim3 grid(p.g.batch * tps, p.g.n_heads);
-  if (grid.x == 0) return cudaSuccess;
-  return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), AttnSmem::TOTAL, st, 1, tm_k, tm_v, p);
+  // CTAs expected to have work: every row tile (dense) or one row tile per sequence (row-sparse, small refresh set)
+  const int expected = p.g.n_heads * p.g.batch * (p.idx ? 1 : tps);
+  const int n_blocks = (p.g.kv_len + BKV - 1) / BKV;
+  // The merge of a key split costs about as much as four key blocks (three cluster-wide barriers and the copies), so
+  // the keys are split only when every CTA still keeps at least four blocks.
+  int ksplit = 1;
+  while (ksplit < 4 && expected * ksplit * 2 <= 160 && ksplit * 2 * 4 <= n_blocks) ksplit *= 2;
+  dim3 grid(p.g.n_heads, p.g.batch * tps, ksplit);
+  if (grid.y == 0) return cudaSuccess;
+  return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), AttnSmem::TOTAL, st, ksplit, tm_k, tm_v, p);
 }
 
 }  // namespace dare

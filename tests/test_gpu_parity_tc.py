@@ -93,3 +93,25 @@ def test_config2_llada_layer_full_size(dare, config2, n_changed):
         parity.compare_step(g, o, x1, MODES[mode], 0.1, shape)
         np.testing.assert_array_equal(g.last_selection(1, 512)["idx"], np.nonzero(ch.reshape(-1))[0])
     g.close()
+
+
+def test_row_sparse_attention_with_key_split(dare):
+    """Batch 1, 2 heads, 2048 keys, few refreshed rows: the row-sparse attention launch splits the keys over a 4-CTA
+    cluster and merges the partial softmax results over distributed shared memory."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=1, seq=2048, prompt=1024)
+    w = wl.make_weights(shape, 13)
+    hs = wl.HiddenStream(shape, 13)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    for n in (37, 150):
+        ch = wl.uniform_positions(hs.rng, shape, n)
+        parity.compare_step(g, o, hs.advance(ch), 3, 0.1, shape)
+    # a ragged key extent as well: window steps keep kv_len = 2048, so use a second layer with 1990 keys
+    shape2 = wl.scaled(shape, seq=1990, prompt=990)
+    hs2 = wl.HiddenStream(shape2, 14)
+    g2 = dare.Layer(shape2, w, kernel_path=dare.PATH_TENSOR)
+    o2 = parity.oracle_layer(shape2, w)
+    parity.compare_step(g2, o2, hs2.first(), 2, 0.1, shape2, first=True)
+    parity.compare_step(g2, o2, hs2.advance(wl.uniform_positions(hs2.rng, shape2, 70)), 2, 0.1, shape2)
+    g.close(); g2.close()
