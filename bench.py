@@ -445,6 +445,87 @@ def run_micro(args):
     print(json.dumps(out))
 
 
+def run_sweep(args):
+    """Crossover sweep on the long-context layer (batch 4, seq 4096 unless overridden): changed-token fraction
+    0..100 % in 5 % steps, uniform and block-clustered patterns, modes kv / o / both against the dense path of the
+    same library.  Prints one JSON line with the per-point times and the break-even fraction per mode and pattern
+    (linear interpolation between grid points; null = no crossover below 100 %)."""
+    import numpy as np
+    import torch
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare, workloads as wl
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    base = wl.LLADA_LONG
+    shape = wl.scaled(base, batch=args.batch or base.batch, seq=args.seq or base.seq,
+                      prompt=(args.seq or base.seq) // 2)
+    layers = make_layers(shape, 2, shape.seed, torch, dev, dare)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(shape.seed)
+    B, S, d = shape.batch, shape.seq, shape.d_model
+    xa = torch.randn((B, S, d), generator=gen, device=dev).to(torch.bfloat16)
+    y = torch.empty_like(xa)
+    rng = np.random.default_rng(shape.seed)
+
+    def changed_mask(frac, pattern):
+        n = int(round(frac * S))
+        if pattern == "uniform":
+            m = wl.uniform_positions(rng, shape, n) if n else np.zeros((B, S), bool)
+        else:
+            m = wl.clustered_positions(rng, shape, step=4 * 9, clustered_per_seq=n, scattered_per_seq=0)
+        return m
+
+    def time_mode(xb, m, steps=6):
+        for lay in layers:
+            lay.reset()
+            lay.step(xa, m, TAU, y)
+        bufs = (xb, xa)
+        for i in range(2):
+            layers[i % 2].step(bufs[(i // 2) & 1], m, TAU, y)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record()
+        for i in range(2, 2 + steps):
+            layers[i % 2].step(bufs[(i // 2) & 1], m, TAU, y)
+        ev1.record()
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / steps * 1e3      # microseconds per layer step
+
+    fracs = [round(0.05 * i, 2) for i in range(21)]
+    out = {"metric": "us_per_layer_step_vs_changed_fraction", "config": {"workload": shape.name, "batch": B, "seq_len": S,
+           "threshold": TAU, "layers_rotated": 2}, "points": [], "break_even": {}}
+    dense_us = time_mode(xa, 0)
+    out["dense_us"] = round(dense_us, 1)
+    for pattern in ("uniform", "clustered"):
+        curves = {"kv": [], "o": [], "both": []}
+        for f in fracs:
+            mask = torch.from_numpy(changed_mask(f, pattern)).to(dev)
+            noise = torch.randn((B, S, d), generator=gen, device=dev) * 1e-3
+            fresh = torch.randn((B, S, d), generator=gen, device=dev)
+            xb = torch.where(mask[:, :, None], fresh, xa.float() + noise).to(torch.bfloat16)
+            del noise, fresh
+            row = {"pattern": pattern, "changed_fraction": f}
+            for name in ("kv", "o", "both"):
+                us = time_mode(xb, MODES[name])
+                sel = layers[0].last_selection(B, S)
+                assert sel["count"] == int(mask.sum().item()), (pattern, f, name, sel["count"])
+                row[name + "_us"] = round(us, 1)
+                curves[name].append(us)
+            out["points"].append(row)
+        for name, ys in curves.items():
+            be = None
+            for i in range(len(fracs) - 1):
+                a, b_ = ys[i] - dense_us, ys[i + 1] - dense_us
+                if a <= 0 < b_:
+                    be = round(fracs[i] + (fracs[i + 1] - fracs[i]) * (-a) / (b_ - a), 3)
+                    break
+            if be is None and ys[0] > dense_us:
+                be = 0.0
+            out["break_even"][f"{pattern}/{name}"] = be
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -458,9 +539,12 @@ def main():
     ap.add_argument("--d-model", type=int, default=0, help="exploration: other layer width (multiple of 128)")
     ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
     ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
+    ap.add_argument("--sweep", action="store_true", help="long-context crossover sweep (config 5) instead")
     ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
     args = ap.parse_args()
-    if args.micro:
+    if args.sweep:
+        run_sweep(args)
+    elif args.micro:
         run_micro(args)
     elif args.impl == "reference":
         run_reference(args)

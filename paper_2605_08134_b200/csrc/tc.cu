@@ -134,13 +134,18 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     if (kv_sparse) {
       p.idx = B.idx; p.count = B.count;
       const int m_tiles = (T_ + 127) / 128;
-      // The refresh set is expected to be small, which makes this projection a stream of the weights: narrower
-      // tiles put twice as many CTAs on it; the reduction split is sized for one row tile.
-      p.n_split = d / 128;
-      const int n_tiles128 = 2 * d / 128;
       prof_mark(L, SLOT_KV_GEMM, st);
-      e = launch_gemm_tc(EPI_KV, 128, S.a_xg, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
-                         pick_splits(n_tiles128, kblocks), st); ++launches;
+      if (m_tiles <= 8) {
+        // Few tokens: the refresh set fits one or two row tiles and the projection is a stream of the weights.
+        // Narrower tiles put twice as many CTAs on it; the reduction split is sized for one row tile.
+        p.n_split = d / 128;
+        const int n_tiles128 = 2 * d / 128;
+        e = launch_gemm_tc(EPI_KV, 128, S.a_xg, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
+                           pick_splits(n_tiles128, kblocks), st); ++launches;
+      } else {
+        // Many tokens: even a small refreshed fraction fills the GPU with full-rate 256-wide tiles.
+        e = launch_gemm_tc(EPI_KV, 256, S.a_xg, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st); ++launches;
+      }
     } else {
       prof_mark(L, SLOT_KV_GEMM, st);
       e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense,

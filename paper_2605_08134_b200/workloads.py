@@ -107,14 +107,18 @@ def clustered_positions(rng, shape: LayerShape, step: int, clustered_per_seq: in
 
     A contiguous run of `clustered_per_seq` positions starts at the first position of the active
     block (block index = step // steps_per_block, wrapping inside the generation region; a run
-    that would pass the end of the sequence wraps to the start of the generation region) plus
+    that would pass the end of the sequence wraps to the start of the generation region, and one
+    longer than the generation region wraps over the whole sequence) plus
     `scattered_per_seq` positions uniform over the remaining ones.  -> bool [B, S].
     """
     gen = shape.seq - shape.prompt
     n_blocks = max(1, gen // shape.block)
     start = ((step // steps_per_block) % n_blocks) * shape.block
     m = np.zeros((shape.batch, shape.seq), bool)
-    run = shape.prompt + (start + np.arange(clustered_per_seq)) % gen
+    if clustered_per_seq <= gen:
+        run = shape.prompt + (start + np.arange(clustered_per_seq)) % gen
+    else:       # a run longer than the generation region goes on through the whole sequence
+        run = (shape.prompt + start + np.arange(clustered_per_seq)) % shape.seq
     for b in range(shape.batch):
         m[b, run] = True
         rest = np.nonzero(~m[b])[0]
