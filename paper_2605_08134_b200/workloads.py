@@ -173,3 +173,44 @@ def two_step_case(shape: LayerShape, changed_per_seq: int, seed: int | None = No
     changed = uniform_positions(hs.rng, shape, changed_per_seq)
     x1 = hs.advance(changed)
     return w, x0, x1, changed
+
+
+@dataclass(frozen=True)
+class StackShape:
+    """A stack of DARE attention layers inside pre-norm SwiGLU blocks (config 4 geometry or a reduced copy)."""
+    name: str
+    n_layers: int
+    layer: LayerShape          # attention geometry; layer.seq = prompt + generation length, layer.prompt = prompt
+    d_ff: int
+    vocab: int
+    gen_len: int
+    seed: int = 3
+
+    @property
+    def mask_id(self) -> int:
+        return self.vocab - 1
+
+
+LLADA_STACK = StackShape("llada8b_stack_32l", 32, scaled(LLADA_LAYER, name="llada8b_stack_layer", seed=3),
+                         12288, 126464, 256)
+
+
+def make_stack_weights(shape: StackShape, seed: int | None = None, std: float = 0.02) -> dict:
+    """All matrices ~ N(0, std^2) rounded to the storage type, gains 1: embedding [V, d], untied head [V, d], and per
+    layer W_Q, W_K, W_V, W_O [d, d], W_gate, W_up [d_ff, d], W_down [d, d_ff]."""
+    s = shape.seed if seed is None else seed
+    rng = np.random.default_rng(s + 104729)
+    lay, d, f = shape.layer, shape.layer.d_model, shape.d_ff
+    draw = lambda *dims: round_to(rng.standard_normal(dims, dtype=np.float32) * np.float32(std), lay.dtype)
+    w = {"emb": draw(shape.vocab, d), "head": draw(shape.vocab, d), "final_gain": np.ones(d, np.float32), "layers": []}
+    for _ in range(shape.n_layers):
+        w["layers"].append({"w_q": draw(d, d), "w_k": draw(d, d), "w_v": draw(d, d), "w_o": draw(d, d),
+                            "rms_gain": np.ones(d, np.float32), "gain2": np.ones(d, np.float32),
+                            "w_gate": draw(f, d), "w_up": draw(f, d), "w_down": draw(d, f)})
+    return w
+
+
+def random_prompt(shape: StackShape, batch: int, seed: int | None = None) -> np.ndarray:
+    """`prompt` random token ids per sequence, never the mask id."""
+    rng = np.random.default_rng((shape.seed if seed is None else seed) + 31)
+    return rng.integers(0, shape.vocab - 1, size=(batch, shape.layer.prompt), dtype=np.int32)
