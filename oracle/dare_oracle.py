@@ -171,12 +171,16 @@ class OracleLayer:
         self.last_idx = None
         self.last_batch_off = None
 
-    def step(self, x, mode, tau, pos_begin=0):
+    def step(self, x, mode, tau, pos_begin=0, adopt=None):
         """One denoising step.  x: [batch, seq_act, d] covering positions
         [pos_begin, pos_begin + seq_act) of every sequence.  Returns y of the same shape.
 
         Side outputs kept on the object: last_scores [batch*seq_act], last_idx (ascending
         flat indices b*seq_act + i of refreshed tokens), last_batch_off [batch+1].
+
+        adopt = (other_mask [batch*seq_act] bool, margin): for comparisons with another implementation inside a
+        long trajectory.  A token whose score lies within `margin` of tau has no well-defined side; there, and only
+        there, the other implementation's decision is taken, so that both keep walking the same trajectory.
         """
         x = np.asarray(x, _F)
         B, S_act, d = x.shape
@@ -208,6 +212,10 @@ class OracleLayer:
             sel = np.ones(T, bool)          # nothing to compare with, or dense recompute asked for
         else:
             sel = refresh_mask(scores, tau)
+            if adopt is not None and self.has_prev:
+                other, margin = adopt
+                near = np.abs(scores - tau) < margin
+                sel = np.where(near, np.asarray(other, bool), sel)
         idx = np.nonzero(sel)[0]
 
         # Sec. 3.2: the stored query is that of the immediately previous step, for every token.

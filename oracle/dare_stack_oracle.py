@@ -61,16 +61,16 @@ class OracleStack:
         for l in self.layers:
             l.reset()
 
-    def forward(self, tokens, pos_begin, mode, taus, keep_inputs=False):
+    def forward(self, tokens, pos_begin, mode, taus, keep_inputs=False, adopt=None):
         """tokens: int [B, S_act] at positions [pos_begin, pos_begin+S_act).  Returns the final-normed hidden states
-        [B, S_act, d].  taus: one threshold per layer."""
+        [B, S_act, d].  taus: one threshold per layer.  adopt: per layer, the (mask, margin) of OracleLayer.step."""
         tokens = np.asarray(tokens)
         x = self.emb[tokens]
         self.layer_inputs = [] if keep_inputs else None
         for l, (layer, lw) in enumerate(zip(self.layers, self.lw)):
             if keep_inputs:
                 self.layer_inputs.append(x.copy())
-            a = layer.step(x, mode, taus[l], pos_begin=pos_begin)
+            a = layer.step(x, mode, taus[l], pos_begin=pos_begin, adopt=None if adopt is None else adopt[l])
             h = x + a
             n = orc.rmsnorm(h, lw["gain2"], self.eps)
             x = h + swiglu_mlp(n, lw["w_gate"], lw["w_up"], lw["w_down"])

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdare.so")
-SOURCES = ["api.cu", "common.cu", "simt.cu", "tc.cu", "gemm_tc.cu", "attn_tc.cu", "select_large.cu"]
+SOURCES = ["api.cu", "common.cu", "simt.cu", "tc.cu", "gemm_tc.cu", "attn_tc.cu", "select_large.cu", "stack.cu"]
 
 
 def _newest(paths):
@@ -19,7 +19,8 @@ def _newest(paths):
 def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "dare.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if not f.endswith(".o")] + \
+        [os.path.join(ROOT, "include", h) for h in os.listdir(os.path.join(ROOT, "include"))]
     return _newest(deps) > os.path.getmtime(LIB)
 
 

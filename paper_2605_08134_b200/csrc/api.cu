@@ -156,14 +156,14 @@ dare_status_t validate_step(dare_layer_t* L, const void* x, int batch, int seq_a
 }
 
 dare_status_t enqueue_step(dare_layer_t* L, const void* x, int batch, int seq_act, int pos_begin, int mode, float tau,
-                           void* y, cudaStream_t st) {
+                           void* y, cudaStream_t st, bool add_input = false) {
   StepGeom g;
   g.batch = batch; g.seq_act = seq_act; g.pos_begin = pos_begin; g.max_seq = L->cfg.max_seq;
   g.kv_len = L->has_prev ? L->kv_len : seq_act;
   g.d = L->cfg.d_model; g.n_heads = L->cfg.n_heads; g.head_dim = L->cfg.head_dim; g.score_head = L->cfg.score_head;
   dare_status_t s;
   if (L->use_tc) {
-    s = step_tc(L, x, g, mode, tau, y, st);
+    s = step_tc(L, x, g, mode, tau, y, st, add_input);
   } else if (L->cfg.dtype == DARE_BF16) {
     s = step_simt<__nv_bfloat16>(L, (const __nv_bfloat16*)x, g, mode, tau, (__nv_bfloat16*)y, st);
   } else {
@@ -177,6 +177,18 @@ dare_status_t enqueue_step(dare_layer_t* L, const void* x, int batch, int seq_ac
 }
 
 }  // namespace
+
+namespace dare {
+// The layer step for callers inside the library (the stack): same validation as dare_layer_step; add_input makes the
+// output x + W_O O (tensor-core path only).
+dare_status_t layer_enqueue(dare_layer* L, const void* x, int batch, int seq_act, int pos_begin, int mode, float tau,
+                            void* y, cudaStream_t st, bool add_input) {
+  dare_status_t s = validate_step(L, x, batch, seq_act, pos_begin, mode, tau, y);
+  if (s != DARE_OK) return s;
+  if (add_input && !L->use_tc) return DARE_ERR_UNSUPPORTED;
+  return enqueue_step(L, x, batch, seq_act, pos_begin, mode, tau, y, st, add_input);
+}
+}  // namespace dare
 
 extern "C" {
 

@@ -76,10 +76,9 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
                                                       T* __restrict__ xn, int d, float eps) {
   constexpr int N = Vec16<T>::N;
   __shared__ float red[32];
-  // This kernel reads only the step's input and writes x_norm, which no kernel still running can be reading (the
-  // launch is released by the previous kernel only after that kernel has seen all of its own predecessors finish).
-  // So it works right away, under the previous kernel's tail, and waits for that kernel only before it exits,
-  // which keeps "kernel N done => kernels < N done" true along the stream.
+  // x may be the output of the previous kernel in the stream (the previous layer of a model), so it is read only
+  // after that kernel has completed.
+  ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const size_t row = blockIdx.x;
   const T* xr = x + row * d;
@@ -131,7 +130,6 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     for (int e = 0; e < N; ++e) t[e] = t[e] * r * gain[vi * N + e];
     Vec16<T>::store(yr + vi * N, t);
   }
-  ptx::pdl_wait();
 }
 
 template <typename T>

@@ -17,7 +17,9 @@
 //   Q    drift score of the scoring head against the stored query (Sec. 3.1), store of the new query, rotary
 //        embedding, bf16 store
 //   K/V  rotary embedding of K, scatter of both rows into the caches at the refresh-set rows (Eq. 3)
-//   OUT  plain bf16 store of y
+//   OUT  bf16 store of y, optionally plus a residual row
+//   SWIGLU  silu(gate) * up of a tile that holds both projections of the same 128 outputs (MLP of a stack)
+//   F32  fp32 store (logits of a stack's LM head)
 #include "layer.h"
 #include "tc.h"
 #include "tc_ptx.cuh"
@@ -49,6 +51,7 @@ struct Cfg {
 constexpr int RB = 6;
 struct RowBatch {
   int tok[RB];
+  int row[RB];            // place of the row in the launch's (possibly gathered) row list
   size_t crow[RB];
   bool ok[RB];
   float4 cs[RB];          // (cos, sin) of the two rotary pairs this lane owns
@@ -65,6 +68,7 @@ __device__ __forceinline__ void load_row_batch(RowBatch& rb, const GemmParams& p
     const int r = z * rows_per_cta + rl;
     rb.ok[k] = rl < rows_per_cta && r < rows_valid;
     const int rc = rb.ok[k] ? r : 0;              // rows that do not exist read row 0's tables and are dropped later
+    rb.row[k] = t0 + rc;
     int pos;
     if (p.idx) {
       rb.tok[k] = p.idx[t0 + rc];
@@ -109,8 +113,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
   // ---- which columns?  Tiles [0, n_split) belong to W0/out0, the rest to W1/out1.
-  const bool is_b1 = nt >= p.n_split;
-  const int n0 = (is_b1 ? nt - p.n_split : nt) * BN;
+  const bool is_b1 = !p.b_pair && nt >= p.n_split;
+  const int n0 = p.b_pair ? nt * (BN / 2) : (is_b1 ? nt - p.n_split : nt) * BN;   // first output column / W row
   const CUtensorMap* tm_b = is_b1 ? &tm_b1 : &tm_b0;
   // ---- which slice of the reduction?
   const int KB = p.K / BK;
@@ -147,7 +151,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
       mbar_arrive_expect_tx(&full_bar[i], STAGE_BYTES);
-      tma_load_2d(smem + i * STAGE_BYTES + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[i]);
+      uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
+      if (p.b_pair) {
+        tma_load_2d(b_dst, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[i]);
+        tma_load_2d(b_dst + Cfg<BN>::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[i]);
+      } else {
+        tma_load_2d(b_dst, tm_b, (kb_begin + i) * BK, n0, &full_bar[i]);
+      }
     }
   }
   pdl_wait();
@@ -193,7 +203,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         uint8_t* a_dst = smem + s * STAGE_BYTES;
         mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
         tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
-        tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
+        if (p.b_pair) {
+          tma_load_2d(a_dst + A_BYTES, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[s]);
+          tma_load_2d(a_dst + A_BYTES + Cfg<BN>::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[s]);
+        } else {
+          tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
+        }
       }
     }
     __syncwarp();
@@ -351,11 +366,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           p.scores[my_tok] = sc;
         }
       }
-      // (3) rotary embedding and bf16 store
+      // (3) the projection's own tail and the store
 #pragma unroll
       for (int k = 0; k < RB; ++k) {
         if (!rb.ok[k]) continue;
-        const size_t orow = p.out_is_cache ? rb.crow[k] : (size_t)rb.tok[k];
+        const size_t orow = p.out_is_cache == 1 ? rb.crow[k] : (p.out_is_cache == 2 ? (size_t)rb.row[k] : (size_t)rb.tok[k]);
+        if (EPI == EPI_SWIGLU) {
+          // columns [0, 128) of a 256-wide tile are the gate, [128, 256) the up projection of the same 128 outputs
+          const float2 g_lo = vlo[k][0], g_hi = vhi[k][0], u_lo = vlo[k][BN / HD - 1], u_hi = vhi[k][BN / HD - 1];
+          __nv_bfloat16* dst = out + orow * p.ld_out + n0;
+          auto act = [](float g, float u) { return g / (1.f + __expf(-g)) * u; };
+          *reinterpret_cast<__nv_bfloat162*>(dst + 2 * lane) = __floats2bfloat162_rn(act(g_lo.x, u_lo.x), act(g_lo.y, u_lo.y));
+          *reinterpret_cast<__nv_bfloat162*>(dst + HD / 2 + 2 * lane) =
+              __floats2bfloat162_rn(act(g_hi.x, u_hi.x), act(g_hi.y, u_hi.y));
+          continue;
+        }
         __nv_bfloat16* dst = out + orow * p.ld_out + n0;
 #pragma unroll
         for (int hh = 0; hh < BN / HD; ++hh) {
@@ -365,6 +390,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const float a0 = lo.x, b0 = hi.x, a1 = lo.y, b1 = hi.y;
             lo.x = a0 * rb.cs[k].x - b0 * rb.cs[k].y; hi.x = a0 * rb.cs[k].y + b0 * rb.cs[k].x;
             lo.y = a1 * rb.cs[k].z - b1 * rb.cs[k].w; hi.y = a1 * rb.cs[k].w + b1 * rb.cs[k].z;
+          }
+          if (EPI == EPI_F32) {
+            float* d32 = p.out_f32 + orow * p.ld_out + n0;
+            *reinterpret_cast<float2*>(d32 + c_lo) = lo;
+            *reinterpret_cast<float2*>(d32 + c_hi) = hi;
+            continue;
+          }
+          if (EPI == EPI_OUT && p.resid != nullptr) {
+            const __nv_bfloat16* rs = p.resid + (size_t)rb.tok[k] * p.ld_resid + n0;
+            const float2 ra = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(rs + c_lo));
+            const float2 rb2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(rs + c_hi));
+            lo.x += ra.x; lo.y += ra.y; hi.x += rb2.x; hi.y += rb2.y;
           }
           *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = __floats2bfloat162_rn(lo.x, lo.y);
           *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = __floats2bfloat162_rn(hi.x, hi.y);
@@ -408,6 +445,8 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
   if (bn == 256) {
     if (epi == EPI_Q) return launch_one<EPI_Q, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_KV) return launch_one<EPI_KV, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_F32) return launch_one<EPI_F32, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     return launch_one<EPI_OUT, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
   }
   if (bn == 128 && epi == EPI_KV) return launch_one<EPI_KV, 128>(a, b0, b1, p, n_tiles, m_tiles, splits, st);

@@ -73,5 +73,7 @@ inline void prof_end(dare_layer* L, cudaStream_t st) {
 }
 dare_status_t tc_create(dare_layer* L);
 void tc_destroy(dare_layer* L);
-dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode, float tau, void* y, cudaStream_t st);
+// add_input: y = x + W_O O instead of y = W_O O (the residual connection of a transformer block)
+dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode, float tau, void* y, cudaStream_t st,
+                      bool add_input = false);
 }  // namespace dare

@@ -31,6 +31,16 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Reduction splits for a launch with `tiles` output tiles: enough CTAs to cover the SMs, never more than the
+// k-blocks or the scratch allow.
+int pick_splits(int tiles, int kblocks) {
+  int s = 1;
+  while (s < 2 && tiles * s * 2 <= 160 && s * 2 <= kblocks) s *= 2;
+  return s;
+}
+
+}  // namespace
+
 // Row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes, the swizzle span) x box_rows rows.
 bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   EncodeTiledFn fn = encode_fn();
@@ -44,16 +54,6 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
-
-// Reduction splits for a launch with `tiles` output tiles: enough CTAs to cover the SMs, never more than the
-// k-blocks or the scratch allow.
-int pick_splits(int tiles, int kblocks) {
-  int s = 1;
-  while (s < 2 && tiles * s * 2 <= 160 && s * 2 <= kblocks) s *= 2;
-  return s;
-}
-
-}  // namespace
 
 bool tc_supported(const dare_layer_config_t& c) {
   return c.dtype == DARE_BF16 && c.head_dim == 128 && c.d_model % 256 == 0;
@@ -80,7 +80,8 @@ void tc_destroy(dare_layer* L) {
   L->tc = nullptr;
 }
 
-dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode, float tau, void* y, cudaStream_t st) {
+dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode, float tau, void* y, cudaStream_t st,
+                      bool add_input) {
   typedef __nv_bfloat16 bf16;
   const Buffers& B = L->buf;
   const TcState& S = *L->tc;
@@ -98,7 +99,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
   base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
-  base.out_is_cache = 0; base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
+  base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
+  base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
   base.debug = nullptr;
   unsigned long long* dbg = L->debug_on ? B.debug : nullptr;
@@ -168,6 +170,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     GemmParams p = base;
     p.a_seq_stride = g.max_seq; p.a_row0 = g.pos_begin;
     p.out0 = (bf16*)y;
+    if (add_input) { p.resid = (const bf16*)x; p.ld_resid = d; }      // y = x + W_O O (residual block)
     p.debug = dbg ? dbg + 24 : nullptr;
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_OUT_GEMM, st);

@@ -7,7 +7,7 @@
 
 namespace dare {
 
-enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2 };
+enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2, EPI_SWIGLU = 3, EPI_F32 = 4 };
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
@@ -23,7 +23,13 @@ struct GemmParams {
   __nv_bfloat16* out0;
   __nv_bfloat16* out1;
   int ld_out;
-  int out_is_cache;      // output rows addressed by cache row (1) or by flat token index (0)
+  int out_is_cache;      // output rows addressed by cache row (1), by flat token index (0), or by the row's place
+                         // in the gathered list (2)
+  const __nv_bfloat16* resid;  // EPI_OUT: rows added to the result (indexed like a token-addressed output), or nullptr
+  int ld_resid;
+  float* out_f32;        // EPI_F32: fp32 output instead of out0
+  int b_pair;            // the W tile is BN/2 rows of W0 followed by BN/2 rows of W1, both at row nt*BN/2 (EPI_SWIGLU:
+                         // gate and up projections of the same BN/2 outputs)
   const float2* rope;    // rotary table [max_seq][head_dim/2]
   float* q_prev;         // stored scoring-head query [cache rows][head_dim], fp32
   float* scores;
@@ -48,6 +54,9 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
 // grid = (n_tiles of bn columns, m_tiles of 128 rows, splits of the reduction dimension = cluster size: 1 or 2);
 // bn = 256 (full tensor rate) or 128 (more CTAs for the weight-streaming K/V projection of a small refresh set).
 // The W tensor maps must have a box of bn rows.
+// Row-major bf16 matrix [rows, cols] as a TMA tensor map with a box of 64 columns x box_rows rows, 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                            const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st);
 

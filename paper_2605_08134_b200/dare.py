@@ -30,6 +30,21 @@ class LayerWeights(C.Structure):
                 ("rms_gain", C.c_void_p)]
 
 
+class StackConfig(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("n_layers", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32),
+                ("mask_id", C.c_int32), ("block", C.c_int32), ("layer", LayerConfig)]
+
+
+class BlockWeights(C.Structure):
+    _fields_ = [("attn", LayerWeights), ("gain2", C.c_void_p), ("w_gate", C.c_void_p), ("w_up", C.c_void_p),
+                ("w_down", C.c_void_p)]
+
+
+class StackWeights(C.Structure):
+    _fields_ = [("emb", C.c_void_p), ("head", C.c_void_p), ("final_gain", C.c_void_p),
+                ("blocks_host", C.POINTER(BlockWeights))]
+
+
 class DareError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -61,6 +76,14 @@ def _load():
         "dare_layer_set_profiling": (C.c_int, [vp, i32]),
         "dare_layer_last_kernel_times": (C.c_int, [vp, vp, vp, i32, C.POINTER(C.c_int)]),
         "dare_kernel_slot_name": (C.c_char_p, [C.c_int]),
+        "dare_stack_workspace_bytes": (sz, [C.POINTER(StackConfig)]),
+        "dare_stack_create": (C.c_int, [C.POINTER(StackConfig), C.POINTER(StackWeights), vp, sz, C.POINTER(vp)]),
+        "dare_stack_reset": (C.c_int, [vp]),
+        "dare_stack_destroy": (C.c_int, [vp]),
+        "dare_stack_layer": (vp, [vp, i32]),
+        "dare_stack_forward": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]),
+        "dare_stack_last_hidden": (C.c_int, [vp, vp, sz, vp]),
+        "dare_stack_decode_step": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
         "dare_layer_debug_timestamps": (C.c_int, [vp, i32, vp, vp]),
         "dare_drift_scores": (C.c_int, [vp, vp, C.c_int64, i32, vp, vp]),
         "dare_select_compact_scratch_bytes": (sz, [C.c_int64]),
@@ -187,6 +210,47 @@ def dare_select_compact_static(scores_ptr, n_tokens, threshold, idx_ptr, count_p
 
 def dare_kernel_slot_name(slot: int) -> str:
     return _lib.dare_kernel_slot_name(slot).decode()
+
+
+def dare_stack_workspace_bytes(cfg: StackConfig) -> int:
+    return _lib.dare_stack_workspace_bytes(C.byref(cfg))
+
+
+def dare_stack_create(cfg: StackConfig, weights: StackWeights, workspace_ptr: int, workspace_bytes: int):
+    """-> (status, handle)"""
+    out = C.c_void_p()
+    st = _lib.dare_stack_create(C.byref(cfg), C.byref(weights), workspace_ptr, workspace_bytes, C.byref(out))
+    return st, out.value
+
+
+def dare_stack_reset(handle) -> int:
+    return _lib.dare_stack_reset(handle)
+
+
+def dare_stack_destroy(handle) -> int:
+    return _lib.dare_stack_destroy(handle)
+
+
+def dare_stack_layer(handle, index: int):
+    return _lib.dare_stack_layer(handle, index)
+
+
+def dare_stack_forward(handle, tokens_ptr, batch, seq_total, seq_act, pos_begin, mode, taus_host_ptr, hidden_ptr,
+                       stream=0) -> int:
+    return _lib.dare_stack_forward(handle, tokens_ptr, batch, seq_total, seq_act, pos_begin, mode, taus_host_ptr,
+                                   hidden_ptr, stream)
+
+
+def dare_stack_last_hidden(handle, dst_host_ptr, nbytes, stream=0) -> int:
+    return _lib.dare_stack_last_hidden(handle, dst_host_ptr, nbytes, stream)
+
+
+def dare_stack_decode_step(handle, tokens_ptr, batch, seq_total, prompt_len, block_index, first, mode, taus_host_ptr,
+                           forced_pos_host_ptr, forced_tok_host_ptr, pos_out_ptr, tok_out_ptr, prob_out_ptr,
+                           stream=0) -> int:
+    return _lib.dare_stack_decode_step(handle, tokens_ptr, batch, seq_total, prompt_len, block_index, first, mode,
+                                       taus_host_ptr, forced_pos_host_ptr, forced_tok_host_ptr, pos_out_ptr,
+                                       tok_out_ptr, prob_out_ptr, stream)
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -316,6 +380,119 @@ class Layer:
     def close(self):
         if getattr(self, "handle", None):
             dare_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class _LayerView(Layer):
+    """A layer that belongs to a stack: same observation calls, no ownership."""
+
+    def __init__(self, handle, shape, torch, device):
+        self.handle, self.shape, self.torch, self.device = handle, shape, torch, device
+        self.tdtype = torch.bfloat16
+
+    def close(self):
+        self.handle = None
+
+
+class Stack:
+    """Convenience wrapper around dare_stack_*: owns the device copies of the weights and the workspace."""
+
+    def __init__(self, sshape, weights: dict, batch: int, device="cuda:0"):
+        import numpy as np
+        import torch
+        self.torch, self.sshape, self.batch = torch, sshape, batch
+        self.device = torch.device(device)
+        lay = sshape.layer
+        dev = lambda a, dt: (a if isinstance(a, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(a, np.float32))) \
+            .to(self.device, dt).contiguous()
+        bf, f32 = torch.bfloat16, torch.float32
+        self._keep = [dev(weights["emb"], bf), dev(weights["head"], bf), dev(weights["final_gain"], f32)]
+        blocks = (BlockWeights * sshape.n_layers)()
+        for l, lw in enumerate(weights["layers"]):
+            t = {k: dev(lw[k], bf) for k in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down")}
+            t["rms_gain"], t["gain2"] = dev(lw["rms_gain"], f32), dev(lw["gain2"], f32)
+            self._keep.append(t)
+            blocks[l] = BlockWeights(LayerWeights(t["w_q"].data_ptr(), t["w_k"].data_ptr(), t["w_v"].data_ptr(),
+                                                  t["w_o"].data_ptr(), t["rms_gain"].data_ptr()),
+                                     t["gain2"].data_ptr(), t["w_gate"].data_ptr(), t["w_up"].data_ptr(),
+                                     t["w_down"].data_ptr())
+        self._blocks = blocks
+        lcfg = make_config(lay.d_model, lay.n_heads, lay.head_dim, batch, lay.seq, lay.rope_theta, lay.rms_eps, BF16, 0,
+                           PATH_TENSOR)
+        self.cfg = StackConfig(C.sizeof(StackConfig), sshape.n_layers, sshape.d_ff, sshape.vocab, sshape.mask_id,
+                               lay.block, lcfg)
+        self.w = StackWeights(self._keep[0].data_ptr(), self._keep[1].data_ptr(), self._keep[2].data_ptr(), blocks)
+        nbytes = dare_stack_workspace_bytes(self.cfg)
+        if nbytes == 0:
+            raise DareError(ERR_UNSUPPORTED, "dare_stack_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        with torch.cuda.device(self.device):
+            st, self.handle = dare_stack_create(self.cfg, self.w, base, nbytes)
+        if st != OK:
+            raise DareError(st, "dare_stack_create")
+
+    def _stream(self):
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def layer(self, index: int) -> "_LayerView":
+        return _LayerView(dare_stack_layer(self.handle, index), self.sshape.layer, self.torch, self.device)
+
+    def reset(self):
+        dare_stack_reset(self.handle)
+
+    def forward(self, tokens, seq_act, pos_begin, mode, taus):
+        """tokens: int32 CUDA tensor [batch, seq_total]; -> bf16 hidden states [batch, seq_act, d_model]."""
+        import numpy as np
+        torch = self.torch
+        taus = np.ascontiguousarray(taus, np.float32)
+        out = torch.empty((tokens.shape[0], seq_act, self.sshape.layer.d_model), dtype=torch.bfloat16, device=self.device)
+        st = dare_stack_forward(self.handle, tokens.data_ptr(), tokens.shape[0], tokens.shape[1], seq_act, pos_begin, mode,
+                                taus.ctypes.data, out.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_stack_forward")
+        return out
+
+    def decode_step(self, tokens, prompt_len, block_index, first, mode, taus, forced=None):
+        """-> (pos, tok, prob) numpy arrays [batch]: the step's own choice; `tokens` is updated in place."""
+        import numpy as np
+        torch = self.torch
+        B = tokens.shape[0]
+        taus = np.ascontiguousarray(taus, np.float32)
+        pos = torch.empty(B, dtype=torch.int32, device=self.device)
+        tok = torch.empty(B, dtype=torch.int32, device=self.device)
+        prob = torch.empty(B, dtype=torch.float32, device=self.device)
+        fp = ft = None
+        if forced is not None:
+            fp = np.ascontiguousarray(forced[0], np.int32)
+            ft = np.ascontiguousarray(forced[1], np.int32)
+        st = dare_stack_decode_step(self.handle, tokens.data_ptr(), B, tokens.shape[1], prompt_len, block_index,
+                                    1 if first else 0, mode, taus.ctypes.data,
+                                    fp.ctypes.data if fp is not None else None, ft.ctypes.data if ft is not None else None,
+                                    pos.data_ptr(), tok.data_ptr(), prob.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_stack_decode_step")
+        torch.cuda.synchronize(self.device)       # the forced arrays are host memory read by an async copy
+        return pos.cpu().numpy(), tok.cpu().numpy(), prob.cpu().numpy()
+
+    def last_hidden(self, batch, seq_act):
+        """-> float32 numpy [batch, seq_act, d_model]: final-normed states of the last pass."""
+        torch = self.torch
+        h = torch.empty((batch, seq_act, self.sshape.layer.d_model), dtype=torch.bfloat16)
+        st = dare_stack_last_hidden(self.handle, h.data_ptr(), h.numel() * 2, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_stack_last_hidden")
+        return h.float().numpy()
+
+    def close(self):
+        if getattr(self, "handle", None):
+            dare_stack_destroy(self.handle)
             self.handle = None
 
     def __del__(self):

@@ -1,0 +1,120 @@
+"""Config 4 on a scaled-down stack: the whole decoding trajectory on the GPU against the stack oracle, step by step,
+teacher-forced (the oracle adopts the GPU's token choice, and the GPU's refresh decision for the few tokens whose
+score lies within the margin of tau, so that both walk the same trajectory and every step is a fresh comparison)."""
+import numpy as np
+import pytest
+
+from oracle import dare_stack_oracle as sto
+from paper_2605_08134_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+MARGIN = 5e-3       # bf16 scores are good to a few 1e-3 (see parity.SCORE_ATOL)
+
+
+@pytest.fixture(scope="module")
+def dare():
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare as d
+    return d
+
+
+def small_stack(L=4, d=256, H=2, d_ff=768, vocab=1024, prompt=64, gen=64, batch=2):
+    lay = wl.scaled(wl.LLADA_LAYER, name="small_stack_layer", d_model=d, n_heads=H, seq=prompt + gen, prompt=prompt,
+                    batch=batch, seed=3)
+    return wl.StackShape("small_stack", L, lay, d_ff, vocab, gen, seed=3)
+
+
+def oracle_stack(shape, w, batch):
+    lay = shape.layer
+    return sto.OracleStack(shape.n_layers, lay.d_model, lay.n_heads, lay.head_dim, shape.d_ff, shape.vocab, batch,
+                           lay.seq, lay.rope_theta, lay.rms_eps, w)
+
+
+@pytest.mark.parametrize("mode", [3, 1])
+def test_small_stack_decoding_trajectory(dare, mode):
+    import torch
+    shape = small_stack()
+    lay = shape.layer
+    B, P, S = 2, lay.prompt, lay.seq
+    w = wl.make_stack_weights(shape)
+    taus = [0.1] * shape.n_layers
+    g = dare.Stack(shape, w, B)
+    o = oracle_stack(shape, w, B)
+    prompt = wl.random_prompt(shape, B)
+    toks_np = np.concatenate([prompt, np.full((B, shape.gen_len), shape.mask_id, np.int32)], axis=1)
+    toks = torch.from_numpy(toks_np.copy()).cuda()
+    agree = 0
+    steps = 0
+    for blk in range(shape.gen_len // lay.block):
+        lo, hi = P + blk * lay.block, P + (blk + 1) * lay.block
+        for _ in range(lay.block):
+            first = steps == 0
+            pos_begin = 0 if first else P
+            S_act = S - pos_begin
+            before = toks_np.copy()
+            gpos, gtok, gprob = g.decode_step(toks, P, blk, first, mode, taus)
+            # the GPU's refresh decisions, per layer, as masks for the oracle to adopt inside the margin
+            adopt = []
+            gsel = []
+            for l in range(shape.n_layers):
+                sel = g.layer(l).last_selection(B, S_act)
+                m = np.zeros(B * S_act, bool); m[sel["idx"]] = True
+                adopt.append((m, MARGIN)); gsel.append(sel)
+            hid = o.forward(before[:, pos_begin:], pos_begin, mode, taus, adopt=adopt)
+            # (1) refresh sets: identical wherever the oracle's score is clear of tau
+            for l in range(shape.n_layers):
+                ol = o.layers[l]
+                np.testing.assert_array_equal(gsel[l]["idx"], ol.last_idx, err_msg=f"step {steps} layer {l}")
+                if not first:
+                    clear = np.abs(ol.last_scores - taus[l]) >= MARGIN
+                    np.testing.assert_allclose(gsel[l]["scores"][clear], ol.last_scores[clear], rtol=0, atol=MARGIN)
+            # (2) final hidden states of the active rows
+            # The states have passed through L layers (each with the bf16 cache roundings that tests/parity.py
+            # describes) and a final normalisation to RMS 1: the max-abs gate is the caches' (2 x) times sqrt(L); the
+            # RMS gate stays at the plain 2e-2.
+            parity.assert_close(f"hidden step {steps}", g.last_hidden(B, S_act), hid, parity.TOL_BF16,
+                                max_factor=2.0 * np.sqrt(shape.n_layers))
+            # (3) the choice: the GPU's (position, token) must be (near-)optimal under the oracle's probabilities
+            for b in range(B):
+                cand = np.nonzero(before[b, lo:hi] == shape.mask_id)[0] + lo
+                lg = o.logits(hid[b, cand - pos_begin])
+                lg[:, shape.mask_id] = -np.inf
+                t, p = sto.top1_prob(lg)
+                assert gpos[b] in cand and gtok[b] != shape.mask_id
+                j = int(np.nonzero(cand == gpos[b])[0][0])
+                mx = lg[j].max()
+                p_gpu_tok = np.exp(lg[j, gtok[b]] - mx) * p[j]               # oracle probability of the GPU's token
+                assert p_gpu_tok >= p.max() * (1 - 5e-2), (steps, b, p_gpu_tok, p.max())
+                assert abs(gprob[b] - p_gpu_tok) <= 5e-2 * p_gpu_tok, (steps, b, gprob[b], p_gpu_tok)
+                agree += int(cand[int(np.argmax(p))] == gpos[b] and t[j] == gtok[b])
+                toks_np[b, gpos[b]] = gtok[b]                                  # teacher forcing: follow the GPU
+            np.testing.assert_array_equal(toks.cpu().numpy(), toks_np)
+            steps += 1
+    assert steps == shape.gen_len and not (toks_np == shape.mask_id).any()
+    # With random N(0, 0.02^2) weights the token distribution is nearly flat (top-1 probability ~ 2.4 / vocab), so many
+    # candidates tie within bf16 resolution; exact agreement of the arg-max is reported, not required.
+    print(f"mode {mode}: {agree} of {steps * B} choices are the oracle's own arg-max")
+    assert agree > 0
+    for l in range(shape.n_layers):
+        assert g.layer(l).status() == 0
+    g.close()
+
+
+def test_stack_argument_checks(dare):
+    import ctypes as C
+    shape = small_stack(L=2)
+    cfg_ok = dare.StackConfig(C.sizeof(dare.StackConfig), 2, 768, 1024, 1023, 32,
+                              dare.make_config(256, 2, 128, 2, 128, 5e5, 1e-5, dare.BF16))
+    assert dare.dare_stack_workspace_bytes(cfg_ok) > 0
+    for field, val in (("d_ff", 100), ("vocab", 1000), ("block", 64), ("mask_id", 5000)):
+        cfg = dare.StackConfig.from_buffer_copy(cfg_ok)
+        setattr(cfg, field, val)
+        assert dare.dare_stack_workspace_bytes(cfg) == 0, field
+    f32 = dare.StackConfig.from_buffer_copy(cfg_ok)
+    f32.layer.dtype = dare.F32
+    assert dare.dare_stack_workspace_bytes(f32) == 0
+    assert dare.dare_stack_reset(None) == dare.ERR_INVALID_ARG
+    assert dare.dare_stack_layer(None, 0) is None
