@@ -445,6 +445,56 @@ def run_micro(args):
     print(json.dumps(out))
 
 
+def run_stack(args):
+    """Config 4: the 32-layer LLaDA-8B-shaped stack with random bf16 weights, 256 prompt + 256 generated tokens in
+    32-token blocks, one denoising step per generated token, both reuse rules against the dense path.  One JSON line:
+    generated tokens per second (wall clock over the whole generation, host loop included)."""
+    import numpy as np
+    import torch
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare, workloads as wl
+    shape = wl.LLADA_STACK
+    lay = shape.layer
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(shape.seed)
+    d, f, V = lay.d_model, shape.d_ff, shape.vocab
+    draw = lambda *dims: (torch.randn(dims, generator=gen, device=dev) * 0.02).to(torch.bfloat16)
+    ones = torch.ones(d, device=dev)
+    w = {"emb": draw(V, d), "head": draw(V, d), "final_gain": ones, "layers": []}
+    for _ in range(shape.n_layers):
+        w["layers"].append({"w_q": draw(d, d), "w_k": draw(d, d), "w_v": draw(d, d), "w_o": draw(d, d), "rms_gain": ones,
+                            "gain2": ones, "w_gate": draw(f, d), "w_up": draw(f, d), "w_down": draw(d, f)})
+    B, P = 1, lay.prompt
+    stack = dare.Stack(shape, w, B, device=dev)
+    prompt = wl.random_prompt(shape, B)
+    taus = [TAU] * shape.n_layers
+    out = {"metric": "generated_tokens_per_s", "unit": "tokens/s", "data": "synthetic", "dtype": "bf16",
+           "config": {"workload": shape.name, "layers": shape.n_layers, "d_model": d, "d_ff": f, "vocab": V,
+                      "prompt": P, "generated": shape.gen_len, "block": lay.block, "batch": B, "threshold": TAU}}
+    for name in ("both", "dense"):
+        best = None
+        for rep in range(2):
+            toks = torch.from_numpy(np.concatenate([prompt, np.full((B, shape.gen_len), shape.mask_id, np.int32)], 1)).to(dev)
+            stack.reset()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            refreshed = 0
+            for step in range(shape.gen_len):
+                stack.decode_step(toks, P, step // lay.block, step == 0, MODES[name], taus)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        assert not bool((toks == shape.mask_id).any())
+        out[name] = {"tokens_per_s": round(shape.gen_len * B / best, 1), "ms_per_token": round(best / shape.gen_len * 1e3, 3)}
+    sel = [stack.layer(l).last_selection(B, lay.seq - P)["count"] for l in range(shape.n_layers)]
+    out["value"] = out["both"]["tokens_per_s"]
+    out["speedup_of_reuse_path"] = round(out["both"]["tokens_per_s"] / out["dense"]["tokens_per_s"], 3)
+    print(json.dumps(out))
+
+
 def run_sweep(args):
     """Crossover sweep on the long-context layer (batch 4, seq 4096 unless overridden): changed-token fraction
     0..100 % in 5 % steps, uniform and block-clustered patterns, modes kv / o / both against the dense path of the
@@ -539,10 +589,13 @@ def main():
     ap.add_argument("--d-model", type=int, default=0, help="exploration: other layer width (multiple of 128)")
     ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
     ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
+    ap.add_argument("--stack", action="store_true", help="full 32-layer stack generation (config 4) instead")
     ap.add_argument("--sweep", action="store_true", help="long-context crossover sweep (config 5) instead")
     ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
     args = ap.parse_args()
-    if args.sweep:
+    if args.stack:
+        run_stack(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.micro:
         run_micro(args)

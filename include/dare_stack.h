@@ -80,6 +80,11 @@ dare_status_t dare_stack_decode_step(dare_stack_t* stack, int32_t* tokens, int b
                                      const int32_t* forced_pos_host, const int32_t* forced_tok_host, int32_t* pos_out,
                                      int32_t* tok_out, float* prob_out, void* cuda_stream);
 
+/* Observation for tests: during every later pass, copy the input x and the output h = x + attention of layer
+ * `layer_index` into the DEVICE buffers x_out / h_out ([batch, seq_act, d_model] bf16 each; NULL = skip;
+ * layer_index < 0 switches the capture off). */
+dare_status_t dare_stack_set_capture(dare_stack_t* stack, int layer_index, void* x_out, void* h_out);
+
 /* Observation for tests: the final-normed hidden states [batch, seq_act, d_model] (bf16) of the last forward pass
  * or decoding step, copied to a HOST buffer of `bytes` bytes (synchronises the stream). */
 dare_status_t dare_stack_last_hidden(dare_stack_t* stack, void* dst_host, size_t bytes, void* cuda_stream);

@@ -206,6 +206,9 @@ struct dare_stack {
   const void* emb;
   const float* final_gain;
   StackBuffers buf;
+  int capture_layer;          // test hook: copy this layer's input and output of every pass (-1 = off)
+  void* capture_x;
+  void* capture_h;
 };
 
 namespace {
@@ -240,8 +243,12 @@ dare_status_t forward(dare_stack* S, const int* tokens, int batch, int seq_total
   const int m_tiles = batch * ((seq_act + 127) / 128);
   for (int l = 0; l < S->cfg.n_layers; ++l) {
     // h = x + DARE attention
+    if (l == S->capture_layer && S->capture_x)
+      cudaMemcpyAsync(S->capture_x, B.xa, (size_t)T_ * d * 2, cudaMemcpyDeviceToDevice, st);
     dare_status_t s = layer_enqueue(S->layers[l], B.xa, batch, seq_act, pos_begin, mode, taus[l], B.hb, st, true);
     if (s != DARE_OK) return s;
+    if (l == S->capture_layer && S->capture_h)
+      cudaMemcpyAsync(S->capture_h, B.hb, (size_t)T_ * d * 2, cudaMemcpyDeviceToDevice, st);
     // n = RMSNorm_2(h)
     launch_rmsnorm<bf16>(B.hb, S->blocks[l].gain2, B.n2, T_, d, lc.rms_eps, st);
     // act = silu(W_G n) * (W_U n)
@@ -299,6 +306,8 @@ dare_status_t dare_stack_create(const dare_stack_config_t* cfg, const dare_stack
   S->cfg.layer.kernel_path = DARE_PATH_TENSOR;
   S->emb = w->emb;
   S->final_gain = w->final_gain;
+  S->capture_layer = -1;
+  S->capture_x = S->capture_h = nullptr;
   const size_t lb = align_up(dare_layer_workspace_bytes(&S->cfg.layer));
   std::vector<void*> layer_ws;
   carve_stack(&S->cfg, (char*)workspace, &S->buf, &layer_ws, lb);
@@ -363,6 +372,16 @@ dare_status_t dare_stack_forward(dare_stack_t* S, const int32_t* tokens, int bat
   for (int l = 0; l < S->cfg.n_layers; ++l)
     if (isnan(taus_host[l])) return DARE_ERR_INVALID_ARG;
   return forward(S, tokens, batch, seq_total, seq_act, pos_begin, mode, taus_host, hidden_out, (cudaStream_t)cuda_stream);
+}
+
+dare_status_t dare_stack_set_capture(dare_stack_t* S, int layer_index, void* x_out, void* h_out) {
+  dare_status_t s = check_stack(S);
+  if (s != DARE_OK) return s;
+  if (layer_index >= (int)S->layers.size()) return DARE_ERR_SHAPE;
+  S->capture_layer = layer_index;
+  S->capture_x = x_out;
+  S->capture_h = h_out;
+  return DARE_OK;
 }
 
 dare_status_t dare_stack_last_hidden(dare_stack_t* S, void* dst_host, size_t bytes, void* cuda_stream) {

@@ -82,6 +82,7 @@ def _load():
         "dare_stack_destroy": (C.c_int, [vp]),
         "dare_stack_layer": (vp, [vp, i32]),
         "dare_stack_forward": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]),
+        "dare_stack_set_capture": (C.c_int, [vp, i32, vp, vp]),
         "dare_stack_last_hidden": (C.c_int, [vp, vp, sz, vp]),
         "dare_stack_decode_step": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
         "dare_layer_debug_timestamps": (C.c_int, [vp, i32, vp, vp]),
@@ -239,6 +240,10 @@ def dare_stack_forward(handle, tokens_ptr, batch, seq_total, seq_act, pos_begin,
                        stream=0) -> int:
     return _lib.dare_stack_forward(handle, tokens_ptr, batch, seq_total, seq_act, pos_begin, mode, taus_host_ptr,
                                    hidden_ptr, stream)
+
+
+def dare_stack_set_capture(handle, layer_index, x_ptr, h_ptr) -> int:
+    return _lib.dare_stack_set_capture(handle, layer_index, x_ptr, h_ptr)
 
 
 def dare_stack_last_hidden(handle, dst_host_ptr, nbytes, stream=0) -> int:
@@ -480,6 +485,12 @@ class Stack:
             raise DareError(st, "dare_stack_decode_step")
         torch.cuda.synchronize(self.device)       # the forced arrays are host memory read by an async copy
         return pos.cpu().numpy(), tok.cpu().numpy(), prob.cpu().numpy()
+
+    def set_capture(self, layer_index, x_buf=None, h_buf=None):
+        st = dare_stack_set_capture(self.handle, layer_index, x_buf.data_ptr() if x_buf is not None else None,
+                                    h_buf.data_ptr() if h_buf is not None else None)
+        if st != OK:
+            raise DareError(st, "dare_stack_set_capture")
 
     def last_hidden(self, batch, seq_act):
         """-> float32 numpy [batch, seq_act, d_model]: final-normed states of the last pass."""

@@ -118,3 +118,92 @@ def test_stack_argument_checks(dare):
     assert dare.dare_stack_workspace_bytes(f32) == 0
     assert dare.dare_stack_reset(None) == dare.ERR_INVALID_ARG
     assert dare.dare_stack_layer(None, 0) is None
+
+
+def _torch_stack_weights(shape, torch, seed=3):
+    """Full-size weights drawn on the GPU: N(0, 0.02^2) in bf16, gains 1."""
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    d, f, V = shape.layer.d_model, shape.d_ff, shape.vocab
+    draw = lambda *dims: (torch.randn(dims, generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+    ones = torch.ones(d, device="cuda")
+    w = {"emb": draw(V, d), "head": draw(V, d), "final_gain": ones, "layers": []}
+    for _ in range(shape.n_layers):
+        w["layers"].append({"w_q": draw(d, d), "w_k": draw(d, d), "w_v": draw(d, d), "w_o": draw(d, d), "rms_gain": ones,
+                            "gain2": ones, "w_gate": draw(f, d), "w_up": draw(f, d), "w_down": draw(d, f)})
+    return w
+
+
+def test_full_size_stack_teacher_forced_layer_checks(dare):
+    """Config 4 at full size: 32 layers, d 4096, SwiGLU 12288, vocab 126464, 256 prompt + 256 generation positions,
+    batch 1, both reuse rules.  The oracle cannot run the whole model, so it checks single layer steps: the state of a
+    layer (caches, stored query) and its input are taken from the GPU, one oracle layer step is run from that state,
+    and refresh set, caches and the layer's output are compared (tokens whose oracle score lies within the margin of
+    tau take the GPU's decision).  The step's token choice is checked against fp64 logits of the GPU's final states."""
+    import torch
+    from oracle import dare_oracle as orc
+    shape = wl.LLADA_STACK
+    lay = shape.layer
+    P, S, d, B = lay.prompt, lay.seq, lay.d_model, 1
+    w = _torch_stack_weights(shape, torch)
+    taus = [0.1] * shape.n_layers
+    g = dare.Stack(shape, w, B)
+    prompt = wl.random_prompt(shape, B)
+    toks = torch.from_numpy(np.concatenate([prompt, np.full((B, shape.gen_len), shape.mask_id, np.int32)], axis=1)).cuda()
+    checks = {1: (0,), 2: (13,), 5: (31,), 33: (7,)}   # step -> layer checked at that step (33: second block)
+    xbuf = torch.empty((B, S - P, d), dtype=torch.bfloat16, device="cuda")
+    hbuf = torch.empty_like(xbuf)
+    head64 = None
+    for step in range(34):
+        first = step == 0
+        blk = step // lay.block
+        layers_now = checks.get(step, ())
+        pre = {}
+        for l in layers_now[:1]:                         # one captured layer per step
+            lv = g.layer(l)
+            pre[l] = lv.read_caches(B, S)
+            g.set_capture(l, xbuf, hbuf)
+        before = toks.cpu().numpy().copy()
+        gpos, gtok, gprob = g.decode_step(toks, P, blk, first, 3, taus)
+        for l in layers_now[:1]:
+            g.set_capture(-1)
+            lv = g.layer(l)
+            lw = w["layers"][l]
+            o = orc.OracleLayer(d, lay.n_heads, lay.head_dim, B, S, lay.rope_theta, lay.rms_eps,
+                                *(lw[k].float().cpu().numpy() for k in ("w_q", "w_k", "w_v", "w_o")), np.ones(d))
+            o.has_prev, o.batch, o.kv_len = True, B, S
+            o.q_prev[:] = pre[l]["q_prev"]; o.k_cache[:] = pre[l]["k"]; o.v_cache[:] = pre[l]["v"]; o.o_cache[:] = pre[l]["o"]
+            sel = lv.last_selection(B, S - P)
+            gm = np.zeros(S - P, bool); gm[sel["idx"]] = True
+            x = xbuf.float().cpu().numpy()
+            y = o.step(x, 3, taus[l], pos_begin=P, adopt=(gm, MARGIN))
+            np.testing.assert_array_equal(sel["idx"], o.last_idx, err_msg=f"step {step} layer {l}")
+            assert 1 <= sel["count"] <= 8                # one new token per step: a handful of refreshed rows at most
+            parity.assert_close(f"h step {step} layer {l}", hbuf.float().cpu().numpy(), x + y, parity.TOL_BF16)
+            post = lv.read_caches(B, S)
+            parity.assert_close("k_cache", post["k"], o.k_cache, parity.TOL_BF16, max_factor=2.0)
+            parity.assert_close("v_cache", post["v"], o.v_cache, parity.TOL_BF16, max_factor=2.0)
+            parity.assert_close("o_cache", post["o"], o.o_cache, parity.TOL_BF16, max_factor=2.0)
+            # rows outside the refresh set: untouched, bit for bit (Eq. 3, Eq. 4)
+            keep = np.ones(S, bool); keep[P + sel["idx"]] = False
+            assert np.array_equal(post["k"][0, keep], pre[l]["k"][0, keep])
+            assert np.array_equal(post["o"][0, keep], pre[l]["o"][0, keep])
+        if step in (0, 2, 33):
+            # the choice under fp64 logits of the GPU's own final states
+            if head64 is None:
+                head64 = w["head"].float().cpu().numpy().astype(np.float64)
+            pos_begin = 0 if first else P
+            hid = g.last_hidden(B, S - pos_begin)
+            lo = P + blk * lay.block
+            cand = np.nonzero(before[0, lo:lo + lay.block] == shape.mask_id)[0] + lo
+            lg = hid[0, cand - pos_begin].astype(np.float64) @ head64.T
+            lg[:, shape.mask_id] = -np.inf
+            t, p = sto.top1_prob(lg)
+            j = int(np.nonzero(cand == gpos[0])[0][0])
+            p_tok = np.exp(lg[j, gtok[0]] - lg[j].max()) * p[j]
+            assert p_tok >= p.max() * (1 - 2e-2), (step, p_tok, p.max())
+            assert abs(gprob[0] - p_tok) <= 2e-2 * p_tok
+    assert not (toks[:, P:P + 32] == shape.mask_id).any() and (toks[:, P + 34:] == shape.mask_id).all()
+    for l in (0, 13, 31):
+        assert g.layer(l).status() == 0
+    g.close()
