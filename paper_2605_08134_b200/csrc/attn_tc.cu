@@ -7,11 +7,16 @@
 // One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 128:
 //   warp 0       TMA producer: K block and V block of the cache (two 64-column boxes each, 128-byte swizzle),
 //                double buffered
-//   warp 1       one thread issues S = Q K^T (M128 N128 K16 x 8) and O_blk = P V (M128 N128 K16 x 8, V as an MN-major
-//                operand) into tensor memory
-//   warps 2-9    softmax: thread <-> (query row, half): both halves read the row of S from tensor memory and agree on
-//                the running maximum; each exponentiates 64 of the 128 keys, writes them as bf16 into the swizzled
-//                P tile in shared memory, and rescales/accumulates its 64 of the 128 output columns in registers.
+//   warp 1       one thread issues S(i) = Q K(i)^T (M128 N128 K16 x 8) into tensor memory; S is double buffered there
+//                and S(i+1) is issued as soon as S(i-1) has been read, so the tensor pipe works on O_blk(i-1) and
+//                S(i+1) while the softmax warps are on S(i)
+//   warp 2       one thread issues O_blk(i) = P(i) V(i) (M128 N128 K16 x 8, V as an MN-major operand); a warp of its
+//                own because issuing eight MMAs next to busy softmax warps takes longer than executing them
+//   warps 3-10   softmax: thread <-> (query row, half): each reads its 64 of the row's 128 scores from tensor memory,
+//                the two halves agree on the running maximum through shared memory; each exponentiates its keys,
+//                writes them as bf16 into the swizzled P tile in shared memory, and rescales/accumulates its 64 of
+//                the 128 output columns in registers (the product of block i-1 is folded in after the exponentials
+//                of block i).
 // Key split: when a launch has few (tile, head) pairs - the row-sparse case with one row tile per sequence - the
 // gridDim.z CTAs of a cluster share a pair, CTA z taking key blocks z, z + gridDim.z, ...  Each CTA leaves its
 // un-normalised accumulator, running maximum and row sum in shared memory; CTA k owns 128/gridDim.z of the rows and
@@ -41,7 +46,8 @@ struct AttnSmem {
   static constexpr int V_OFF = K_OFF + 2 * K_BYTES;    // 2 buffers
   static constexpr int P_OFF = V_OFF + 2 * V_BYTES;
   static constexpr int L_OFF = P_OFF + P_BYTES;        // float[2][128] partial row sums
-  static constexpr int BAR_OFF = L_OFF + 2 * BQ * 4;
+  static constexpr int MX_OFF = L_OFF + 2 * BQ * 4;     // float[2][2][128] half-row maxima, by key-block parity
+  static constexpr int BAR_OFF = MX_OFF + 4 * BQ * 4;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;
   // after the key loop the operand buffers are idle; the merge of a key split reuses them:
   static constexpr int DUMP_OFF = 0;                   // this CTA's accumulator [128 rows][128 cols] fp32, 64 KB
@@ -49,9 +55,17 @@ struct AttnSmem {
   static constexpr int RECV_OFF = STAT_OFF + 2 * BQ * 4;    // up to 3 senders x (rows x 512 B + rows x 8 B)
 };
 
-constexpr int kThreads = 320;
+// 2^x for x <= 0 on the special-function unit; results below the normal range flush to zero (they are softmax
+// weights 2^-126 times smaller than the row's largest).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+constexpr int kThreads = 352;
 constexpr int kSoftmaxThreads = 256;
-constexpr uint32_t kTmemCols = 256;     // S: columns [0, 128), O_blk: columns [128, 256)
+constexpr uint32_t kTmemCols = 512;     // S of even / odd key blocks: columns [0, 128) / [128, 256); O_blk: [256, 384)
 
 }  // namespace
 
@@ -64,14 +78,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::BAR_OFF);
   uint64_t* k_full = bars;          // [2]
   uint64_t* v_full = bars + 2;      // [2]
-  uint64_t* kv_empty = bars + 4;    // [2]
-  uint64_t* s_full = bars + 6;
-  uint64_t* p_full = bars + 7;
-  uint64_t* o_full = bars + 8;
-  uint64_t* o_free = bars + 9;
-  uint64_t* recv_bar = bars + 10;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
+  uint64_t* k_empty = bars + 4;     // [2]
+  uint64_t* v_empty = bars + 6;     // [2]
+  uint64_t* s_full = bars + 8;      // [2]
+  uint64_t* s_free = bars + 10;     // [2]
+  uint64_t* p_full = bars + 12;
+  uint64_t* o_full = bars + 13;
+  uint64_t* recv_bar = bars + 14;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
   float* l_part = reinterpret_cast<float*>(smem + S::L_OFF);
+  float* mx_part = reinterpret_cast<float*>(smem + S::MX_OFF);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.x;
@@ -92,11 +108,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (p.batch_off[b] + tile * BQ >= p.batch_off[b + 1]) return;
   }
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
-    mbar_init(s_full, 1);
-    mbar_init(p_full, kSoftmaxThreads);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1); mbar_init(&s_free[i], kSoftmaxThreads / 32);
+    }
+    mbar_init(p_full, kSoftmaxThreads / 32);
     mbar_init(o_full, 1);
-    mbar_init(o_free, kSoftmaxThreads);
     mbar_init(recv_bar, 1);
     fence_mbar_init();
     if (ksplit > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)((ksplit - 1) * rows_own * (HD * 4 + 8)));
@@ -144,7 +161,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + BKV;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * BKV;
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   if (active) {
@@ -152,13 +169,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (lane == 0) {
       for (int i = 0; i < n_blocks; ++i) {
         const int buf = i & 1;
-        mbar_wait(&kv_empty[buf], ((i >> 1) & 1) ^ 1, p.status);
         uint8_t* kd = smem + S::K_OFF + buf * S::K_BYTES;
         uint8_t* vd = smem + S::V_OFF + buf * S::V_BYTES;
         const int row = kv_row0 + (z + i * ksplit) * BKV;
+        mbar_wait(&k_empty[buf], ((i >> 1) & 1) ^ 1, p.status);     // S(i-2) = Q K(i-2)^T has been computed
         mbar_arrive_expect_tx(&k_full[buf], S::K_BYTES);
         tma_load_2d(kd, &tm_k, h * HD, row, &k_full[buf]);
         tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[buf]);
+        mbar_wait(&v_empty[buf], ((i >> 1) & 1) ^ 1, p.status);     // O_blk(i-2) = P(i-2) V(i-2) has been computed
         mbar_arrive_expect_tx(&v_full[buf], S::V_BYTES);
         tma_load_2d(vd, &tm_v, h * HD, row, &v_full[buf]);
         tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[buf]);
@@ -166,122 +184,143 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
     __syncwarp();
   } else if (warp == 1) {
+    // ---- S(i) = Q K(i)^T, issued as soon as the softmax warps have read S(i-2) out of its buffer: while they work
+    // on S(i) the tensor pipe computes O_blk(i-1) and S(i+1)
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
-      constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
-      const uint32_t q_addr = smem_u32(smem + S::Q_OFF);
-      const uint32_t p_addr = smem_u32(smem + S::P_OFF);
-      auto issue_qk = [&](int i) {
-        const int buf = i & 1;
-        mbar_wait(&k_full[buf], (i >> 1) & 1, p.status);
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(smem + S::K_OFF + buf * S::K_BYTES);
-#pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint64_t a = smem_desc_k_sw128(q_addr + (kk >> 2) * (BQ * 128) + (kk & 3) * 32);
-          const uint64_t bd = smem_desc_k_sw128(k_addr + (kk >> 2) * (BKV * 128) + (kk & 3) * 32);
-          umma_ss(tmem_s, a, bd, idesc_qk, kk != 0 ? 1u : 0u);
-        }
-        umma_commit(s_full);
-      };
-      if (n_blocks > 0) issue_qk(0);
+      const uint64_t q_desc = smem_desc_k_sw128(smem_u32(smem + S::Q_OFF));
       for (int i = 0; i < n_blocks; ++i) {
         const int buf = i & 1;
-        mbar_wait(p_full, i & 1, p.status);                 // P(i) is in shared memory, S(i) has been read
-        mbar_wait(&v_full[buf], (i >> 1) & 1, p.status);
-        if (i > 0) mbar_wait(o_free, (i - 1) & 1, p.status);  // O_blk(i-1) has been read out of tensor memory
+        if (i >= 2) mbar_wait(&s_free[buf], ((i >> 1) - 1) & 1, p.status);
+        mbar_wait(&k_full[buf], (i >> 1) & 1, p.status);
         tc_fence_after();
-        const uint32_t v_addr = smem_u32(smem + S::V_OFF + buf * S::V_BYTES);
+        const uint64_t k_desc = smem_desc_k_sw128(smem_u32(smem + S::K_OFF + buf * S::K_BYTES));
 #pragma unroll
-        for (int ks = 0; ks < BKV / 16; ++ks) {
-          const uint64_t a = smem_desc_k_sw128(p_addr + (ks >> 2) * (BQ * 128) + (ks & 3) * 32);
-          const uint64_t bd = smem_desc_mn_sw128(v_addr + ks * (16 * 128), BKV * 128);
-          umma_ss(tmem_o, a, bd, idesc_pv, ks != 0 ? 1u : 0u);
-        }
+        for (int kk = 0; kk < HD / 16; ++kk)
+          umma_ss(tmem_s + buf * BKV, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
+                  k_desc + (((kk >> 2) * (BKV * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk != 0 ? 1u : 0u);
+        umma_commit(&s_full[buf]);
+        umma_commit(&k_empty[buf]);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ---- O_blk(i) = P(i) V(i), from its own warp so that its issue does not queue behind the score products'
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
+      const uint64_t p_desc = smem_desc_k_sw128(smem_u32(smem + S::P_OFF));
+      for (int i = 0; i < n_blocks; ++i) {
+        const int buf = i & 1;
+        // P(i) is in shared memory and O_blk(i-1) has been read out of tensor memory
+        mbar_wait(p_full, i & 1, p.status);
+        mbar_wait(&v_full[buf], (i >> 1) & 1, p.status);
+        tc_fence_after();
+        const uint64_t v_desc = smem_desc_mn_sw128(smem_u32(smem + S::V_OFF + buf * S::V_BYTES), BKV * 128);
+#pragma unroll
+        for (int ks = 0; ks < BKV / 16; ++ks)
+          umma_ss(tmem_o, p_desc + (((ks >> 2) * (BQ * 128) + (ks & 3) * 32) >> 4), v_desc + ((ks * (16 * 128)) >> 4),
+                  idesc_pv, ks != 0 ? 1u : 0u);
         umma_commit(o_full);
-        umma_commit(&kv_empty[buf]);
-        if (i + 1 < n_blocks) issue_qk(i + 1);
+        umma_commit(&v_empty[buf]);
       }
     }
     __syncwarp();
   } else {
     // ---- softmax and output accumulation
-    const int sw = warp - 2;                    // 0..7
+    const int sw = warp - 3;                    // 0..7
     const int half = sw >> 2;                   // which 32 keys of a block / which 64 output columns
     const int quarter = warp & 3;               // TMEM lane quarter of this warp
     const int r = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)HD) * 1.4426950408889634f;   // softmax scale folded into the exp2 argument
-    float m = -INFINITY, l = 0.f;
+    float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
     float acc[64];
 #pragma unroll
     for (int i = 0; i < 64; ++i) acc[i] = 0.f;
     uint8_t* ps = smem + S::P_OFF;
 
     for (int i = 0; i < n_blocks; ++i) {
-      mbar_wait(s_full, i & 1, p.status);
+      const uint32_t tmem_si = tmem_s + (i & 1) * BKV;
+      mbar_wait(&s_full[i & 1], (i >> 1) & 1, p.status);
       tc_fence_after();
-      if (dbg && i == 0 && threadIdx.x == 64) p.debug[2] = globaltimer_ns();
+      if (dbg && i == 0 && threadIdx.x == 96) p.debug[2] = globaltimer_ns();
       const int key0 = (z + i * ksplit) * BKV;
       const bool ragged = key0 + BKV > g.kv_len;      // last block: keys past kv_len do not exist
-      float mx = m;
-      // the other half's 64 scores only matter for the row maximum
-#pragma unroll
-      for (int cgrp = 0; cgrp < 2; ++cgrp) {
-        float so[32];
-        tmem_ld_32x32(tmem_s + lane_addr + (half ^ 1) * 64 + cgrp * 32, so);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float v = (ragged && key0 + (half ^ 1) * 64 + cgrp * 32 + j >= g.kv_len) ? -INFINITY : so[j];
-          mx = fmaxf(mx, v);
-        }
-      }
       float s_mine[64];
       {
         float t0_[32], t1_[32];
-        tmem_ld_32x32(tmem_s + lane_addr + half * 64, t0_);
-        tmem_ld_32x32(tmem_s + lane_addr + half * 64 + 32, t1_);
+        tmem_ld_32x32(tmem_si + lane_addr + half * 64, t0_);
+        tmem_ld_32x32(tmem_si + lane_addr + half * 64 + 32, t1_);
 #pragma unroll
         for (int j = 0; j < 32; ++j) { s_mine[j] = t0_[j]; s_mine[32 + j] = t1_[j]; }
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_free[i & 1]);            // this warp's part of S(i) is in registers
       if (ragged) {
 #pragma unroll
         for (int j = 0; j < 64; ++j)
           if (key0 + half * 64 + j >= g.kv_len) s_mine[j] = -INFINITY;
       }
+      // row maximum: four independent chains over this half, then the other half's through shared memory (the two
+      // threads of a row sit in the two warps of one tensor-memory lane quarter and meet on that quarter's barrier)
+      float mx4[4] = {s_mine[0], s_mine[1], s_mine[2], s_mine[3]};
 #pragma unroll
-      for (int j = 0; j < 64; ++j) mx = fmaxf(mx, s_mine[j]);
-      const float alpha = exp2f((m - mx) * c);
+      for (int j = 4; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s_mine[j]);
+      const float mx_half = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      float* mxp = mx_part + (i & 1) * 2 * BQ;
+      mxp[half * BQ + r] = mx_half;
+      asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
+      const float mx = fmaxf(m, fmaxf(mx_half, mxp[(half ^ 1) * BQ + r]));
+      const float alpha = fast_exp2((m - mx) * c);
       m = mx;
       const float mc = mx * c;
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < 64; ++j) {
-        s_mine[j] = exp2f(fmaf(s_mine[j], c, -mc));
-        sum += s_mine[j];
+        s_mine[j] = fast_exp2(fmaf(s_mine[j], c, -mc));
+        sum4[j & 3] += s_mine[j];
       }
+      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l = l * alpha + sum;
+      uint4 pk[8];
+#pragma unroll
+      for (int v = 0; v < 8; ++v) pk[v] = pack8_bf16(s_mine + 8 * v);
+      // The previous block's product has had the whole softmax above to finish: fold it into the accumulator (its
+      // completion also frees the P tile).
+      if (i > 0) {
+        mbar_wait(o_full, (i - 1) & 1, p.status);
+        tc_fence_after();
+#pragma unroll
+        for (int cgrp = 0; cgrp < 2; ++cgrp) {
+          float o[32];
+          tmem_ld_32x32(tmem_o + lane_addr + half * 64 + cgrp * 32, o);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha_prev, o[j]);
+        }
+      }
+      alpha_prev = alpha;
       // P row segment: this half's 64 keys are one 128-byte row of 64-key chunk `half`, 8 swizzled 16-byte units
 #pragma unroll
       for (int v = 0; v < 8; ++v)
-        *reinterpret_cast<uint4*>(ps + half * (BQ * 128) + r * 128 + ((v ^ (r & 7)) << 4)) = pack8_bf16(s_mine + 8 * v);
+        *reinterpret_cast<uint4*>(ps + half * (BQ * 128) + r * 128 + ((v ^ (r & 7)) << 4)) = pk[v];
       fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(p_full);
-
-      mbar_wait(o_full, i & 1, p.status);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full);
+    }
+    if (n_blocks > 0) {
+      mbar_wait(o_full, (n_blocks - 1) & 1, p.status);
       tc_fence_after();
 #pragma unroll
       for (int cgrp = 0; cgrp < 2; ++cgrp) {
         float o[32];
         tmem_ld_32x32(tmem_o + lane_addr + half * 64 + cgrp * 32, o);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha, o[j]);
+        for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha_prev, o[j]);
       }
-      tc_fence_before();
-      mbar_arrive(o_free);
     }
-    if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
+    if (dbg && threadIdx.x == 96) p.debug[3] = globaltimer_ns();
     // ---- combine the two halves' row sums
     l_part[half * BQ + r] = l;
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
@@ -321,7 +360,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     tc_fence_before();
     cluster_sync_all();                                  // every CTA of the cluster is past its key loop
     tc_fence_after();
-    if (warp == 2 && lane < ksplit && lane != z) {
+    if (warp == 3 && lane < ksplit && lane != z) {
       // hand the rows owned by CTA `lane` to it: the rows, their maxima, their sums
       const int k = lane;
       const int slot = z < k ? z : z - 1;
