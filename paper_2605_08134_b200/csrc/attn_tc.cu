@@ -4,19 +4,23 @@
 // The result rows are written straight into the attention-output cache at their cache rows; rows that are not
 // computed keep their cached value (Alg. 2 lines 9-10).
 //
-// One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 128:
-//   warp 0       TMA producer: K block and V block of the cache (two 64-column boxes each, 128-byte swizzle),
-//                double buffered
-//   warp 1       one thread issues S(i) = Q K(i)^T (M128 N128 K16 x 8) into tensor memory; S is double buffered there
-//                and S(i+1) is issued as soon as S(i-1) has been read, so the tensor pipe works on O_blk(i-1) and
-//                S(i+1) while the softmax warps are on S(i)
-//   warp 2       one thread issues O_blk(i) = P(i) V(i) (M128 N128 K16 x 8, V as an MN-major operand); a warp of its
-//                own because issuing eight MMAs next to busy softmax warps takes longer than executing them
-//   warps 3-10   softmax: thread <-> (query row, half): each reads its 64 of the row's 128 scores from tensor memory,
-//                the two halves agree on the running maximum through shared memory; each exponentiates its keys,
-//                writes them as bf16 into the swizzled P tile in shared memory, and rescales/accumulates its 64 of
-//                the 128 output columns in registers (the product of block i-1 is folded in after the exponentials
-//                of block i).
+// One CTA = one head x one tile of up to 128 query rows of one sequence, walking the keys in blocks of 128.  The key
+// blocks alternate between two independent streams (even blocks: stream 0, odd blocks: stream 1); each stream has
+// its own running maximum, row sum and accumulator, and the two are merged at the end like the partials of a key
+// split.  While one stream's softmax warps are busy on the special-function unit the other stream's are moving
+// data, so both the tensor pipe and the exponentials stay busy.  Per stream:
+//   warp s       TMA producer: K block and V block of the cache (two 64-column boxes each, 128-byte swizzle)
+//   warp 2+s     one lane issues S = Q K^T (M128 N128 K16 x 8, both operands in shared memory) and O += P V
+//                (M128 N128 K16 x 8, P read from tensor memory, V from shared memory as an MN-major operand)
+//   warps 4+4s.. four softmax warps, thread <-> query row: reads its row of S from tensor memory, exponentiates, and
+//                writes P as bf16 over the first 64 columns of S (two keys per 32-bit column, the layout of a
+//                tensor-memory A operand), so P never passes through shared memory.  O accumulates in tensor
+//                memory; it is rescaled in place only when the running maximum has grown by more than 2^8 (the
+//                exponentials are taken against the older maximum until then, which changes nothing in exact
+//                arithmetic: numerator and row sum share the factor).
+// A single-CTA MMA with both operands in shared memory reads 8 KB per 64 cycles there, all the bandwidth shared
+// memory has; the TMA writes of K and V and any P traffic come on top.  Shared-memory traffic, not the tensor pipe,
+// bounds this kernel, which is why P stays in tensor memory.
 // Key split: when a launch has few (tile, head) pairs - the row-sparse case with one row tile per sequence - the
 // gridDim.z CTAs of a cluster share a pair, CTA z taking key blocks z, z + gridDim.z, ...  Each CTA leaves its
 // un-normalised accumulator, running maximum and row sum in shared memory; CTA k owns 128/gridDim.z of the rows and
@@ -40,20 +44,21 @@ struct AttnSmem {
   static constexpr int Q_BYTES = BQ * HD * 2;          // two 64-column chunks of [128 x 128 B]
   static constexpr int K_BYTES = BKV * HD * 2;         // two chunks of [64 x 128 B]
   static constexpr int V_BYTES = BKV * HD * 2;
-  static constexpr int P_BYTES = BQ * BKV * 2;         // two 64-key chunks of [128 x 128 B]
   static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = Q_OFF + Q_BYTES;        // 2 buffers
-  static constexpr int V_OFF = K_OFF + 2 * K_BYTES;    // 2 buffers
-  static constexpr int P_OFF = V_OFF + 2 * V_BYTES;
-  static constexpr int L_OFF = P_OFF + P_BYTES;        // float[2][128] partial row sums
-  static constexpr int MX_OFF = L_OFF + 2 * BQ * 4;     // float[2][2][128] half-row maxima, by key-block parity
-  static constexpr int BAR_OFF = MX_OFF + 4 * BQ * 4;
+  static constexpr int K_OFF = Q_OFF + Q_BYTES;        // one buffer per stream
+  static constexpr int V_OFF = K_OFF + 2 * K_BYTES;    // two buffers per stream: V(j) is wanted last in a block and
+                                                       // its buffer is released last, so one buffer leaves no slack
+  static constexpr int BAR_OFF = V_OFF + 4 * V_BYTES;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;
+  // merge of the two streams: a stream's running maxima [128] and row sums [128] go to its first V buffer, idle
+  // after its last product
   // after the key loop the operand buffers are idle; the merge of a key split reuses them:
   static constexpr int DUMP_OFF = 0;                   // this CTA's accumulator [128 rows][128 cols] fp32, 64 KB
   static constexpr int STAT_OFF = DUMP_OFF + BQ * HD * 4;   // running maximum [128], row sum [128]
   static constexpr int RECV_OFF = STAT_OFF + 2 * BQ * 4;    // up to 3 senders x (rows x 512 B + rows x 8 B)
 };
+static_assert(AttnSmem::TOTAL <= 232448, "shared memory");
+// (the key-split buffers may overlap the streams' statistics: they are filled after the statistics were read)
 
 // 2^x for x <= 0 on the special-function unit; results below the normal range flush to zero (they are softmax
 // weights 2^-126 times smaller than the row's largest).
@@ -63,9 +68,11 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 256;
-constexpr uint32_t kTmemCols = 512;     // S of even / odd key blocks: columns [0, 128) / [128, 256); O_blk: [256, 384)
+// S of stream 0 / 1: columns [0, 128) / [128, 256), P over the first 64 of them; O: [256, 384) / [384, 512)
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleStep = 8.f;     // log2 of the growth of the running maximum that triggers a rescale of O
 
 }  // namespace
 
@@ -76,30 +83,48 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::BAR_OFF);
+  // one of each per stream
   uint64_t* k_full = bars;          // [2]
-  uint64_t* v_full = bars + 2;      // [2]
-  uint64_t* k_empty = bars + 4;     // [2]
-  uint64_t* v_empty = bars + 6;     // [2]
-  uint64_t* s_full = bars + 8;      // [2]
-  uint64_t* s_free = bars + 10;     // [2]
-  uint64_t* p_full = bars + 12;
-  uint64_t* o_full = bars + 13;
-  uint64_t* recv_bar = bars + 14;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
-  float* l_part = reinterpret_cast<float*>(smem + S::L_OFF);
-  float* mx_part = reinterpret_cast<float*>(smem + S::MX_OFF);
+  uint64_t* k_empty = bars + 2;     // [2]
+  uint64_t* s_full = bars + 4;      // [2]
+  uint64_t* p_full = bars + 6;      // [2]
+  uint64_t* o_full = bars + 8;      // [2]
+  uint64_t* v_full = bars + 10;     // [2 streams][2 buffers]
+  uint64_t* v_empty = bars + 14;    // [2 streams][2 buffers]
+  uint64_t* recv_bar = bars + 18;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.x;
+  // the warp index through a shuffle, so that the compiler knows it (and every role decision and shared-memory
+  // descriptor derived from it) to be uniform over the warp
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int ksplit = gridDim.z;                      // = cluster size along z
   const int z = ksplit > 1 ? (int)cluster_ctarank() : 0;
   const int rows_own = BQ / ksplit;                   // rows of the tile this CTA writes out
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
   const StepGeom& g = p.g;
-  // blockIdx.y = tile * batch + b: the first row tile of every sequence comes first in launch order, so that in the
-  // row-sparse case the CTAs that have work are scheduled before the (many) tiles past the refresh set
-  const int tile = blockIdx.y / g.batch, b = blockIdx.y - tile * g.batch;
+  // CTA -> (head, sequence, row tile), in launch order:
+  //   row-sparse: heads fastest, then sequences, then row tiles: the first row tile of every sequence comes first,
+  //               so that the CTAs that have work are scheduled before the (many) tiles past the refresh set
+  //   dense     : row tiles fastest, then heads, then sequences: the CTAs resident at any time share the K and V of
+  //               a few (sequence, head) pairs, which then stay in the L2 instead of being streamed from HBM by
+  //               every row tile again
+  int h, b, tile;
+  {
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+    if (p.idx != nullptr) {
+      h = lin % g.n_heads;
+      const int rest = lin / g.n_heads;
+      tile = rest / g.batch;
+      b = rest - tile * g.batch;
+    } else {
+      const int tps = (g.seq_act + BQ - 1) / BQ;
+      tile = lin % tps;
+      const int rest = lin / tps;
+      h = rest % g.n_heads;
+      b = rest / g.n_heads;
+    }
+  }
 
   // Row tiles past the first one of a sequence are usually empty in the row-sparse case: they look at the refresh
   // set before spending anything on set-up.
@@ -109,18 +134,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_empty[i], 1);
-      mbar_init(&s_full[i], 1); mbar_init(&s_free[i], kSoftmaxThreads / 32);
+      mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[2 * i], 1); mbar_init(&v_full[2 * i + 1], 1);
+      mbar_init(&v_empty[2 * i], 1); mbar_init(&v_empty[2 * i + 1], 1);
+      mbar_init(&s_full[i], 1); mbar_init(&o_full[i], 1);
+      mbar_init(&p_full[i], kSoftmaxThreads / 64);     // one arrival per softmax warp of the stream
     }
-    mbar_init(p_full, kSoftmaxThreads / 32);
-    mbar_init(o_full, 1);
     mbar_init(recv_bar, 1);
     fence_mbar_init();
     if (ksplit > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)((ksplit - 1) * rows_own * (HD * 4 + 8)));
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
-  if (warp == 1) {
+  if (warp == 2) {
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
@@ -142,18 +168,45 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int n_blocks_all = (g.kv_len + BKV - 1) / BKV;
   const int n_blocks = n_blocks_all > z ? (n_blocks_all - z + ksplit - 1) / ksplit : 0;   // blocks z, z + ksplit, ...
   const int kv_row0 = b * g.max_seq;
+  // The first K and V block of each stream start now, by the thread that initialised the barriers, so that they are
+  // in flight while the Q tile is gathered.
+  if (threadIdx.x == 0 && active) {
+    for (int s2 = 0; s2 < 2 && s2 < n_blocks; ++s2) {
+      const int row = kv_row0 + (z + s2 * ksplit) * BKV;
+      uint8_t* kd = smem + S::K_OFF + s2 * S::K_BYTES;
+      uint8_t* vd = smem + S::V_OFF + 2 * s2 * S::V_BYTES;
+      mbar_arrive_expect_tx(&k_full[s2], S::K_BYTES);
+      tma_load_2d(kd, &tm_k, h * HD, row, &k_full[s2]);
+      tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[s2]);
+      mbar_arrive_expect_tx(&v_full[2 * s2], S::V_BYTES);
+      tma_load_2d(vd, &tm_v, h * HD, row, &v_full[2 * s2]);
+      tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[2 * s2]);
+    }
+  }
   // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
-  {
+  if (active) {
     uint8_t* qs = smem + S::Q_OFF;
-    for (int u = threadIdx.x; active && u < BQ * 16; u += kThreads) {
-      const int r = u >> 4, unit = u & 15;           // 16 units of 8 bf16 per row
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < rows_valid) {
-        const int t = p.idx ? p.idx[row0 + r] : row0 + r;
-        v = *reinterpret_cast<const uint4*>(p.q + (size_t)t * g.d + h * HD + unit * 8);
-      }
+    constexpr int QU = (BQ * 16 + kThreads - 1) / kThreads;   // 16-byte units per thread
+    int tok[QU];
+    uint4 qv[QU];
+    // all index loads first, then all row loads, then the stores: one memory round trip each instead of one per unit
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int u = threadIdx.x + k * kThreads, r = u >> 4;    // 16 units of 8 bf16 per row
+      tok[k] = -1;
+      if (u < BQ * 16 && r < rows_valid) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
+    }
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int unit = (threadIdx.x + k * kThreads) & 15;
+      qv[k] = make_uint4(0u, 0u, 0u, 0u);
+      if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
+    }
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int u = threadIdx.x + k * kThreads, r = u >> 4, unit = u & 15;
       const int chunk = unit >> 3, uc = unit & 7;
-      *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + r * 128 + ((uc ^ (r & 7)) << 4)) = v;
+      if (u < BQ * 16) *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + r * 128 + ((uc ^ (r & 7)) << 4)) = qv[k];
     }
     fence_proxy_async_smem();
   }
@@ -161,194 +214,213 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * BKV;
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   if (active) {
-  if (warp == 0) {
-    if (lane == 0) {
-      for (int i = 0; i < n_blocks; ++i) {
-        const int buf = i & 1;
-        uint8_t* kd = smem + S::K_OFF + buf * S::K_BYTES;
-        uint8_t* vd = smem + S::V_OFF + buf * S::V_BYTES;
-        const int row = kv_row0 + (z + i * ksplit) * BKV;
-        mbar_wait(&k_empty[buf], ((i >> 1) & 1) ^ 1, p.status);     // S(i-2) = Q K(i-2)^T has been computed
-        mbar_arrive_expect_tx(&k_full[buf], S::K_BYTES);
-        tma_load_2d(kd, &tm_k, h * HD, row, &k_full[buf]);
-        tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[buf]);
-        mbar_wait(&v_empty[buf], ((i >> 1) & 1) ^ 1, p.status);     // O_blk(i-2) = P(i-2) V(i-2) has been computed
-        mbar_arrive_expect_tx(&v_full[buf], S::V_BYTES);
-        tma_load_2d(vd, &tm_v, h * HD, row, &v_full[buf]);
-        tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[buf]);
+  // stream of this warp (producers 0/1, issuers 2/3, softmax warps 4-7 / 8-11) and its share of the key blocks:
+  // local blocks st, st + 2, ... of this CTA's blocks, local block i being key block z + i * ksplit
+  const int st = warp < 4 ? (warp & 1) : ((warp - 4) >> 2);
+  const int n_st = (n_blocks - st + 1) / 2;
+  const int n_other = n_blocks - n_st;
+  const uint32_t tmem_s = tmem_base + st * BKV, tmem_o = tmem_base + 2 * BKV + st * HD;
+  // The producer and issuer warps run their loops converged (every lane polls the barriers); one elected lane
+  // issues the copies and the MMAs.  Their operands are then warp-uniform values, which is what those instructions take.
+  if (warp < 2) {
+    uint8_t* kd = smem + S::K_OFF + st * S::K_BYTES;
+    for (int j = 1; j < n_st; ++j) {                        // block 0 of the stream was started before the Q gather
+      const int vb = 2 * st + (j & 1);
+      uint8_t* vd = smem + S::V_OFF + vb * S::V_BYTES;
+      const int row = kv_row0 + (z + (2 * j + st) * ksplit) * BKV;
+      mbar_wait(&k_empty[st], (j & 1) ^ 1, p.status);       // S(j-1) = Q K(j-1)^T has been computed
+      if (elect_one()) {
+        mbar_arrive_expect_tx(&k_full[st], S::K_BYTES);
+        tma_load_2d(kd, &tm_k, h * HD, row, &k_full[st]);
+        tma_load_2d(kd + S::K_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[st]);
       }
+      __syncwarp();
+      mbar_wait(&v_empty[vb], ((j >> 1) & 1) ^ 1, p.status);       // O += P(j-2) V(j-2) has been computed
+      if (elect_one()) {
+        mbar_arrive_expect_tx(&v_full[vb], S::V_BYTES);
+        tma_load_2d(vd, &tm_v, h * HD, row, &v_full[vb]);
+        tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[vb]);
+      }
+      __syncwarp();
     }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ---- S(i) = Q K(i)^T, issued as soon as the softmax warps have read S(i-2) out of its buffer: while they work
-    // on S(i) the tensor pipe computes O_blk(i-1) and S(i+1)
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
-      const uint64_t q_desc = smem_desc_k_sw128(smem_u32(smem + S::Q_OFF));
-      for (int i = 0; i < n_blocks; ++i) {
-        const int buf = i & 1;
-        if (i >= 2) mbar_wait(&s_free[buf], ((i >> 1) - 1) & 1, p.status);
-        mbar_wait(&k_full[buf], (i >> 1) & 1, p.status);
-        tc_fence_after();
-        const uint64_t k_desc = smem_desc_k_sw128(smem_u32(smem + S::K_OFF + buf * S::K_BYTES));
+  } else if (warp < 4) {
+    constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
+    constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
+    const uint64_t q_desc = smem_desc_k_sw128(smem_u32(smem + S::Q_OFF));
+    const uint64_t k_desc = smem_desc_k_sw128(smem_u32(smem + S::K_OFF + st * S::K_BYTES));
+    const uint64_t v_desc0 = smem_desc_mn_sw128(smem_u32(smem + S::V_OFF + 2 * st * S::V_BYTES), BKV * 128);
+    auto issue_qk = [&](int j) {
+      mbar_wait(&k_full[st], j & 1, p.status);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
-          umma_ss(tmem_s + buf * BKV, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
+          umma_ss(tmem_s, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
                   k_desc + (((kk >> 2) * (BKV * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk != 0 ? 1u : 0u);
-        umma_commit(&s_full[buf]);
-        umma_commit(&k_empty[buf]);
+        umma_commit(&s_full[st]);
+        umma_commit(&k_empty[st]);
       }
-    }
-    __syncwarp();
-  } else if (warp == 2) {
-    // ---- O_blk(i) = P(i) V(i), from its own warp so that its issue does not queue behind the score products'
-    if (lane == 0) {
-      constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
-      const uint64_t p_desc = smem_desc_k_sw128(smem_u32(smem + S::P_OFF));
-      for (int i = 0; i < n_blocks; ++i) {
-        const int buf = i & 1;
-        // P(i) is in shared memory and O_blk(i-1) has been read out of tensor memory
-        mbar_wait(p_full, i & 1, p.status);
-        mbar_wait(&v_full[buf], (i >> 1) & 1, p.status);
-        tc_fence_after();
-        const uint64_t v_desc = smem_desc_mn_sw128(smem_u32(smem + S::V_OFF + buf * S::V_BYTES), BKV * 128);
+      __syncwarp();
+    };
+    if (n_st > 0) issue_qk(0);
+    for (int j = 0; j < n_st; ++j) {
+      mbar_wait(&p_full[st], j & 1, p.status);      // P(j) has replaced S(j) in tensor memory
+      const int vb = 2 * st + (j & 1);
+      mbar_wait(&v_full[vb], (j >> 1) & 1, p.status);
+      tc_fence_after();
+      if (elect_one()) {
+        const uint64_t v_desc = v_desc0 + (uint64_t)((j & 1) * (S::V_BYTES >> 4));
 #pragma unroll
-        for (int ks = 0; ks < BKV / 16; ++ks)
-          umma_ss(tmem_o, p_desc + (((ks >> 2) * (BQ * 128) + (ks & 3) * 32) >> 4), v_desc + ((ks * (16 * 128)) >> 4),
-                  idesc_pv, ks != 0 ? 1u : 0u);
-        umma_commit(o_full);
-        umma_commit(&v_empty[buf]);
+        for (int ks = 0; ks < BKV / 16; ++ks)       // 16 keys of P = 8 columns
+          umma_ts(tmem_o, tmem_s + ks * 8, v_desc + ((ks * (16 * 128)) >> 4), idesc_pv, (j | ks) != 0 ? 1u : 0u);
+        umma_commit(&o_full[st]);
+        umma_commit(&v_empty[vb]);
       }
+      __syncwarp();
+      // the tensor pipe runs MMAs in issue order: the next scores overwrite P(j) only after the product above read it
+      if (j + 1 < n_st) issue_qk(j + 1);
     }
-    __syncwarp();
   } else {
-    // ---- softmax and output accumulation
-    const int sw = warp - 3;                    // 0..7
-    const int half = sw >> 2;                   // which 32 keys of a block / which 64 output columns
+    // ---- softmax of this stream's blocks: thread <-> query row
     const int quarter = warp & 3;               // TMEM lane quarter of this warp
     const int r = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)HD) * 1.4426950408889634f;   // softmax scale folded into the exp2 argument
-    float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
-    float acc[64];
-#pragma unroll
-    for (int i = 0; i < 64; ++i) acc[i] = 0.f;
-    uint8_t* ps = smem + S::P_OFF;
+    float m = -INFINITY, l = 0.f;               // maximum the exponentials are taken against; row sum against it
 
-    for (int i = 0; i < n_blocks; ++i) {
-      const uint32_t tmem_si = tmem_s + (i & 1) * BKV;
-      mbar_wait(&s_full[i & 1], (i >> 1) & 1, p.status);
+    for (int j = 0; j < n_st; ++j) {
+      mbar_wait(&s_full[st], j & 1, p.status);
       tc_fence_after();
-      if (dbg && i == 0 && threadIdx.x == 96) p.debug[2] = globaltimer_ns();
-      const int key0 = (z + i * ksplit) * BKV;
-      const bool ragged = key0 + BKV > g.kv_len;      // last block: keys past kv_len do not exist
-      float s_mine[64];
-      {
-        float t0_[32], t1_[32];
-        tmem_ld_32x32(tmem_si + lane_addr + half * 64, t0_);
-        tmem_ld_32x32(tmem_si + lane_addr + half * 64 + 32, t1_);
+      if (dbg && j == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
+      const int key0 = (z + (2 * j + st) * ksplit) * BKV;
+      const int n_keys = min(BKV, g.kv_len - key0);   // the last block may be ragged: keys past kv_len do not exist
+      // the row of S: four loads in flight together
+      float v[128];
+      tmem_ld_32x32_nowait(tmem_s + lane_addr, v);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 32, v + 32);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 64, v + 64);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 96, v + 96);
+      tmem_ld_wait();
+      if (n_keys < BKV) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) { s_mine[j] = t0_[j]; s_mine[32 + j] = t1_[j]; }
+        for (int i = 0; i < 128; ++i)
+          if (i >= n_keys) v[i] = -INFINITY;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_free[i & 1]);            // this warp's part of S(i) is in registers
-      if (ragged) {
+      // row maximum (four independent chains)
+      float mx4[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
-        for (int j = 0; j < 64; ++j)
-          if (key0 + half * 64 + j >= g.kv_len) s_mine[j] = -INFINITY;
-      }
-      // row maximum: four independent chains over this half, then the other half's through shared memory (the two
-      // threads of a row sit in the two warps of one tensor-memory lane quarter and meet on that quarter's barrier)
-      float mx4[4] = {s_mine[0], s_mine[1], s_mine[2], s_mine[3]};
+      for (int i = 4; i < 128; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], v[i]);
+      const float m_new = fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+      if (j == 0) {
+        m = m_new;
+      } else {
+        const bool grow = (m_new - m) * c > kRescaleStep;
+        if (__any_sync(0xffffffffu, grow)) {
+          // O and the row sum move to the new maximum; the product that last wrote O has to be complete
+          const float alpha = grow ? fast_exp2((m - m_new) * c) : 1.f;
+          if (grow) { m = m_new; l *= alpha; }
+          mbar_wait(&o_full[st], (j - 1) & 1, p.status);
+          tc_fence_after();
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            float o[32];
+            tmem_ld_32x32(tmem_o + lane_addr + ch * 32, o);
 #pragma unroll
-      for (int j = 4; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s_mine[j]);
-      const float mx_half = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      float* mxp = mx_part + (i & 1) * 2 * BQ;
-      mxp[half * BQ + r] = mx_half;
-      asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
-      const float mx = fmaxf(m, fmaxf(mx_half, mxp[(half ^ 1) * BQ + r]));
-      const float alpha = fast_exp2((m - mx) * c);
-      m = mx;
-      const float mc = mx * c;
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        s_mine[j] = fast_exp2(fmaf(s_mine[j], c, -mc));
-        sum4[j & 3] += s_mine[j];
-      }
-      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      l = l * alpha + sum;
-      uint4 pk[8];
-#pragma unroll
-      for (int v = 0; v < 8; ++v) pk[v] = pack8_bf16(s_mine + 8 * v);
-      // The previous block's product has had the whole softmax above to finish: fold it into the accumulator (its
-      // completion also frees the P tile).
-      if (i > 0) {
-        mbar_wait(o_full, (i - 1) & 1, p.status);
-        tc_fence_after();
-#pragma unroll
-        for (int cgrp = 0; cgrp < 2; ++cgrp) {
-          float o[32];
-          tmem_ld_32x32(tmem_o + lane_addr + half * 64 + cgrp * 32, o);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha_prev, o[j]);
+            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+            tmem_st_32x32(tmem_o + lane_addr + ch * 32, o);
+          }
         }
       }
-      alpha_prev = alpha;
-      // P row segment: this half's 64 keys are one 128-byte row of 64-key chunk `half`, 8 swizzled 16-byte units
+      // exponentials against m (masked keys: 2^-inf = 0), row sum
+      const float mc = m * c;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int v = 0; v < 8; ++v)
-        *reinterpret_cast<uint4*>(ps + half * (BQ * 128) + r * 128 + ((v ^ (r & 7)) << 4)) = pk[v];
-      fence_proxy_async_smem();
+      for (int i = 0; i < 128; ++i) {
+        v[i] = fast_exp2(fmaf(v[i], c, -mc));
+        sum4[i & 3] += v[i];
+      }
+      // P as bf16 over the first 64 columns of this row of S: column i = keys (2i, 2i+1)
+      {
+        float pk[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+          pk[i] = __uint_as_float(*reinterpret_cast<uint32_t*>(&h2));
+        }
+        tmem_st_32x32_nowait(tmem_s + lane_addr, pk);
+        tmem_st_32x32_nowait(tmem_s + lane_addr + 32, pk + 32);
+        tmem_st_wait();
+      }
+      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
+      if (lane == 0) mbar_arrive(&p_full[st]);
     }
-    if (n_blocks > 0) {
-      mbar_wait(o_full, (n_blocks - 1) & 1, p.status);
+    if (n_st > 0) {
+      mbar_wait(&o_full[st], (n_st - 1) & 1, p.status);
       tc_fence_after();
+    }
+    if (dbg && threadIdx.x == 128) p.debug[3] = globaltimer_ns();
+    // ---- merge the two streams: thread (stream st, row r) finishes columns [64 st, 64 st + 64) of the row
+    float* stat_mine = reinterpret_cast<float*>(smem + S::V_OFF + 2 * st * S::V_BYTES);
+    const float* stat_other = reinterpret_cast<const float*>(smem + S::V_OFF + 2 * (st ^ 1) * S::V_BYTES);
+    stat_mine[r] = m;
+    stat_mine[BQ + r] = l;
+    tc_fence_before();
+    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+    tc_fence_after();
+    const float m_o = n_other > 0 ? stat_other[r] : -INFINITY, l_o = n_other > 0 ? stat_other[BQ + r] : 0.f;
+    const float m_all = fmaxf(m, m_o);
+    const float w_mine = n_st > 0 ? fast_exp2((m - m_all) * c) : 0.f;
+    const float w_other = n_other > 0 ? fast_exp2((m_o - m_all) * c) : 0.f;
+    const float l_row = w_mine * l + w_other * l_o;
+    const uint32_t t_mine = tmem_o + lane_addr + st * 64;
+    const uint32_t t_other = tmem_base + 2 * BKV + (st ^ 1) * HD + lane_addr + st * 64;
+    float acc[64];
 #pragma unroll
-      for (int cgrp = 0; cgrp < 2; ++cgrp) {
-        float o[32];
-        tmem_ld_32x32(tmem_o + lane_addr + half * 64 + cgrp * 32, o);
+    for (int cgrp = 0; cgrp < 2; ++cgrp) {
+      float a[32];
+      if (n_st > 0) {
+        tmem_ld_32x32(t_mine + cgrp * 32, a);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[cgrp * 32 + j] = fmaf(acc[cgrp * 32 + j], alpha_prev, o[j]);
+        for (int i = 0; i < 32; ++i) acc[cgrp * 32 + i] = a[i] * w_mine;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[cgrp * 32 + i] = 0.f;
+      }
+      if (n_other > 0) {
+        tmem_ld_32x32(t_other + cgrp * 32, a);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[cgrp * 32 + i] = fmaf(a[i], w_other, acc[cgrp * 32 + i]);
       }
     }
-    if (dbg && threadIdx.x == 96) p.debug[3] = globaltimer_ns();
-    // ---- combine the two halves' row sums
-    l_part[half * BQ + r] = l;
-    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
-    const float l_row = l_part[r] + l_part[BQ + r];
     if (ksplit == 1) {
       // normalise, store
       const float inv = 1.f / l_row;
       if (r < rows_valid) {
         const int t = p.idx ? p.idx[row0 + r] : row0 + r;
-        __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + half * 64;
+        __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + st * 64;
 #pragma unroll
         for (int i = 0; i < 64; ++i) acc[i] *= inv;
 #pragma unroll
         for (int v = 0; v < 8; ++v) reinterpret_cast<uint4*>(dst)[v] = pack8_bf16(acc + 8 * v);
       }
     } else {
-      // key split: leave the un-normalised row, its maximum and its sum in shared memory for the merge
-      asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");      // every l_part read is done
+      // key split: leave the un-normalised row, its maximum and its sum in shared memory for the merge.  The
+      // operand buffers those go to are idle: both streams' last products were complete before the barrier above.
       float* dump = reinterpret_cast<float*>(smem + S::DUMP_OFF) + (size_t)r * HD;
 #pragma unroll
       for (int v = 0; v < 16; ++v) {
-        const int unit = half * 16 + v;                  // 32 sixteen-byte units per 512-byte row, XOR-swizzled
+        const int unit = st * 16 + v;                    // 32 sixteen-byte units per 512-byte row, XOR-swizzled
         *reinterpret_cast<float4*>(dump + ((unit ^ (r & 7)) << 2)) =
             make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
       }
-      if (half == 0) {
+      if (st == 0) {
         float* stat = reinterpret_cast<float*>(smem + S::STAT_OFF);
-        stat[r] = m;
+        stat[r] = m_all;
         stat[BQ + r] = l_row;
       }
       fence_proxy_async_smem();
@@ -360,7 +432,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     tc_fence_before();
     cluster_sync_all();                                  // every CTA of the cluster is past its key loop
     tc_fence_after();
-    if (warp == 3 && lane < ksplit && lane != z) {
+    if (warp == 4 && lane < ksplit && lane != z) {
       // hand the rows owned by CTA `lane` to it: the rows, their maxima, their sums
       const int k = lane;
       const int slot = z < k ? z : z - 1;
@@ -416,7 +488,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // nobody leaves while a copy out of its shared memory may still be in flight (its receiver has seen it land)
   if (ksplit > 1) cluster_sync_all(); else __syncthreads();
   if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
-  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
