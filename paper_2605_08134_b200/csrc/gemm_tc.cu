@@ -2,9 +2,10 @@
 // Alg. 1 lines 2, 7, 11).  One CTA = one 128 x 256 output tile over one slice of the reduction dimension:
 //   warp 0    TMA producer: a 128-row A tile and a 256-row W tile per 64 k-elements (128 bytes per row, 128-byte
 //             swizzle) into a ring of 4 stages
-//   warp 1    allocates tensor memory; one thread issues tcgen05.mma (M = 128, N = 256, K = 16: a single-CTA MMA
-//             costs about the same time whatever its N, so only the widest N runs the tensor pipe at full rate)
-//             into a 128 x 256 fp32 accumulator and commits each stage back to the producer
+//   warp 1    allocates tensor memory; one elected lane issues tcgen05.mma (M = 128, N = 256, K = 16) into a
+//             128 x 256 fp32 accumulator and commits each stage back to the producer.  The tensor pipe runs at full
+//             rate down to N = 128, but what an SM can pull from the L2 bounds the main loop of these projections,
+//             and the widest tile re-reads the least per flop.
 //   warps 2-5 epilogue: each thread owns one output row (one TMEM lane)
 // Split-K: when a launch has too few tiles to fill the GPU, the two CTAs of a thread-block cluster share a tile, each
 // over half of the reduction.  Every CTA first moves its fp32 accumulator from tensor memory into its own shared
@@ -102,7 +103,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   uint64_t* recv_bar = accum_bar + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(recv_bar + 1);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the warp index through a shuffle: the compiler then knows the role decisions and the descriptors derived from
+  // it to be uniform over the warp
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int nt = blockIdx.x, mt = blockIdx.y;
   const int splits = gridDim.z;                 // = cluster size along z
   const int z = (int)cluster_ctarank();
@@ -193,13 +196,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   RowBatch rb;
 
   if (active) {
+  // The producer and the MMA warp run their loops converged (every lane polls the barriers) and one elected lane
+  // issues: the operands of the copies and MMAs are then warp-uniform values, which is what those instructions take.
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int i = 0; i < n_early; ++i)          // the W halves of these stages are already on their way
         tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
-      for (int i = n_early; i < nkb; ++i) {
-        const int s = i % STAGES;
-        mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
+    }
+    __syncwarp();
+    for (int i = n_early; i < nkb; ++i) {
+      const int s = i % STAGES;
+      mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
+      if (elect_one()) {
         uint8_t* a_dst = smem + s * STAGE_BYTES;
         mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
         tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
@@ -210,16 +218,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
         }
       }
+      __syncwarp();
     }
-    __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(BM, BN);
-      for (int i = 0; i < nkb; ++i) {
-        const int s = i % STAGES;
-        mbar_wait(&full_bar[s], (i / STAGES) & 1, p.status);
-        tc_fence_after();
-        if (dbg && i == 0) p.debug[2] = globaltimer_ns();
+    constexpr uint32_t idesc = idesc_bf16(BM, BN);
+    for (int i = 0; i < nkb; ++i) {
+      const int s = i % STAGES;
+      mbar_wait(&full_bar[s], (i / STAGES) & 1, p.status);
+      tc_fence_after();
+      if (dbg && i == 0 && lane == 0) p.debug[2] = globaltimer_ns();
+      if (elect_one()) {
         const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
         const uint64_t a_desc = smem_desc_k_sw128(a_addr);
         const uint64_t b_desc = smem_desc_k_sw128(a_addr + A_BYTES);
@@ -227,10 +235,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int k = 0; k < BK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
           umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
         umma_commit(&empty_bar[s]);
+        if (i == nkb - 1) umma_commit(accum_bar);      // by the thread that issued the MMAs it covers
       }
-      umma_commit(accum_bar);
+      __syncwarp();
     }
-    __syncwarp();
   } else {
     // While the main loop runs, pull the table rows the finishing pass of this CTA will read into the L2
     // (dense tiles; 512 bytes = 4 lines per row and table).

@@ -145,7 +145,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
         e = launch_gemm_tc(EPI_KV, 128, S.a_xg, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
                            pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
-        // Many tokens: even a small refreshed fraction fills the GPU with full-rate 256-wide tiles.
+        // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
         e = launch_gemm_tc(EPI_KV, 256, S.a_xg, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st); ++launches;
       }
     } else {

@@ -52,7 +52,8 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
                                 cudaStream_t st);
 
 // grid = (n_tiles of bn columns, m_tiles of 128 rows, splits of the reduction dimension = cluster size: 1 or 2);
-// bn = 256 (full tensor rate) or 128 (more CTAs for the weight-streaming K/V projection of a small refresh set).
+// bn = 256 (least re-reading per flop) or 128 (more CTAs for the weight-streaming K/V projection of a small refresh
+// set).
 // The W tensor maps must have a box of bn rows.
 // Row-major bf16 matrix [rows, cols] as a TMA tensor map with a box of 64 columns x box_rows rows, 128-byte swizzle.
 bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
