@@ -282,7 +282,7 @@ def run_ours(args):
             rows.append({"kernel": name, "us": round(us, 2)})
     dom = max((r for r in rows if "bound" in r), key=lambda r: r["us"])
     # DRAM bytes per launch of that kernel from one ncu capture of this workload (profiles/ holds the summaries)
-    ncu_traffic = {"q_gemm": 38.5e6, "kv_gemm": 69.0e6, "out_gemm": 38.2e6}
+    ncu_traffic = {"q_gemm": 38.4e6, "kv_gemm": 69.3e6, "out_gemm": 37.9e6}
     roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
                 "unit": dom["unit"], "frac": dom["frac"],
                 "traffic": ncu_traffic.get(dom["kernel"]) if shape.name == wl.LLADA_LAYER.name else None,

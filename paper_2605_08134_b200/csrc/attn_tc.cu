@@ -297,6 +297,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (dbg && j == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
       const int key0 = (z + (2 * j + st) * ksplit) * BKV;
       const int n_keys = min(BKV, g.kv_len - key0);   // the last block may be ragged: keys past kv_len do not exist
+      // O and the row sum move to a new maximum only when it grew by more than kRescaleStep (in log2 units); the
+      // product that last wrote O has to be complete before O is rescaled in place
+      auto settle_max = [&](float m_new) {
+        if (j == 0) {
+          m = m_new;
+        } else {
+          const bool grow = (m_new - m) * c > kRescaleStep;
+          if (__any_sync(0xffffffffu, grow)) {
+            const float alpha = grow ? fast_exp2((m - m_new) * c) : 1.f;
+            if (grow) { m = m_new; l *= alpha; }
+            mbar_wait(&o_full[st], (j - 1) & 1, p.status);
+            tc_fence_after();
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+              float o[32];
+              tmem_ld_32x32(tmem_o + lane_addr + ch * 32, o);
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] *= alpha;
+              tmem_st_32x32(tmem_o + lane_addr + ch * 32, o);
+            }
+          }
+        }
+      };
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       // the row of S: four loads in flight together
       float v[128];
       tmem_ld_32x32_nowait(tmem_s + lane_addr, v);
@@ -313,30 +337,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       float mx4[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
       for (int i = 4; i < 128; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], v[i]);
-      const float m_new = fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
-      if (j == 0) {
-        m = m_new;
-      } else {
-        const bool grow = (m_new - m) * c > kRescaleStep;
-        if (__any_sync(0xffffffffu, grow)) {
-          // O and the row sum move to the new maximum; the product that last wrote O has to be complete
-          const float alpha = grow ? fast_exp2((m - m_new) * c) : 1.f;
-          if (grow) { m = m_new; l *= alpha; }
-          mbar_wait(&o_full[st], (j - 1) & 1, p.status);
-          tc_fence_after();
-#pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            float o[32];
-            tmem_ld_32x32(tmem_o + lane_addr + ch * 32, o);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] *= alpha;
-            tmem_st_32x32(tmem_o + lane_addr + ch * 32, o);
-          }
-        }
-      }
+      settle_max(fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]))));
       // exponentials against m (masked keys: 2^-inf = 0), row sum
       const float mc = m * c;
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < 128; ++i) {
         v[i] = fast_exp2(fmaf(v[i], c, -mc));
@@ -488,6 +491,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // nobody leaves while a copy out of its shared memory may still be in flight (its receiver has seen it land)
   if (ksplit > 1) cluster_sync_all(); else __syncthreads();
   if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
+  if (p.debug != nullptr && threadIdx.x == 0) {      // latest end over the CTAs that had work, and their number
+    atomicMax(&p.debug[6], globaltimer_ns());
+    atomicAdd(&p.debug[7], 1ull);
+  }
   if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
 }
 

@@ -115,3 +115,60 @@ def test_row_sparse_attention_with_key_split(dare):
     parity.compare_step(g2, o2, hs2.first(), 2, 0.1, shape2, first=True)
     parity.compare_step(g2, o2, hs2.advance(wl.uniform_positions(hs2.rng, shape2, 70)), 2, 0.1, shape2)
     g.close(); g2.close()
+
+
+def test_single_key_block(dare):
+    """kv_len below one key block: one of the attention kernel's two key-block streams has nothing to do."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=2, seq=96, prompt=32)
+    w = wl.make_weights(shape, 12)
+    hs = wl.HiddenStream(shape, 12)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    for mode in (3, 2, 0):
+        parity.compare_step(g, o, hs.advance(wl.uniform_positions(hs.rng, shape, 17)), mode, 0.1, shape)
+    g.close()
+
+
+def test_peaked_softmax_rescales_the_accumulator(dare):
+    """Sharp attention (large query/key projections): the running row maximum of a key-block stream jumps by more
+    than the kernel's lazy-rescaling step (2^8), so the in-place rescale of the tensor-memory accumulator runs.
+    The jump is checked on the oracle's own scores.  With logits this large the bf16 rounding of Q and K, which
+    both kernel paths share and the fp64 oracle does not, dominates the distance to the oracle, so the tensor path
+    is held to the CUDA-core path here (same rounded operands, fp32 softmax over all keys at once) and only the
+    index set to the oracle."""
+    from oracle import dare_oracle as orc
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=1, seq=1280, prompt=640)
+    w = wl.make_weights(shape, 44)
+    for k in ("w_q", "w_k"):
+        w[k] = wl.round_to(w[k] * np.float32(6.0), shape.dtype)
+    hs = wl.HiddenStream(shape, 44)
+    x0 = hs.first()
+    ch = wl.uniform_positions(hs.rng, shape, 150)
+    x1 = hs.advance(ch)
+    # the oracle's logits of step 0: does some row's maximum over the blocks of one stream grow by > 8 / log2(e)?
+    xn = orc.rmsnorm(x0[0], w["rms_gain"], shape.rms_eps)
+    pos = np.arange(shape.seq)
+    q = orc.rope(orc.linear(xn, w["w_q"]), pos, shape.n_heads, shape.head_dim, shape.rope_theta)
+    k = orc.rope(orc.linear(xn, w["w_k"]), pos, shape.n_heads, shape.head_dim, shape.rope_theta)
+    jumps = 0
+    for h in range(shape.n_heads):
+        sl = slice(h * 128, (h + 1) * 128)
+        logit = q[:, sl] @ k[:, sl].T / np.sqrt(128.0)
+        blockmax = logit.reshape(shape.seq, shape.seq // 128, 128).max(axis=2)      # [row, block]
+        for st in range(2):
+            bm = blockmax[:, st::2]
+            run = np.maximum.accumulate(bm, axis=1)
+            jumps += int(((run[:, 1:] - run[:, :-1]) > 8.0 / np.log2(np.e)).sum())
+    assert jumps > 50, jumps
+    a = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    b = dare.Layer(shape, w, kernel_path=dare.PATH_SIMT)
+    o = parity.oracle_layer(shape, w)
+    for x, mode in ((x0, 0), (x1, 3)):
+        ya = a.step(parity.to_device(x, shape), mode, 0.1)
+        yb = b.step(parity.to_device(x, shape), mode, 0.1)
+        o.step(x, mode, 0.1)
+        parity.assert_close("tensor vs cuda-core", ya.float().cpu().numpy(), yb.float().cpu().numpy(), 2e-2)
+    np.testing.assert_array_equal(a.last_selection(1, shape.seq)["idx"], o.last_idx)
+    np.testing.assert_array_equal(a.last_selection(1, shape.seq)["idx"], b.last_selection(1, shape.seq)["idx"])
+    a.close(); b.close()
