@@ -70,13 +70,7 @@ size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) 
   B.debug = (unsigned long long*)take((64 + 3 * 1024) * sizeof(unsigned long long));
   B.x_stage = take(Tm * d * e);
   B.y_stage = take(Tm * d * e);
-  if (use_tc) {
-    B.xg = take((Tm + 128) * d * e);  // gathered rows of x_norm, padded to a whole tile
-    B.tmp = nullptr;
-  } else {
-    B.xg = nullptr;
-    B.tmp = (float*)take(Tm * 2 * d * sizeof(float));
-  }
+  B.tmp = use_tc ? nullptr : (float*)take(Tm * 2 * d * sizeof(float));
   return off;
 }
 
@@ -114,8 +108,7 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
   prof_mark(L, SLOT_SELECT, st);
-  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, nullptr,
-                nullptr, 0, st); ++launches;
+  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st); ++launches;
   // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
   const int* kv_idx = kv_sparse ? B.idx : nullptr;
   const int* kv_cnt = kv_sparse ? B.count : nullptr;
@@ -258,7 +251,6 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
     if (e == cudaSuccess) e = cudaMemset(L->buf.kc, 0, cache_bytes);
     if (e == cudaSuccess) e = cudaMemset(L->buf.vc, 0, cache_bytes);
     if (e == cudaSuccess) e = cudaMemset(L->buf.oc, 0, cache_bytes);
-    if (e == cudaSuccess && L->buf.xg) e = cudaMemset(L->buf.xg, 0, cache_bytes + (size_t)128 * cfg->d_model * 2);
   }
   if (e == cudaSuccess) {
     launch_rope_table(L->buf.rope_cs, cfg->max_seq, cfg->head_dim, (double)cfg->rope_theta, 0);

@@ -149,23 +149,15 @@ template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, 
 // written as an ascending index list by warp ballot + popcount + a block prefix sum over warp totals; the
 // staleness counters of Sec. 4 are updated in the same pass.  A CTA walks the tokens in chunks of 1024, which
 // keeps the list ordered without any inter-CTA hand-off (T <= a few 10^4 per layer step).
-// With a gather attached (Alg. 1 line 6: x_norm restricted to the refresh set) the kernel runs on several CTAs:
-// every CTA repeats the cheap compaction for itself, CTA 0 publishes it, and CTA c copies the rows r of the
-// compacted matrix with r % gridDim.x == c.
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
-                                                      int* __restrict__ batch_off, int* __restrict__ delta,
-                                                      const uint4* __restrict__ gather_src,
-                                                      uint4* __restrict__ gather_dst, int row_vecs) {
-  extern __shared__ int my_rows[];          // tokens whose rows this CTA copies (gather only)
+                                                      int* __restrict__ batch_off, int* __restrict__ delta) {
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const bool publish = blockIdx.x == 0;
-  const int G = gridDim.x;
   int base = 0;
   for (int start = 0; start < T; start += 1024) {
     const int t = start + threadIdx.x;
@@ -189,52 +181,32 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
     __syncthreads();
     if (sel) {
       const int out = base + warp_excl[warp] + lane_prefix;
-      if (publish) idx[out] = t;
-      if (gather_dst != nullptr && out % G == (int)blockIdx.x) my_rows[out / G] = t;
+      idx[out] = t;
     }
-    if (publish && valid) {
+    if (valid) {
       const int cr = g.cache_row(t);
       delta[cr] = sel ? 0 : delta[cr] + 1;
     }
     base += chunk_total;
     __syncthreads();
   }
-  if (publish) {
-    if (threadIdx.x == 0) *count = base;
-    // start of each sequence's slice: lower bound of b*seq_act in the ascending list
-    for (int b = threadIdx.x; b <= g.batch; b += blockDim.x) {
-      const int key = b * g.seq_act;
-      int lo = 0, hi = base;
-      while (lo < hi) {
-        int mid = (lo + hi) >> 1;
-        if (idx[mid] < key) lo = mid + 1; else hi = mid;
-      }
-      batch_off[b] = lo;
+  if (threadIdx.x == 0) *count = base;
+  // start of each sequence's slice: lower bound of b*seq_act in the ascending list
+  for (int b = threadIdx.x; b <= g.batch; b += blockDim.x) {
+    const int key = b * g.seq_act;
+    int lo = 0, hi = base;
+    while (lo < hi) {
+      int mid = (lo + hi) >> 1;
+      if (idx[mid] < key) lo = mid + 1; else hi = mid;
     }
-  }
-  if (gather_dst != nullptr) {
-    const int mine = base > (int)blockIdx.x ? (base - (int)blockIdx.x + G - 1) / G : 0;
-    for (int k = 0; k < mine; ++k) {
-      const uint4* s = gather_src + (size_t)my_rows[k] * row_vecs;
-      uint4* o = gather_dst + ((size_t)k * G + blockIdx.x) * row_vecs;
-      for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) o[v] = s[v];
-    }
+    batch_off[b] = lo;
   }
 }
 
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, const void* gather_src, void* gather_dst, int row_bytes,
-                   cudaStream_t st) {
-  const int T = g.tokens();
-  int grid = 1;
-  size_t smem = 0;
-  if (gather_dst != nullptr) {
-    grid = T < 64 ? (T > 0 ? T : 1) : 64;
-    smem = ((size_t)(T + grid - 1) / grid + 1) * sizeof(int);
-  }
-  launch_pdl(select_kernel, dim3(grid), dim3(1024), smem, st, 1, scores, tau, (select_all || scores == nullptr) ? 1 : 0,
-             g, idx, count, batch_off, delta, reinterpret_cast<const uint4*>(gather_src),
-             reinterpret_cast<uint4*>(gather_dst), row_bytes / 16);
+                   int* batch_off, int* delta, cudaStream_t st) {
+  launch_pdl(select_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, (select_all || scores == nullptr) ? 1 : 0, g, idx,
+             count, batch_off, delta);
 }
 
 // ------------------------------------------------------------------------------------------------ row gather

@@ -63,10 +63,8 @@ void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaS
 template <typename T>
 void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st);
 // Threshold + ballot/prefix-sum compaction + staleness update.  `scores == nullptr` or `select_all` selects all.
-// With gather_dst != nullptr the rows src[idx[r]] (row_bytes each, multiple of 16) are also copied to dst[r].
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, const void* gather_src, void* gather_dst, int row_bytes,
-                   cudaStream_t st);
+                   int* batch_off, int* delta, cudaStream_t st);
 template <typename T>
 void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
 

@@ -131,8 +131,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     pdl_wait();
     if (mt * BM >= min(*p.count, p.m_total)) return;     // uniform over the cluster
   }
+  // Gathered A operand: the four epilogue warps fetch the rows of the refresh set themselves, 16 bytes at a time,
+  // into the swizzled tile layout (the TMA producer then only brings the W tiles); each of them arrives on a stage
+  // once its rows of that stage have landed.
+  const bool gather = p.gather_src != nullptr;
+  const uint32_t tx_bytes = gather ? (uint32_t)Cfg<BN>::B_BYTES : (uint32_t)STAGE_BYTES;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], gather ? 5 : 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(accum_bar, 1);
     mbar_init(recv_bar, 1);
     fence_mbar_init();
@@ -153,7 +158,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int n_early = likely ? (nkb < STAGES ? nkb : STAGES) : 0;
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
-      mbar_arrive_expect_tx(&full_bar[i], STAGE_BYTES);
+      mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
       uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
       if (p.b_pair) {
         tma_load_2d(b_dst, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[i]);
@@ -199,7 +204,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // The producer and the MMA warp run their loops converged (every lane polls the barriers) and one elected lane
   // issues: the operands of the copies and MMAs are then warp-uniform values, which is what those instructions take.
   if (warp == 0) {
-    if (elect_one()) {
+    if (!gather && elect_one()) {
       for (int i = 0; i < n_early; ++i)          // the W halves of these stages are already on their way
         tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
     }
@@ -209,8 +214,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
       if (elect_one()) {
         uint8_t* a_dst = smem + s * STAGE_BYTES;
-        mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
-        tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
+        mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
+        if (!gather) tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
         if (p.b_pair) {
           tma_load_2d(a_dst + A_BYTES, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[s]);
           tma_load_2d(a_dst + A_BYTES + Cfg<BN>::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[s]);
@@ -252,6 +257,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
     // the table reads of this warp's first rows of the finishing pass: in flight for the whole main loop
     load_row_batch<EPI>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+    if (gather) {
+      // One stage of the A tile = 128 rows x 128 bytes (64 k-elements).  A warp takes 32 rows; one of its copy
+      // instructions covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row, so every
+      // request is a whole 128-byte line.
+      const int r_own = quarter * 32 + lane;                   // the row whose token this lane looks up
+      const int tok_own = r_own < rows_valid ? p.idx[t0 + r_own] : -1;
+      const uint8_t* src_k[8];
+      uint32_t dst_k[8], bytes_k[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int rw = k * 4 + (lane >> 3), r = quarter * 32 + rw, u = lane & 7;
+        const int tok = __shfl_sync(0xffffffffu, tok_own, rw);
+        src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)(tok >= 0 ? tok : 0) * p.K * 2 +
+                   (size_t)kb_begin * (BK * 2) + u * 16;
+        bytes_k[k] = tok >= 0 ? 16u : 0u;                       // rows past the refresh set are zero-filled
+        dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
+      }
+      constexpr int LAG = STAGES - 2;                           // copy groups in flight per thread
+      for (int i = 0; i < nkb + LAG; ++i) {
+        if (i < nkb) {
+          const int s = i % STAGES;
+          mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)i * (BK * 2), bytes_k[k]);
+        }
+        cp_async_commit();                                      // (empty groups at the tail keep the lag uniform)
+        if (i >= LAG) {
+          cp_async_wait<LAG>();                                 // this thread's copies of stage i - LAG have landed
+          fence_proxy_async_smem();                             // ... and are visible to the tensor core's reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full_bar[(i - LAG) % STAGES]);
+        }
+      }
+    }
     mbar_wait(accum_bar, 0, p.status);
     tc_fence_after();
     if (dbg && threadIdx.x == 64) p.debug[3] = globaltimer_ns();
@@ -421,8 +461,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
   } else if (warp == 0 && lane == 0) {
     // a tile past the refresh set: complete the stages whose W halves were started early, then let them land
-    for (int i = 0; i < n_early; ++i) tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, 0, &full_bar[i]);
-    for (int i = 0; i < n_early; ++i) mbar_wait(&full_bar[i], 0, p.status);
+    if (!gather) {
+      for (int i = 0; i < n_early; ++i) tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, 0, &full_bar[i]);
+      for (int i = 0; i < n_early; ++i) mbar_wait(&full_bar[i], 0, p.status);
+    } else {
+      // the barrier also counts the four gathering warps, which do not run here: stand in for them
+      for (int i = 0; i < n_early; ++i) {
+        for (int k = 0; k < 4; ++k) mbar_arrive(&full_bar[i]);
+        mbar_wait(&full_bar[i], 0, p.status);
+      }
+    }
   }
   tc_fence_before();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)

@@ -23,7 +23,6 @@ struct Buffers {
   unsigned long long* debug;  // [64] kernel phase timestamps (diagnostics, written by block (0,0) when enabled)
   void* x_stage;    // [T, d] staging for the host-buffer entry point
   void* y_stage;
-  void* xg;         // tensor-core path: gathered x_norm rows
   float* tmp;       // SIMT path: fp32 projection results [T, 2d]
 };
 

@@ -7,7 +7,7 @@
 namespace dare {
 
 struct TcState {
-  CUtensorMap a_xn, a_xg, a_oc;            // A operands, box 64 x 128 rows
+  CUtensorMap a_xn, a_oc;                  // A operands, box 64 x 128 rows
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 256 rows
   CUtensorMap w_k128, w_v128;              // weights, box 64 x 128 rows
   CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 128 rows (keys)
@@ -64,7 +64,7 @@ dare_status_t tc_create(dare_layer* L) {
   TcState* s = new (std::nothrow) TcState();
   if (!s) return DARE_ERR_INVALID_ARG;
   const uint64_t Tm = (uint64_t)L->cfg.max_batch * L->cfg.max_seq, d = L->cfg.d_model;
-  bool ok = make_map(&s->a_xn, L->buf.xn, Tm, d, 128) && make_map(&s->a_xg, L->buf.xg, Tm + 128, d, 128) &&
+  bool ok = make_map(&s->a_xn, L->buf.xn, Tm, d, 128) &&
             make_map(&s->a_oc, L->buf.oc, Tm, d, 128) && make_map(&s->w_q, L->w.w_q, d, d, 256) &&
             make_map(&s->w_k, L->w.w_k, d, d, 256) && make_map(&s->w_v, L->w.w_v, d, d, 256) &&
             make_map(&s->w_o, L->w.w_o, d, d, 256) && make_map(&s->w_k128, L->w.w_k, d, d, 128) &&
@@ -98,6 +98,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   GemmParams base;
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
+  base.gather_src = nullptr;
   base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
   base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
@@ -123,9 +124,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   }
   // lines 4-5 + Sec. 4
   prof_mark(L, SLOT_SELECT, st);
-  // (+ Alg. 1 line 6 when K/V reuse is on: the refresh set's rows of x_norm, compacted, for the gathered projection)
-  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta,
-                kv_sparse ? B.xn : nullptr, kv_sparse ? B.xg : nullptr, d * 2, st); ++launches;
+  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st);
+  ++launches;
   // K/V projection with rotary embedding and cache scatter
   {
     GemmParams p = base;
@@ -134,7 +134,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     p.debug = dbg ? dbg + 8 : nullptr;
     const int n_tiles = 2 * d / 256;
     if (kv_sparse) {
-      p.idx = B.idx; p.count = B.count;
+      // Alg. 1 line 6: the projection fetches the refresh set's rows of x_norm by index as its A operand
+      p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.xn;
       const int m_tiles = (T_ + 127) / 128;
       prof_mark(L, SLOT_KV_GEMM, st);
       if (m_tiles <= 8) {
@@ -142,11 +143,11 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
         // Narrower tiles put twice as many CTAs on it; the reduction split is sized for one row tile.
         p.n_split = d / 128;
         const int n_tiles128 = 2 * d / 128;
-        e = launch_gemm_tc(EPI_KV, 128, S.a_xg, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
+        e = launch_gemm_tc(EPI_KV, 128, S.a_xn, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
                            pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
-        e = launch_gemm_tc(EPI_KV, 256, S.a_xg, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st); ++launches;
+        e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st); ++launches;
       }
     } else {
       prof_mark(L, SLOT_KV_GEMM, st);

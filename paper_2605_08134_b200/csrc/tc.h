@@ -18,6 +18,8 @@ struct GemmParams {
   int a_row0;            // first row of the window in A's row space
   const int* idx;        // gathered: token of each A row (ascending refresh set), else nullptr
   const int* count;      // gathered: device count of rows, else nullptr
+  const __nv_bfloat16* gather_src;  // gathered: the matrix [*, K] whose rows idx[] the kernel fetches itself as its A
+                                    // operand (Alg. 1 line 6); nullptr: A comes through the tensor map
   StepGeom g;
   int n_split;           // n-tiles [0, n_split) use W0/out0, the rest W1/out1
   __nv_bfloat16* out0;

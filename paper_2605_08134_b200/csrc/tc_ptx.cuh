@@ -211,6 +211,15 @@ __device__ __forceinline__ void tmem_st_32x32_nowait(uint32_t taddr, const float
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// ---- asynchronous 16-byte copies global -> shared (Ampere-style), for operand rows fetched by index ----
+// src_bytes = 16 copies, 0 fills the 16 bytes with zeros (the source address still has to be valid).
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gsrc, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // ---- programmatic dependent launch ----
 // A kernel launched with the programmatic-serialization attribute may start while its predecessor in the stream is
 // still running.  pdl_wait() blocks until the predecessor has completed and its writes are visible; everything
