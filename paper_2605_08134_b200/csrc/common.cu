@@ -162,6 +162,9 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
   for (int start = 0; start < T; start += 1024) {
     const int t = start + threadIdx.x;
     const bool valid = t < T;
+    // both loads of the token first (score and staleness counter): one memory round trip instead of two
+    const int cr = valid ? g.cache_row(t) : 0;
+    const int stale = valid ? delta[cr] : 0;
     bool sel = false;
     if (valid) sel = select_all ? true : !(scores[t] <= tau);
     const unsigned bal = __ballot_sync(0xffffffffu, sel);
@@ -179,27 +182,19 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
       if (lane == 31) chunk_total = inc;
     }
     __syncthreads();
-    if (sel) {
-      const int out = base + warp_excl[warp] + lane_prefix;
-      idx[out] = t;
-    }
     if (valid) {
-      const int cr = g.cache_row(t);
-      delta[cr] = sel ? 0 : delta[cr] + 1;
+      const int out = base + warp_excl[warp] + lane_prefix;     // place of this token in the list, were it selected
+      if (sel) idx[out] = t;
+      // a sequence starts at this token: its slice of the ascending list starts here
+      if (t % g.seq_act == 0) batch_off[t / g.seq_act] = out;
+      delta[cr] = sel ? 0 : stale + 1;
     }
     base += chunk_total;
     __syncthreads();
   }
-  if (threadIdx.x == 0) *count = base;
-  // start of each sequence's slice: lower bound of b*seq_act in the ascending list
-  for (int b = threadIdx.x; b <= g.batch; b += blockDim.x) {
-    const int key = b * g.seq_act;
-    int lo = 0, hi = base;
-    while (lo < hi) {
-      int mid = (lo + hi) >> 1;
-      if (idx[mid] < key) lo = mid + 1; else hi = mid;
-    }
-    batch_off[b] = lo;
+  if (threadIdx.x == 0) {
+    *count = base;
+    batch_off[g.batch] = base;
   }
 }
 
