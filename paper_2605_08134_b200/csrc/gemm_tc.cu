@@ -6,7 +6,9 @@
 //             128 x 256 fp32 accumulator and commits each stage back to the producer.  The tensor pipe runs at full
 //             rate down to N = 128, but what an SM can pull from the L2 bounds the main loop of these projections,
 //             and the widest tile re-reads the least per flop.
-//   warps 2-5 epilogue: each thread owns one output row (one TMEM lane)
+//   warps 2-7 wait for the accumulator (warps 2-5 are also the A-operand producers of a gathered launch); afterwards
+//             all warps finish rows, and move the accumulator out of tensor memory first (thread <-> row; with eight
+//             warps the two warps of a TMEM lane quarter take half of the columns each)
 // Split-K: when a launch has too few tiles to fill the GPU, the two CTAs of a thread-block cluster share a tile, each
 // over half of the reduction.  Every CTA first moves its fp32 accumulator from tensor memory into its own shared
 // memory (the operand ring is idle by then).  The halves are then combined by a reduce-scatter over distributed
@@ -48,8 +50,20 @@ struct Cfg {
 // row-per-warp reads); [128 KB, 192 KB) the partner's partial of the 64 rows this CTA owns (split-K only).
 }  // namespace
 
-// Finishing pass, per warp: RB rows at a time (rows rl0, rl0 + 6, ...); their table reads are issued together.
-constexpr int RB = 6;
+// Finishing pass, per warp: RB rows at a time (rows rl0, rl0 + #warps, ...); their table reads are issued together.
+// Warps of a CTA: producer, MMA issuer, the rest wait for the accumulator; all of them finish rows.
+#ifndef DARE_GEMM_WARPS_NARROW
+#define DARE_GEMM_WARPS_NARROW 6
+#endif
+#ifndef DARE_GEMM_WARPS_WIDE
+#define DARE_GEMM_WARPS_WIDE 8
+#endif
+template <int BN>
+struct Warps {
+  static constexpr int N = BN == 128 ? DARE_GEMM_WARPS_NARROW : DARE_GEMM_WARPS_WIDE;
+  static constexpr int RB = N == 8 ? 4 : 6;          // rows a warp finishes at a time
+};
+template <int RB>
 struct RowBatch {
   int tok[RB];
   int row[RB];            // place of the row in the launch's (possibly gathered) row list
@@ -59,13 +73,13 @@ struct RowBatch {
   float2 qa[RB], qb[RB];  // stored query of the scoring head: elements 2*lane.. and 64 + 2*lane..
 };
 
-template <int EPI>
-__device__ __forceinline__ void load_row_batch(RowBatch& rb, const GemmParams& p, int rl0, int z, int rows_per_cta,
+template <int EPI, int RB, int kWarps>
+__device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParams& p, int rl0, int z, int rows_per_cta,
                                                int rows_valid, int t0, int pos0, size_t crow0, bool rotate,
                                                bool score_tile, int lane) {
 #pragma unroll
   for (int k = 0; k < RB; ++k) {
-    const int rl = rl0 + 6 * k;
+    const int rl = rl0 + kWarps * k;
     const int r = z * rows_per_cta + rl;
     rb.ok[k] = rl < rows_per_cta && r < rows_valid;
     const int rc = rb.ok[k] ? r : 0;              // rows that do not exist read row 0's tables and are dropped later
@@ -90,10 +104,11 @@ __device__ __forceinline__ void load_row_batch(RowBatch& rb, const GemmParams& p
 }
 
 template <int EPI, int BN>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(Warps<BN>::N * 32, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
   constexpr int STAGES = Cfg<BN>::STAGES, STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
+  constexpr int kWarps = Warps<BN>::N, RB = Warps<BN>::RB;
   constexpr int PROW_BYTES = Cfg<BN>::PROW_BYTES, RECV_OFFSET = Cfg<BN>::RECV_OFFSET;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -198,7 +213,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
   const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
-  RowBatch rb;
+  RowBatch<RB> rb;
 
   if (active) {
   // The producer and the MMA warp run their loops converged (every lane polls the barriers) and one elected lane
@@ -248,7 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // While the main loop runs, pull the table rows the finishing pass of this CTA will read into the L2
     // (dense tiles; 512 bytes = 4 lines per row and table).
     if (p.idx == nullptr) {
-      for (int i = threadIdx.x - 64; i < rows_per_cta * 4; i += 128) {
+      for (int i = threadIdx.x - 64; i < rows_per_cta * 4; i += (kWarps - 2) * 32) {
         const int r = z * rows_per_cta + (i >> 2);
         if (r >= rows_valid) break;
         if (rotate) prefetch_l2(p.rope + (size_t)(pos0 + r) * (HD / 2) + (i & 3) * 16);
@@ -256,8 +271,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
     // the table reads of this warp's first rows of the finishing pass: in flight for the whole main loop
-    load_row_batch<EPI>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
-    if (gather) {
+    load_row_batch<EPI, RB, kWarps>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+    if (gather && warp < 6) {
       // One stage of the A tile = 128 rows x 128 bytes (64 k-elements).  A warp takes 32 rows; one of its copy
       // instructions covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row, so every
       // request is a whole 128-byte line.
@@ -300,20 +315,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   // The table reads of the first rows the producer and MMA warps will finish start now (those of the other warps
   // started before the main loop) and land during the exchange below.
-  if (warp < 2) load_row_batch<EPI>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+  if (warp < 2) load_row_batch<EPI, RB, kWarps>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
 
   // ---- every CTA of the cluster has finished its main loop: the rings are free to receive partial rows
   tc_fence_before();
   if (splits > 1) cluster_sync_all(); else __syncthreads();
   tc_fence_after();
   if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[32] = globaltimer_ns();
-  if (warp >= 2) {
-    // this warp's 32 rows of the partial accumulator: tensor memory -> own shared memory, thread <-> row
+  if (kWarps == 8 || warp >= 2) {
+    // The partial accumulator: tensor memory -> own shared memory, thread <-> row.  With eight warps the two warps
+    // of a lane quarter (w and w + 4) take half of the columns each; with six, warps 2-5 take a quarter each.
     const int r = quarter * 32 + lane;
     const uint32_t dst = smem_u32(smem + (size_t)r * PROW_BYTES);
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    constexpr int ch_n = kWarps == 8 ? BN / 64 : BN / 32;
+    const int ch0 = kWarps == 8 ? (warp >> 2) * ch_n : 0;
 #pragma unroll 1
-    for (int ch = 0; ch < BN / 32; ++ch) {
+    for (int ch = ch0; ch < ch0 + ch_n; ++ch) {
       float v[32];
       tmem_ld_32x32(t_lane + ch * 32, v);
 #pragma unroll
@@ -325,8 +343,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const int owner = r / rows_per_cta;
       if (owner != z) {                            // hand the 32 rows to their owner: one 32 KB bulk copy
         fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
+        if (kWarps == 8) asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory");   // both warps of the quarter
+        else __syncwarp();
+        if ((kWarps != 8 || warp < 4) && lane == 0) {
           const int rl0 = quarter * 32 - owner * rows_per_cta;
           const uint32_t src = smem_u32(smem + (size_t)(quarter * 32) * PROW_BYTES);
           const uint32_t rdst = map_to_cta(smem_u32(smem + RECV_OFFSET + (size_t)rl0 * PROW_BYTES), (uint32_t)owner);
@@ -346,14 +365,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   {
     __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
 #pragma unroll 1
-    for (int rl0 = warp; rl0 < rows_per_cta; rl0 += 6 * RB) {
-      if (rl0 != warp) load_row_batch<EPI>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
-      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[34 + (rl0 - warp) / (6 * RB) * 2] = globaltimer_ns();
+    for (int rl0 = warp; rl0 < rows_per_cta; rl0 += kWarps * RB) {
+      if (rl0 != warp) load_row_batch<EPI, RB, kWarps>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[34 + (rl0 - warp) / (kWarps * RB) * 2] = globaltimer_ns();
       // (1) combine the partial rows: lane <-> pairs (2*lane, 2*lane+1) of each head
       float2 vlo[RB][BN / HD], vhi[RB][BN / HD];
 #pragma unroll
       for (int k = 0; k < RB; ++k) {
-        const int rl = rb.ok[k] ? rl0 + 6 * k : warp;     // rows that do not exist re-read an existing one
+        const int rl = rb.ok[k] ? rl0 + kWarps * k : warp;     // rows that do not exist re-read an existing one
 #pragma unroll
         for (int hh = 0; hh < BN / HD; ++hh) {
           const int c_lo = hh * HD + 2 * lane, c_hi = c_lo + HD / 2;
@@ -455,7 +474,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = __floats2bfloat162_rn(hi.x, hi.y);
         }
       }
-      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[35 + (rl0 - warp) / (6 * RB) * 2] = globaltimer_ns();
+      if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[35 + (rl0 - warp) / (kWarps * RB) * 2] = globaltimer_ns();
     }
   }
   if (dbg && threadIdx.x == 64) p.debug[5] = globaltimer_ns();
@@ -491,7 +510,7 @@ static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pdl(kern, dim3(n_tiles, m_tiles, splits), dim3(192), SMEM_TOTAL, st, splits, a, b0, b1, p);
+  return launch_pdl(kern, dim3(n_tiles, m_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, splits, a, b0, b1, p);
 }
 
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
