@@ -73,13 +73,24 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 
 template <typename T, int MAXV>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, const float* __restrict__ gain,
-                                                      T* __restrict__ xn, int d, float eps) {
+                                                      T* __restrict__ xn, int d, float eps,
+                                                      unsigned long long* dbg) {
   constexpr int N = Vec16<T>::N;
   __shared__ float red[32];
+  if (dbg && threadIdx.x == 0) {
+    const unsigned long long t = ptx::globaltimer_ns();
+    if (blockIdx.x == 0) dbg[0] = t;
+    atomicMax(&dbg[4], t);                     // latest CTA start
+  }
   // x may be the output of the previous kernel in the stream (the previous layer of a model), so it is read only
   // after that kernel has completed.
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
+  if (dbg && threadIdx.x == 0) {
+    const unsigned long long t = ptx::globaltimer_ns();
+    if (blockIdx.x == 0) dbg[2] = t;
+    atomicMax(&dbg[3], t);                     // latest return from the wait
+  }
   const size_t row = blockIdx.x;
   const T* xr = x + row * d;
   T* yr = xn + row * d;
@@ -130,19 +141,22 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     for (int e = 0; e < N; ++e) t[e] = t[e] * r * gain[vi * N + e];
     Vec16<T>::store(yr + vi * N, t);
   }
+  if (dbg && threadIdx.x == 0) atomicMax(&dbg[5], ptx::globaltimer_ns());   // latest CTA end
 }
 
 template <typename T>
-void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st) {
+void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st,
+                    unsigned long long* dbg) {
   if (rows <= 0) return;
   int nvec = d / Vec16<T>::N;
   int threads = nvec >= 512 ? 256 : (nvec >= 128 ? 128 : ((nvec + 31) / 32) * 32);
   if (threads > 256) threads = 256;
-  launch_pdl(rmsnorm_kernel<T, 2>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps);
+  launch_pdl(rmsnorm_kernel<T, 2>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps, dbg);
 }
-template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t);
+template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t,
+                                    unsigned long long*);
 template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, __nv_bfloat16*, int, int, float,
-                                            cudaStream_t);
+                                            cudaStream_t, unsigned long long*);
 
 // ------------------------------------------------------------------------------------------------ selection
 // Eq. 2 and its complement: token t is refreshed iff !(s_t <= tau) (a NaN score refreshes).  The refresh set is

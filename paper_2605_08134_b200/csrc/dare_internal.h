@@ -61,7 +61,8 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 // ---- kernels common to both paths (common.cu) -------------------------------------------------------------
 void launch_rope_table(float* cs, int max_seq, int head_dim, double theta, cudaStream_t st);
 template <typename T>
-void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st);
+void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st,
+                    unsigned long long* dbg = nullptr);
 // Threshold + ballot/prefix-sum compaction + staleness update.  `scores == nullptr` or `select_all` selects all.
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
                    int* batch_off, int* delta, cudaStream_t st);

@@ -110,7 +110,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   prof_begin(L);
   // Alg. 1/2 line 1
   prof_mark(L, SLOT_NORM, st);
-  launch_rmsnorm<bf16>((const bf16*)x, L->w.rms_gain, (bf16*)B.xn, T_, d, L->cfg.rms_eps, st); ++launches;
+  launch_rmsnorm<bf16>((const bf16*)x, L->w.rms_gain, (bf16*)B.xn, T_, d, L->cfg.rms_eps, st, dbg ? dbg + 40 : nullptr);
+  ++launches;
   // line 2 + line 3 + stored-query update + rotary embedding, one kernel
   {
     GemmParams p = base;
