@@ -68,6 +68,13 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// max(a, b, c) in one instruction
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 256;
 // S of stream 0 / 1: columns [0, 128) / [128, 256), P over the first 64 of them; O: [256, 384) / [384, 512)
@@ -333,30 +340,36 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         for (int i = 0; i < 128; ++i)
           if (i >= n_keys) v[i] = -INFINITY;
       }
-      // row maximum (four independent chains)
-      float mx4[4] = {v[0], v[1], v[2], v[3]};
+      // row maximum: four independent chains of three-input maxima
+      float mx4[4];
 #pragma unroll
-      for (int i = 4; i < 128; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], v[i]);
-      settle_max(fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]))));
-      // exponentials against m (masked keys: 2^-inf = 0), row sum
-      const float mc = m * c;
+      for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(v[k], v[4 + k]);
 #pragma unroll
-      for (int i = 0; i < 128; ++i) {
-        v[i] = fast_exp2(fmaf(v[i], c, -mc));
-        sum4[i & 3] += v[i];
+      for (int i = 8; i < 128; i += 8) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mx4[k] = fmax3(mx4[k], v[i + k], v[i + 4 + k]);
       }
-      // P as bf16 over the first 64 columns of this row of S: column i = keys (2i, 2i+1)
-      {
-        float pk[64];
+      settle_max(fmax3(m, fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+      // exponentials against m (masked keys: 2^-inf = 0) and the row sum, the scaling and the sum two keys per
+      // instruction (packed fp32)
+      const float2 c2 = make_float2(c, c), nmc2 = make_float2(-m * c, -m * c);
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      // P as bf16 over the first 64 columns of this row of S: column i = keys (2i, 2i+1); packed as it is produced,
+      // so that the scores leave the register file pair by pair
+      float pk[64];
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-          pk[i] = __uint_as_float(*reinterpret_cast<uint32_t*>(&h2));
-        }
-        tmem_st_32x32_nowait(tmem_s + lane_addr, pk);
-        tmem_st_32x32_nowait(tmem_s + lane_addr + 32, pk + 32);
-        tmem_st_wait();
+      for (int i = 0; i < 128; i += 2) {
+        float2 e = __ffma2_rn(make_float2(v[i], v[i + 1]), c2, nmc2);
+        e.x = fast_exp2(e.x);
+        e.y = fast_exp2(e.y);
+        sum2[(i >> 1) & 1] = __fadd2_rn(sum2[(i >> 1) & 1], e);
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
+        pk[i >> 1] = __uint_as_float(*reinterpret_cast<uint32_t*>(&h2));
       }
+      sum4[0] = sum2[0].x; sum4[1] = sum2[0].y; sum4[2] = sum2[1].x; sum4[3] = sum2[1].y;
+      tmem_st_32x32_nowait(tmem_s + lane_addr, pk);
+      tmem_st_32x32_nowait(tmem_s + lane_addr + 32, pk + 32);
+      tmem_st_wait();
       l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       tc_fence_before();
       __syncwarp();
