@@ -152,7 +152,11 @@ dare_status_t dare_layer_last_selection(dare_layer_t* layer, int32_t* idx_host, 
 dare_status_t dare_layer_read_caches(dare_layer_t* layer, void* k_host, void* v_host, void* o_host,
                                      float* q_prev_host, void* cuda_stream);
 
-/* Checkpoint / resume of the reuse state (previous query, K/V/O caches, staleness, step bookkeeping). */
+/* Checkpoint / resume of the reuse state (previous query, K/V/O caches, staleness, step bookkeeping).
+ * The library's own cache of projected outputs (W_O O by cache row, which lets a step with many tokens that reuses
+ * attention outputs project only the refreshed rows: the paper's Alg. 2 line 11 projects every row, and a reused
+ * row projects to what it projected to before) is derived data and not part of the state: after an import the next
+ * steps project every row again until one of them has covered every cached row. */
 size_t dare_layer_state_bytes(const dare_layer_t* layer);
 dare_status_t dare_layer_export_state(dare_layer_t* layer, void* dst_host, size_t bytes, void* cuda_stream);
 dare_status_t dare_layer_import_state(dare_layer_t* layer, const void* src_host, size_t bytes, void* cuda_stream);

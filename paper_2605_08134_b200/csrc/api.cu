@@ -71,6 +71,7 @@ size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) 
   B.x_stage = take(Tm * d * e);
   B.y_stage = take(Tm * d * e);
   B.tmp = use_tc ? nullptr : (float*)take(Tm * 2 * d * sizeof(float));
+  B.yc = use_tc ? take(Tm * d * e) : nullptr;
   return off;
 }
 
@@ -230,6 +231,7 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->w = *w;
   L->use_tc = use_tc;
   L->has_prev = false;
+  L->yc_valid = false;
   L->batch = 0;
   L->kv_len = 0;
   L->last_launches = 0;
@@ -293,6 +295,7 @@ dare_status_t dare_layer_reset(dare_layer_t* L) {
   dare_status_t s = check_handle(L);
   if (s != DARE_OK) return s;
   L->has_prev = false;
+  L->yc_valid = false;
   L->batch = 0;
   L->kv_len = 0;
   return DARE_OK;
@@ -435,6 +438,8 @@ dare_status_t dare_layer_import_state(dare_layer_t* L, const void* src_host, siz
   }
   CUDA_TRY(cudaStreamSynchronize(st));
   L->has_prev = h.has_prev != 0;
+  L->yc_valid = false;                 // the projected-output cache is not part of the state: rebuilt by the next
+                                       // step that projects every cached row
   L->batch = h.batch;
   L->kv_len = h.kv_len;
   return DARE_OK;

@@ -218,6 +218,32 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
              count, batch_off, delta);
 }
 
+// ------------------------------------------------------------------------------------------------ reused rows
+// One warp per token row; rows refreshed in this step (staleness 0) are written by the projection itself.
+template <typename T>
+__global__ void __launch_bounds__(256) copy_reused_rows_kernel(const T* __restrict__ yc, T* __restrict__ y,
+                                                               const int* __restrict__ delta, StepGeom g) {
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= g.tokens()) return;
+  const int cr = g.cache_row(t);
+  if (delta[cr] == 0) return;
+  const uint4* s = reinterpret_cast<const uint4*>(yc + (size_t)cr * g.d);
+  uint4* o = reinterpret_cast<uint4*>(y + (size_t)t * g.d);
+  const int nvec = g.d * (int)sizeof(T) / 16;
+  for (int v = threadIdx.x & 31; v < nvec; v += 32) o[v] = s[v];
+}
+
+template <typename T>
+void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st) {
+  const int T_ = g.tokens();
+  if (T_ <= 0) return;
+  launch_pdl(copy_reused_rows_kernel<T>, dim3((T_ + 7) / 8), dim3(256), 0, st, 1, yc, y, delta, g);
+}
+template void launch_copy_reused_rows<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, const int*, const StepGeom&,
+                                                     cudaStream_t);
+
 // ------------------------------------------------------------------------------------------------ row gather
 // dst[r, :] = src[idx[r], :] for r < *count (Alg. 1 line 6: x_norm restricted to the refresh set).
 template <typename T>

@@ -64,6 +64,10 @@ template <typename T>
 void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st,
                     unsigned long long* dbg = nullptr);
 // Threshold + ballot/prefix-sum compaction + staleness update.  `scores == nullptr` or `select_all` selects all.
+// y[t] = yc[cache_row(t)] for the tokens of the step that were not refreshed (staleness counter != 0 after the
+// selection of the step): the rows a gathered output projection leaves out.
+template <typename T>
+void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st);
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
                    int* batch_off, int* delta, cudaStream_t st);
 template <typename T>

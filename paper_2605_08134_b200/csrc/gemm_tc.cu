@@ -284,7 +284,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       for (int k = 0; k < 8; ++k) {
         const int rw = k * 4 + (lane >> 3), r = quarter * 32 + rw, u = lane & 7;
         const int tok = __shfl_sync(0xffffffffu, tok_own, rw);
-        src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)(tok >= 0 ? tok : 0) * p.K * 2 +
+        const int srow = tok < 0 ? 0 : (p.gather_cache_rows ? p.g.cache_row(tok) : tok);
+        src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)srow * p.K * 2 +
                    (size_t)kb_begin * (BK * 2) + u * 16;
         bytes_k[k] = tok >= 0 ? 16u : 0u;                       // rows past the refresh set are zero-filled
         dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
@@ -470,8 +471,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const float2 rb2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(rs + c_hi));
             lo.x += ra.x; lo.y += ra.y; hi.x += rb2.x; hi.y += rb2.y;
           }
-          *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = __floats2bfloat162_rn(lo.x, lo.y);
-          *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = __floats2bfloat162_rn(hi.x, hi.y);
+          const __nv_bfloat162 o_lo = __floats2bfloat162_rn(lo.x, lo.y), o_hi = __floats2bfloat162_rn(hi.x, hi.y);
+          *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = o_lo;
+          *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = o_hi;
+          if (EPI == EPI_OUT && p.out1 != nullptr) {       // second copy, by cache row: the projected-output cache
+            __nv_bfloat16* dst2 = p.out1 + rb.crow[k] * p.ld_out + n0;
+            *reinterpret_cast<__nv_bfloat162*>(dst2 + c_lo) = o_lo;
+            *reinterpret_cast<__nv_bfloat162*>(dst2 + c_hi) = o_hi;
+          }
         }
       }
       if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[35 + (rl0 - warp) / (kWarps * RB) * 2] = globaltimer_ns();

@@ -23,6 +23,7 @@ struct Buffers {
   unsigned long long* debug;  // [64] kernel phase timestamps (diagnostics, written by block (0,0) when enabled)
   void* x_stage;    // [T, d] staging for the host-buffer entry point
   void* y_stage;
+  void* yc;         // tensor-core path: cache of projected outputs y = W_O O by cache row (gathered output projection)
   float* tmp;       // SIMT path: fp32 projection results [T, 2d]
 };
 
@@ -44,6 +45,7 @@ struct dare_layer {
   size_t workspace_bytes;
   bool use_tc;
   bool has_prev;
+  bool yc_valid;    // the projected-output cache holds the current W_O O of every cached row
   int batch;
   int kv_len;
   int last_launches;

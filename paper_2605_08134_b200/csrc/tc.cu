@@ -98,7 +98,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   GemmParams base;
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
-  base.gather_src = nullptr;
+  base.gather_src = nullptr; base.gather_cache_rows = 0;
   base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
   base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
@@ -167,18 +167,39 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
-  // output projection of every row of the window, read from the O cache
+  // Output projection, read from the O cache.  Alg. 2 line 11 projects every row of the window.  A row whose
+  // attention output was reused projects to what it projected to before (W_O acts row by row), so with many tokens
+  // the library keeps those projections by cache row and, on a step that reuses attention outputs, projects the
+  // refresh set's rows only (fetched from the O cache by index, like the rows of the gathered K/V projection) and
+  // copies the others.  With few tokens the projection is a stream of W_O whatever the row count, and stays dense.
   {
+    const bool many = m_tiles_dense > 8 && !add_input;
+    const bool y_sparse = o_sparse && many && L->yc_valid;
     GemmParams p = base;
     p.a_seq_stride = g.max_seq; p.a_row0 = g.pos_begin;
     p.out0 = (bf16*)y;
+    if (many) p.out1 = (bf16*)B.yc;                                   // kept by cache row for later steps
     if (add_input) { p.resid = (const bf16*)x; p.ld_resid = d; }      // y = x + W_O O (residual block)
     p.debug = dbg ? dbg + 24 : nullptr;
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_OUT_GEMM, st);
-    e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense,
-                       pick_splits(n_tiles * m_tiles_dense, kblocks), st); ++launches;
-    if (e != cudaSuccess) return DARE_ERR_CUDA;
+    if (y_sparse) {
+      p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.oc; p.gather_cache_rows = 1;
+      e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, 1, st); ++launches;
+      if (e != cudaSuccess) return DARE_ERR_CUDA;
+      launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
+    } else {
+      e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense,
+                         pick_splits(n_tiles * m_tiles_dense, kblocks), st); ++launches;
+      if (e != cudaSuccess) return DARE_ERR_CUDA;
+      // the cache is complete once a dense projection has covered every cached row, and stays so while every
+      // later step maintains it
+      if (many) {
+        if (g.pos_begin == 0 && g.seq_act == g.kv_len) L->yc_valid = true;
+      } else {
+        L->yc_valid = false;
+      }
+    }
   }
   prof_end(L, st);
   L->last_launches = launches;

@@ -172,3 +172,36 @@ def test_peaked_softmax_rescales_the_accumulator(dare):
     np.testing.assert_array_equal(a.last_selection(1, shape.seq)["idx"], o.last_idx)
     np.testing.assert_array_equal(a.last_selection(1, shape.seq)["idx"], b.last_selection(1, shape.seq)["idx"])
     a.close(); b.close()
+
+
+def test_gathered_output_projection_windows_and_state(dare):
+    """Many tokens per step (more than eight row tiles): on steps that reuse attention outputs the output projection
+    runs over the refresh set only and the other rows come from the cache of projected rows.  Checked against the
+    oracle over full-extent and window steps in every mode, and across an export/import of the layer state (which
+    does not carry that cache: the next step projects every row again)."""
+    import torch
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=2, seq=1280, prompt=256)
+    w = wl.make_weights(shape, 31)
+    hs = wl.HiddenStream(shape, 31)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    parity.compare_step(g, o, hs.advance(wl.uniform_positions(hs.rng, shape, 200)), 3, 0.1, shape)
+    p = shape.prompt
+    for mode in (2, 1, 3):            # window of 1024 positions x 2 sequences = 16 row tiles
+        x = hs.advance(wl.uniform_positions(hs.rng, shape, 120))
+        parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), mode, 0.1, shape, pos_begin=p)
+    # state to a second handle: same results from there on
+    n = dare.dare_layer_state_bytes(g.handle)
+    blob = torch.empty(n, dtype=torch.uint8).pin_memory()
+    assert dare.dare_layer_export_state(g.handle, blob.data_ptr(), n) == 0
+    g2 = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    assert dare.dare_layer_import_state(g2.handle, blob.data_ptr(), n) == 0
+    for mode in (2, 3):
+        x = hs.advance(wl.uniform_positions(hs.rng, shape, 90))
+        xw = np.ascontiguousarray(x[:, p:])
+        y2 = g2.step(parity.to_device(xw, shape), mode, 0.1, pos_begin=p)
+        _, yo = parity.compare_step(g, o, xw, mode, 0.1, shape, pos_begin=p)
+        np.testing.assert_array_equal(g2.last_selection(2, shape.seq - p)["idx"], o.last_idx)
+        parity.assert_close("imported handle y", y2.float().cpu().numpy(), yo, 2e-2)
+    g.close(); g2.close()
