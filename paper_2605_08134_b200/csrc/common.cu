@@ -160,10 +160,82 @@ template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, 
 
 // ------------------------------------------------------------------------------------------------ selection
 // Eq. 2 and its complement: token t is refreshed iff !(s_t <= tau) (a NaN score refreshes).  The refresh set is
-// written as an ascending index list by warp ballot + popcount + a block prefix sum over warp totals; the
-// staleness counters of Sec. 4 are updated in the same pass.  A CTA walks the tokens in chunks of 1024, which
-// keeps the list ordered without any inter-CTA hand-off (T <= a few 10^4 per layer step).
+// written as an ascending index list: every thread takes four consecutive tokens of a chunk of 4096, a warp scan
+// and a scan over the warp totals give each thread its place; the staleness counters of Sec. 4 and the start of
+// every sequence's slice of the list come out of the same pass.  One CTA walks the chunks, which keeps the list
+// ordered without any inter-CTA hand-off (T <= a few 10^4 per layer step).
+constexpr int kSelPerThread = 4;
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
+                                                      StepGeom g, int* __restrict__ idx, int* __restrict__ count,
+                                                      int* __restrict__ batch_off, int* __restrict__ delta) {
+  __shared__ int warp_tot[32];
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
+  const int T = g.tokens();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int base = 0;
+  for (int start = 0; start < T; start += 1024 * kSelPerThread) {
+    const int t0 = start + threadIdx.x * kSelPerThread;
+    // all loads of the chunk first (scores and staleness counters): one memory round trip
+    float sc[kSelPerThread];
+    int cr[kSelPerThread], stale[kSelPerThread];
+#pragma unroll
+    for (int k = 0; k < kSelPerThread; ++k) {
+      const int t = t0 + k;
+      sc[k] = 0.f; cr[k] = 0; stale[k] = 0;
+      if (t < T) {
+        cr[k] = g.cache_row(t);
+        if (!select_all) sc[k] = scores[t];
+        stale[k] = delta[cr[k]];
+      }
+    }
+    bool sel[kSelPerThread];
+    int mine = 0;
+#pragma unroll
+    for (int k = 0; k < kSelPerThread; ++k) {
+      sel[k] = t0 + k < T && (select_all ? true : !(sc[k] <= tau));
+      mine += sel[k] ? 1 : 0;
+    }
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    // (32 warp totals: every thread sums the ones before its warp; lane w of a warp holds total w)
+    const int wt = warp_tot[lane];
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 32; ++w) {
+      const int v = __shfl_sync(0xffffffffu, wt, w);
+      before += w < warp ? v : 0;
+      total += v;
+    }
+    int out = base + before + inc - mine;
+#pragma unroll
+    for (int k = 0; k < kSelPerThread; ++k) {
+      const int t = t0 + k;
+      if (t < T) {
+        // a sequence starts at this token: its slice of the ascending list starts at the current place
+        if (t % g.seq_act == 0) batch_off[t / g.seq_act] = out;
+        if (sel[k]) idx[out++] = t;
+        delta[cr[k]] = sel[k] ? 0 : stale[k] + 1;
+      }
+    }
+    base += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    *count = base;
+    batch_off[g.batch] = base;
+  }
+}
+
+// The same for short steps: one token per thread and chunk of 1024, warp ballot + popcount (less index arithmetic
+// per token, which is what a step of a few hundred tokens pays for).
+__global__ void __launch_bounds__(1024) select_small_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
                                                       int* __restrict__ batch_off, int* __restrict__ delta) {
   __shared__ int warp_excl[32];
@@ -214,8 +286,11 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
 
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
                    int* batch_off, int* delta, cudaStream_t st) {
-  launch_pdl(select_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, (select_all || scores == nullptr) ? 1 : 0, g, idx,
-             count, batch_off, delta);
+  const int all = (select_all || scores == nullptr) ? 1 : 0;
+  if (g.tokens() <= 2048)
+    launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta);
+  else
+    launch_pdl(select_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta);
 }
 
 // ------------------------------------------------------------------------------------------------ reused rows
