@@ -79,6 +79,12 @@ constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 256;
 // S of stream 0 / 1: columns [0, 128) / [128, 256), P over the first 64 of them; O: [256, 384) / [384, 512)
 constexpr uint32_t kTmemCols = 512;
+#ifndef DARE_ATTN_PAIR_MIN_DENSE
+#define DARE_ATTN_PAIR_MIN_DENSE 128      // dense launches with longer windows take the two-tile kernel
+#endif
+#ifndef DARE_ATTN_PAIR_MIN_SPARSE
+#define DARE_ATTN_PAIR_MIN_SPARSE 1024    // row-sparse launches from this window length on
+#endif
 constexpr float kRescaleStep = 8.f;     // log2 of the growth of the running maximum that triggers a rescale of O
 
 }  // namespace
@@ -511,11 +517,318 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+// ------------------------------------------------------------------------------------------------ two query tiles
+// The variant for launches with many query rows per (sequence, head): one CTA = one head x up to 256 query rows, i.e.
+// two 128-row tiles, each with its own softmax warps, issuer warp, S/P and O regions of tensor memory - the two
+// streams of the kernel above - but now the streams walk the same key blocks and share them: every K and V block is
+// brought into shared memory once for both tiles, which halves what a CTA pulls from the L2 per flop (that traffic,
+// 64 KB per key block and tile, is what the kernel above runs into when every SM does it at once).  No merge at the
+// end: a stream owns its rows.
+namespace {
+struct PairSmem {
+  static constexpr int Q_BYTES = BQ * HD * 2;
+  static constexpr int KV_BYTES = BKV * HD * 2;
+  static constexpr int Q_OFF = 0;                        // two tiles
+  static constexpr int K_OFF = Q_OFF + 2 * Q_BYTES;      // ring of 2
+  static constexpr int V_OFF = K_OFF + 2 * KV_BYTES;     // ring of 2
+  static constexpr int BAR_OFF = V_OFF + 2 * KV_BYTES;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;
+};
+static_assert(PairSmem::TOTAL <= 232448, "shared memory");
+constexpr int kPairRows = 2 * BQ;
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                 const AttnParams p) {
+  using S = PairSmem;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::BAR_OFF);
+  uint64_t* k_full = bars;          // [2 ring slots]
+  uint64_t* k_empty = bars + 2;     // [2]: one arrival per stream
+  uint64_t* v_full = bars + 4;      // [2]
+  uint64_t* v_empty = bars + 6;     // [2]: one arrival per stream
+  uint64_t* s_full = bars + 8;      // [2 streams]
+  uint64_t* p_full = bars + 10;     // [2 streams]
+  uint64_t* o_full = bars + 12;     // [2 streams]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+  const StepGeom& g = p.g;
+  // CTA -> (head, sequence, 256-row tile): same launch orders as the kernel above
+  const int tps = (g.seq_act + kPairRows - 1) / kPairRows;
+  int h, b, tile;
+  {
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+    if (p.idx != nullptr) {
+      h = lin % g.n_heads;
+      const int rest = lin / g.n_heads;
+      tile = rest / g.batch;
+      b = rest - tile * g.batch;
+    } else {
+      tile = lin % tps;
+      const int rest = lin / tps;
+      h = rest % g.n_heads;
+      b = rest / g.n_heads;
+    }
+  }
+  if (p.idx != nullptr && tile > 0) {
+    pdl_wait();
+    if (p.batch_off[b] + tile * kPairRows >= p.batch_off[b + 1]) return;
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&k_empty[i], 2); mbar_init(&v_empty[i], 2);
+      mbar_init(&s_full[i], 1); mbar_init(&o_full[i], 1);
+      mbar_init(&p_full[i], kSoftmaxThreads / 64);
+    }
+    fence_mbar_init();
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
+  if (warp == 2) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  pdl_wait();
+  pdl_launch_dependents();
+  // ---- rows of the two tiles (uniform over the CTA)
+  int row0 = 0, rows_all = 0;
+  bool active = true;
+  if (p.idx != nullptr) {
+    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
+    row0 = lo + tile * kPairRows;
+    active = row0 < hi;
+    rows_all = min(kPairRows, hi - row0);
+  } else {
+    row0 = b * g.seq_act + tile * kPairRows;
+    rows_all = min(kPairRows, g.seq_act - tile * kPairRows);
+  }
+  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  const int kv_row0 = b * g.max_seq;
+  auto load_kv = [&](int i) {        // one thread: key block i into ring slot i & 1
+    const int slot = i & 1, row = kv_row0 + i * BKV;
+    uint8_t* kd = smem + S::K_OFF + slot * S::KV_BYTES;
+    uint8_t* vd = smem + S::V_OFF + slot * S::KV_BYTES;
+    mbar_arrive_expect_tx(&k_full[slot], S::KV_BYTES);
+    tma_load_2d(kd, &tm_k, h * HD, row, &k_full[slot]);
+    tma_load_2d(kd + S::KV_BYTES / 2, &tm_k, h * HD + 64, row, &k_full[slot]);
+    mbar_arrive_expect_tx(&v_full[slot], S::KV_BYTES);
+    tma_load_2d(vd, &tm_v, h * HD, row, &v_full[slot]);
+    tma_load_2d(vd + S::KV_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[slot]);
+  };
+  // the first two key blocks start now, by the thread that initialised the barriers: in flight during the Q gather
+  if (threadIdx.x == 0 && active) {
+    for (int i = 0; i < 2 && i < n_blocks; ++i) load_kv(i);
+  }
+  // ---- both Q tiles: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
+  if (active) {
+    constexpr int QU = (kPairRows * 16 + kThreads - 1) / kThreads;
+    int tok[QU];
+    uint4 qv[QU];
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int u = threadIdx.x + k * kThreads, r = u >> 4;
+      tok[k] = -1;
+      if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
+    }
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int unit = (threadIdx.x + k * kThreads) & 15;
+      qv[k] = make_uint4(0u, 0u, 0u, 0u);
+      if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
+    }
+#pragma unroll
+    for (int k = 0; k < QU; ++k) {
+      const int u = threadIdx.x + k * kThreads, r = u >> 4, unit = u & 15;
+      const int chunk = unit >> 3, uc = unit & 7, rt = r & (BQ - 1);
+      uint8_t* qs = smem + S::Q_OFF + (r >> 7) * S::Q_BYTES;
+      if (u < kPairRows * 16) *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + rt * 128 + ((uc ^ (rt & 7)) << 4)) = qv[k];
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (active) {
+  // stream = query tile: warps 2/3 issue for tile 0/1, softmax warps 4-7 / 8-11; warp 0 brings the key blocks
+  const int st = warp < 4 ? (warp & 1) : ((warp - 4) >> 2);
+  const int rows_valid = max(0, min(BQ, rows_all - st * BQ));       // rows of this stream's tile
+  const bool st_active = rows_valid > 0;                             // the second tile of a short tail is empty
+  const uint32_t tmem_s = tmem_base + st * BKV, tmem_o = tmem_base + 2 * BKV + st * HD;
+  if (warp == 0) {
+    for (int i = 2; i < n_blocks; ++i) {
+      const int slot = i & 1;
+      // both streams have finished with block i - 2: their score products ...
+      mbar_wait(&k_empty[slot], ((i >> 1) & 1) ^ 1, p.status);
+      // ... and their P V products
+      mbar_wait(&v_empty[slot], ((i >> 1) & 1) ^ 1, p.status);
+      if (elect_one()) load_kv(i);
+      __syncwarp();
+    }
+  } else if (warp == 2 || warp == 3) {
+    constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
+    constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
+    const uint64_t q_desc = smem_desc_k_sw128(smem_u32(smem + S::Q_OFF + st * S::Q_BYTES));
+    const uint64_t k_desc0 = smem_desc_k_sw128(smem_u32(smem + S::K_OFF));
+    const uint64_t v_desc0 = smem_desc_mn_sw128(smem_u32(smem + S::V_OFF), BKV * 128);
+    if (!st_active) {
+      // an empty tile still releases the ring slots it shares: one arrival per block and barrier, never ahead of
+      // the block's data
+      for (int i = 0; i < n_blocks; ++i) {
+        const int slot = i & 1;
+        mbar_wait(&k_full[slot], (i >> 1) & 1, p.status);
+        if (elect_one()) mbar_arrive(&k_empty[slot]);
+        __syncwarp();
+        mbar_wait(&v_full[slot], (i >> 1) & 1, p.status);
+        if (elect_one()) mbar_arrive(&v_empty[slot]);
+        __syncwarp();
+      }
+    } else {
+      auto issue_qk = [&](int i) {
+        const int slot = i & 1;
+        mbar_wait(&k_full[slot], (i >> 1) & 1, p.status);
+        tc_fence_after();
+        if (elect_one()) {
+          const uint64_t k_desc = k_desc0 + (uint64_t)(slot * (S::KV_BYTES >> 4));
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk)
+            umma_ss(tmem_s, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
+                    k_desc + (((kk >> 2) * (BKV * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk != 0 ? 1u : 0u);
+          umma_commit(&s_full[st]);
+          umma_commit(&k_empty[slot]);
+        }
+        __syncwarp();
+      };
+      if (n_blocks > 0) issue_qk(0);
+      for (int i = 0; i < n_blocks; ++i) {
+        const int slot = i & 1;
+        mbar_wait(&p_full[st], i & 1, p.status);      // P(i) has replaced S(i) in tensor memory
+        mbar_wait(&v_full[slot], (i >> 1) & 1, p.status);
+        tc_fence_after();
+        if (elect_one()) {
+          const uint64_t v_desc = v_desc0 + (uint64_t)(slot * (S::KV_BYTES >> 4));
+#pragma unroll
+          for (int ks = 0; ks < BKV / 16; ++ks)
+            umma_ts(tmem_o, tmem_s + ks * 8, v_desc + ((ks * (16 * 128)) >> 4), idesc_pv, (i | ks) != 0 ? 1u : 0u);
+          umma_commit(&o_full[st]);
+          umma_commit(&v_empty[slot]);
+        }
+        __syncwarp();
+        if (i + 1 < n_blocks) issue_qk(i + 1);        // in issue order behind the product that reads P(i)
+      }
+    }
+  } else if (warp >= 4 && st_active) {
+    // ---- softmax of this tile: thread <-> query row (as in the kernel above, over every key block)
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float c = rsqrtf((float)HD) * 1.4426950408889634f;
+    float m = -INFINITY, l = 0.f;
+    for (int j = 0; j < n_blocks; ++j) {
+      mbar_wait(&s_full[st], j & 1, p.status);
+      tc_fence_after();
+      const int n_keys = min(BKV, g.kv_len - j * BKV);
+      float v[128];
+      tmem_ld_32x32_nowait(tmem_s + lane_addr, v);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 32, v + 32);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 64, v + 64);
+      tmem_ld_32x32_nowait(tmem_s + lane_addr + 96, v + 96);
+      tmem_ld_wait();
+      if (n_keys < BKV) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i >= n_keys) v[i] = -INFINITY;
+      }
+      float mx4[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(v[k], v[4 + k]);
+#pragma unroll
+      for (int i = 8; i < 128; i += 8) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mx4[k] = fmax3(mx4[k], v[i + k], v[i + 4 + k]);
+      }
+      const float m_new = fmax3(m, fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (j == 0) {
+        m = m_new;
+      } else {
+        const bool grow = (m_new - m) * c > kRescaleStep;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? fast_exp2((m - m_new) * c) : 1.f;
+          if (grow) { m = m_new; l *= alpha; }
+          mbar_wait(&o_full[st], (j - 1) & 1, p.status);
+          tc_fence_after();
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            float o[32];
+            tmem_ld_32x32(tmem_o + lane_addr + ch * 32, o);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+            tmem_st_32x32(tmem_o + lane_addr + ch * 32, o);
+          }
+        }
+      }
+      const float2 c2 = make_float2(c, c), nmc2 = make_float2(-m * c, -m * c);
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      float pk[64];
+#pragma unroll
+      for (int i = 0; i < 128; i += 2) {
+        float2 e = __ffma2_rn(make_float2(v[i], v[i + 1]), c2, nmc2);
+        e.x = fast_exp2(e.x);
+        e.y = fast_exp2(e.y);
+        sum2[(i >> 1) & 1] = __fadd2_rn(sum2[(i >> 1) & 1], e);
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
+        pk[i >> 1] = __uint_as_float(*reinterpret_cast<uint32_t*>(&h2));
+      }
+      tmem_st_32x32_nowait(tmem_s + lane_addr, pk);
+      tmem_st_32x32_nowait(tmem_s + lane_addr + 32, pk + 32);
+      tmem_st_wait();
+      l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[st]);
+    }
+    if (n_blocks > 0) {
+      mbar_wait(&o_full[st], (n_blocks - 1) & 1, p.status);
+      tc_fence_after();
+    }
+    // ---- normalise and store this row (the tensor-memory loads are warp-wide; rows past the tile's end only skip
+    // the store)
+    {
+      const bool ok = r < rows_valid;
+      const float inv = 1.f / l;
+      const int rr = st * BQ + (ok ? r : 0);
+      const int t = p.idx ? p.idx[row0 + rr] : row0 + rr;
+      __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        float o[32];
+        tmem_ld_32x32(tmem_o + lane_addr + ch * 32, o);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] *= inv;
+        if (ok) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) reinterpret_cast<uint4*>(dst + ch * 32)[v4] = pack8_bf16(o + 8 * v4);
+        }
+      }
+    }
+  }
+  }  // active
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
+}
+
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem::TOTAL);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::TOTAL);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -527,6 +840,18 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
   // the keys are split only when every CTA still keeps at least four blocks.
   int ksplit = 1;
   while (ksplit < 4 && expected * ksplit * 2 <= 160 && ksplit * 2 * 4 <= n_blocks) ksplit *= 2;
+  // Many query rows per sequence (and enough work to fill the GPU without a key split): two tiles per CTA share
+  // the key blocks.  A row-sparse launch cannot know the size of the refresh set; the window length decides: long
+  // windows are where refresh sets of several tiles are.
+  const int tps2 = (p.g.seq_act + kPairRows - 1) / kPairRows;
+  const bool pair = ksplit == 1 &&
+                    (p.idx ? p.g.seq_act >= DARE_ATTN_PAIR_MIN_SPARSE && p.g.n_heads * p.g.batch >= 64
+                           : p.g.seq_act > DARE_ATTN_PAIR_MIN_DENSE && p.g.n_heads * p.g.batch * tps2 >= 148);
+  if (pair) {
+    dim3 grid(p.g.n_heads, p.g.batch * tps2, 1);
+    if (grid.y == 0) return cudaSuccess;
+    return launch_pdl(attn_pair_kernel, grid, dim3(kThreads), PairSmem::TOTAL, st, 1, tm_k, tm_v, p);
+  }
   dim3 grid(p.g.n_heads, p.g.batch * tps, ksplit);
   if (grid.y == 0) return cudaSuccess;
   return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), AttnSmem::TOTAL, st, ksplit, tm_k, tm_v, p);

@@ -205,3 +205,21 @@ def test_gathered_output_projection_windows_and_state(dare):
         np.testing.assert_array_equal(g2.last_selection(2, shape.seq - p)["idx"], o.last_idx)
         parity.assert_close("imported handle y", y2.float().cpu().numpy(), yo, 2e-2)
     g.close(); g2.close()
+
+
+def test_two_tile_attention_ragged(dare):
+    """Sizes that send dense and row-sparse attention to the kernel with two query tiles per CTA (many rows per
+    sequence and enough (head, sequence) pairs to fill the GPU), with everything ragged: 1100 keys (8 blocks + 76),
+    windows whose last 256-row tile holds 76 rows (its second tile empty), refresh sets that end inside a tile."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=1024, n_heads=8, batch=8, seq=1100, prompt=76)
+    w = wl.make_weights(shape, 52)
+    hs = wl.HiddenStream(shape, 52)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    parity.compare_step(g, o, hs.advance(wl.uniform_positions(hs.rng, shape, 300)), 3, 0.1, shape)
+    p = shape.prompt
+    for mode, n in ((2, 150), (0, 10)):   # window of 1024 positions: row-sparse, then dense
+        x = hs.advance(wl.uniform_positions(hs.rng, shape, n))
+        parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), mode, 0.1, shape, pos_begin=p)
+    g.close()
