@@ -191,6 +191,10 @@ def test_gathered_output_projection_windows_and_state(dare):
     for mode in (2, 1, 3):            # window of 1024 positions x 2 sequences = 16 row tiles
         x = hs.advance(wl.uniform_positions(hs.rng, shape, 120))
         parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), mode, 0.1, shape, pos_begin=p)
+    # nothing refreshed (every row copied from the cache of projected rows), then everything refreshed
+    for tau in (float("inf"), -1.0):
+        x = hs.advance(wl.uniform_positions(hs.rng, shape, 60))
+        parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), 3, tau, shape, pos_begin=p)
     # state to a second handle: same results from there on
     n = dare.dare_layer_state_bytes(g.handle)
     blob = torch.empty(n, dtype=torch.uint8).pin_memory()
