@@ -227,3 +227,33 @@ def test_two_tile_attention_ragged(dare):
         x = hs.advance(wl.uniform_positions(hs.rng, shape, n))
         parity.compare_step(g, o, np.ascontiguousarray(x[:, p:]), mode, 0.1, shape, pos_begin=p)
     g.close()
+
+
+@pytest.mark.parametrize("geom", ["llada_layer", "many_tokens"])
+def test_tensor_path_is_deterministic(dare, geom):
+    """Two handles, same weights, same steps: bit-identical outputs and caches (fixed reduction orders in the split-K
+    exchange, the stream merge and the key split; no result depends on scheduling)."""
+    import torch
+    if geom == "llada_layer":
+        shape = wl.LLADA_LAYER
+        changed, modes = 67, (3, 3, 2, 1, 0)
+    else:
+        shape = wl.scaled(wl.LLADA_LAYER, d_model=1024, n_heads=8, batch=8, seq=1280, prompt=256)
+        changed, modes = 200, (3, 2, 3, 1, 0)
+    w = wl.make_weights(shape, 77)
+    hs = wl.HiddenStream(shape, 77)
+    xs = [hs.first()] + [hs.advance(wl.uniform_positions(hs.rng, shape, changed)) for _ in modes]
+    outs = []
+    for rep in range(2):
+        g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+        ys = [g.step(parity.to_device(xs[0], shape), 3, 0.1).clone()]
+        for x, mode in zip(xs[1:], modes):
+            ys.append(g.step(parity.to_device(x, shape), mode, 0.1).clone())
+        torch.cuda.synchronize()
+        c = g.read_caches(shape.batch, shape.seq)
+        outs.append((ys, c))
+        g.close()
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    for k in ("k", "v", "o", "q_prev"):
+        np.testing.assert_array_equal(outs[0][1][k], outs[1][1][k])
