@@ -484,6 +484,11 @@ dare_status_t dare_layer_debug_timestamps(dare_layer_t* L, int enable, uint64_t*
     CUDA_TRY(cudaMemcpyAsync(out_host, L->buf.debug, (64 + 3 * 1024) * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
   }
+  if (enable && !L->debug_on) {
+    // cleared once, when the stamps are switched on (not per step: a memset in the stream would break the kernels'
+    // launch overlap); the stamps are plain stores or maxima of a clock that only grows
+    CUDA_TRY(cudaMemsetAsync(L->buf.debug, 0, (64 + 3 * 1024) * sizeof(uint64_t), st));
+  }
   L->debug_on = enable != 0;
   return DARE_OK;
 }

@@ -82,6 +82,20 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     if (blockIdx.x == 0) dbg[0] = t;
     atomicMax(&dbg[4], t);                     // latest CTA start
   }
+  // The gain is a weight: it does not depend on the previous kernel in the stream and is read while that one drains.
+  const int nvec0 = d / N;
+  float gn[MAXV][N];
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec0) {
+#pragma unroll
+      for (int e = 0; e < N; e += 4) {
+        const float4 t = *reinterpret_cast<const float4*>(gain + vi * N + e);
+        gn[i][e] = t.x; gn[i][e + 1] = t.y; gn[i][e + 2] = t.z; gn[i][e + 3] = t.w;
+      }
+    }
+  }
   // x may be the output of the previous kernel in the stream (the previous layer of a model), so it is read only
   // after that kernel has completed.
   ptx::pdl_wait();
@@ -118,19 +132,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
   for (int i = 0; i < MAXV; ++i) {
     int vi = threadIdx.x + i * blockDim.x;
     if (vi < nvec) {
-      float g[N];
-      if (N == 4) {
-        float4 t = *reinterpret_cast<const float4*>(gain + vi * N);
-        g[0] = t.x; g[1] = t.y; g[2] = t.z; g[3] = t.w;
-      } else {
 #pragma unroll
-        for (int e = 0; e < N; e += 4) {
-          float4 t = *reinterpret_cast<const float4*>(gain + vi * N + e);
-          g[e] = t.x; g[e + 1] = t.y; g[e + 2] = t.z; g[e + 3] = t.w;
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < N; ++e) v[i][e] = v[i][e] * r * g[e];
+      for (int e = 0; e < N; ++e) v[i][e] = v[i][e] * r * gn[i][e];
       Vec16<T>::store(yr + vi * N, v[i]);
     }
   }

@@ -105,7 +105,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
   base.debug = nullptr;
   unsigned long long* dbg = L->debug_on ? B.debug : nullptr;
-  if (dbg) cudaMemsetAsync(dbg, 0, (64 + 3 * 1024) * sizeof(unsigned long long), st);
+  // (no clearing between steps: a copy or memset in the stream would break the kernels' launch overlap; the stamps
+  // are plain stores or maxima of a clock that only grows)
 
   prof_begin(L);
   // Alg. 1/2 line 1
