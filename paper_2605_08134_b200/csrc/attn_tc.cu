@@ -163,9 +163,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
-  // The set-up above overlapped the tail of the previous kernel in the stream; its results are needed from here on.
-  pdl_wait();
-  pdl_launch_dependents();
+  // The previous kernel in the stream (the K/V projection) writes the K and V caches only.  The queries and the
+  // refresh set come from kernels further back, which are complete by the time any CTA of this grid runs (every
+  // kernel lets its successor start only after its own wait): they are read without waiting, so that the gather
+  // of the Q tile overlaps the projection's tail.  Warp 0 waits right away and starts the first K and V blocks.
   // ---- rows of this tile (uniform over the CTA)
   int row0 = 0, rows_valid = 0;
   bool active = true;
@@ -181,8 +182,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int n_blocks_all = (g.kv_len + BKV - 1) / BKV;
   const int n_blocks = n_blocks_all > z ? (n_blocks_all - z + ksplit - 1) / ksplit : 0;   // blocks z, z + ksplit, ...
   const int kv_row0 = b * g.max_seq;
-  // The first K and V block of each stream start now, by the thread that initialised the barriers, so that they are
-  // in flight while the Q tile is gathered.
+  // The first K and V block of each stream start as soon as the projection is complete, by the thread that
+  // initialised the barriers, so that they are in flight while the Q tile is gathered.
+  if (warp == 0) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   if (threadIdx.x == 0 && active) {
     for (int s2 = 0; s2 < 2 && s2 < n_blocks; ++s2) {
       const int row = kv_row0 + (z + s2 * ksplit) * BKV;
@@ -196,32 +201,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       tma_load_2d(vd + S::V_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[2 * s2]);
     }
   }
-  // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
-  if (active) {
+  // ---- Q tile: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units), by the
+  // warps other than warp 0
+  if (active && warp != 0) {
     uint8_t* qs = smem + S::Q_OFF;
-    constexpr int QU = (BQ * 16 + kThreads - 1) / kThreads;   // 16-byte units per thread
+    constexpr int kGather = kThreads - 32;
+    constexpr int QU = (BQ * 16 + kGather - 1) / kGather;     // 16-byte units per thread
+    const int u0 = (int)threadIdx.x - 32;
     int tok[QU];
     uint4 qv[QU];
     // all index loads first, then all row loads, then the stores: one memory round trip each instead of one per unit
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int u = threadIdx.x + k * kThreads, r = u >> 4;    // 16 units of 8 bf16 per row
+      const int u = u0 + k * kGather, r = u >> 4;              // 16 units of 8 bf16 per row
       tok[k] = -1;
       if (u < BQ * 16 && r < rows_valid) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int unit = (threadIdx.x + k * kThreads) & 15;
+      const int unit = (u0 + k * kGather) & 15;
       qv[k] = make_uint4(0u, 0u, 0u, 0u);
       if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int u = threadIdx.x + k * kThreads, r = u >> 4, unit = u & 15;
+      const int u = u0 + k * kGather, r = u >> 4, unit = u & 15;
       const int chunk = unit >> 3, uc = unit & 7;
       if (u < BQ * 16) *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + r * 128 + ((uc ^ (r & 7)) << 4)) = qv[k];
     }
     fence_proxy_async_smem();
+  }
+  if (warp != 0) {
+    pdl_wait();                       // every thread waits before it can touch what the projection wrote, or leave
+    pdl_launch_dependents();
   }
   tc_fence_before();
   __syncthreads();
@@ -591,8 +603,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     tmem_alloc(tmem_slot, kTmemCols);
     tmem_relinquish();
   }
-  pdl_wait();
-  pdl_launch_dependents();
+  // (as in the kernel above: queries and refresh set are read without waiting for the K/V projection; warp 0 waits
+  // right away and starts the first key blocks, the other warps gather the Q tiles first)
   // ---- rows of the two tiles (uniform over the CTA)
   int row0 = 0, rows_all = 0;
   bool active = true;
@@ -618,35 +630,46 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     tma_load_2d(vd, &tm_v, h * HD, row, &v_full[slot]);
     tma_load_2d(vd + S::KV_BYTES / 2, &tm_v, h * HD + 64, row, &v_full[slot]);
   };
-  // the first two key blocks start now, by the thread that initialised the barriers: in flight during the Q gather
+  // the first two key blocks start as soon as the projection is complete, by the thread that initialised the
+  // barriers: in flight during the Q gather
+  if (warp == 0) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   if (threadIdx.x == 0 && active) {
     for (int i = 0; i < 2 && i < n_blocks; ++i) load_kv(i);
   }
   // ---- both Q tiles: gathered rows -> shared memory in the K-major 128-byte-swizzled layout (16-byte units)
-  if (active) {
-    constexpr int QU = (kPairRows * 16 + kThreads - 1) / kThreads;
+  if (active && warp != 0) {
+    constexpr int kGather = kThreads - 32;
+    constexpr int QU = (kPairRows * 16 + kGather - 1) / kGather;
+    const int u0 = (int)threadIdx.x - 32;
     int tok[QU];
     uint4 qv[QU];
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int u = threadIdx.x + k * kThreads, r = u >> 4;
+      const int u = u0 + k * kGather, r = u >> 4;
       tok[k] = -1;
       if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int unit = (threadIdx.x + k * kThreads) & 15;
+      const int unit = (u0 + k * kGather) & 15;
       qv[k] = make_uint4(0u, 0u, 0u, 0u);
       if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
-      const int u = threadIdx.x + k * kThreads, r = u >> 4, unit = u & 15;
+      const int u = u0 + k * kGather, r = u >> 4, unit = u & 15;
       const int chunk = unit >> 3, uc = unit & 7, rt = r & (BQ - 1);
       uint8_t* qs = smem + S::Q_OFF + (r >> 7) * S::Q_BYTES;
       if (u < kPairRows * 16) *reinterpret_cast<uint4*>(qs + chunk * (BQ * 128) + rt * 128 + ((uc ^ (rt & 7)) << 4)) = qv[k];
     }
     fence_proxy_async_smem();
+  }
+  if (warp != 0) {
+    pdl_wait();
+    pdl_launch_dependents();
   }
   tc_fence_before();
   __syncthreads();

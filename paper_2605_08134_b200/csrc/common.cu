@@ -71,7 +71,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-template <typename T, int MAXV>
+// kEarlyGain: the gain (a weight, independent of the previous kernel in the stream) is read before the dependency
+// wait, which takes one memory round trip off a short step's critical path; it costs registers (half the resident
+// CTAs), so steps with many rows, which are bandwidth-bound, read it afterwards.
+template <typename T, int MAXV, bool kEarlyGain>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, const float* __restrict__ gain,
                                                       T* __restrict__ xn, int d, float eps,
                                                       unsigned long long* dbg) {
@@ -82,11 +85,10 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     if (blockIdx.x == 0) dbg[0] = t;
     atomicMax(&dbg[4], t);                     // latest CTA start
   }
-  // The gain is a weight: it does not depend on the previous kernel in the stream and is read while that one drains.
   const int nvec0 = d / N;
-  float gn[MAXV][N];
+  float gn[kEarlyGain ? MAXV : 1][N];
 #pragma unroll
-  for (int i = 0; i < MAXV; ++i) {
+  for (int i = 0; i < (kEarlyGain ? MAXV : 0); ++i) {
     const int vi = threadIdx.x + i * blockDim.x;
     if (vi < nvec0) {
 #pragma unroll
@@ -132,8 +134,15 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
   for (int i = 0; i < MAXV; ++i) {
     int vi = threadIdx.x + i * blockDim.x;
     if (vi < nvec) {
+      if (!kEarlyGain) {
 #pragma unroll
-      for (int e = 0; e < N; ++e) v[i][e] = v[i][e] * r * gn[i][e];
+        for (int e = 0; e < N; e += 4) {
+          const float4 t = *reinterpret_cast<const float4*>(gain + vi * N + e);
+          gn[0][e] = t.x; gn[0][e + 1] = t.y; gn[0][e + 2] = t.z; gn[0][e + 3] = t.w;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < N; ++e) v[i][e] = v[i][e] * r * gn[kEarlyGain ? i : 0][e];
       Vec16<T>::store(yr + vi * N, v[i]);
     }
   }
@@ -154,7 +163,10 @@ void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float
   int nvec = d / Vec16<T>::N;
   int threads = nvec >= 512 ? 256 : (nvec >= 128 ? 128 : ((nvec + 31) / 32) * 32);
   if (threads > 256) threads = 256;
-  launch_pdl(rmsnorm_kernel<T, 2>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps, dbg);
+  if (rows <= 2048)
+    launch_pdl(rmsnorm_kernel<T, 2, true>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps, dbg);
+  else
+    launch_pdl(rmsnorm_kernel<T, 2, false>, dim3(rows), dim3(threads), 0, st, 1, x, gain, xn, d, eps, dbg);
 }
 template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t,
                                     unsigned long long*);
