@@ -257,16 +257,20 @@ def run_ours(args):
     n_o = n if (mode & 2) else T
     # algorithmic work per launch (what the DARE step itself must move or compute, never the dense work avoided):
     #   projections: 2*M*d*d flop each; the K/V projection of a small refresh set is a stream of both weight
-    #   matrices (2*d*d*2 bytes) plus the gathered rows in and the K, V rows out (3*n*d*2 bytes);
-    #   attention: 4*rows*S*d flop; RMSNorm: read + write of [T, d] bf16; selection: scores in, index list out,
-    #   plus the compacted copy of the refresh set's x_norm rows (read + write) when K/V reuse is on.
+    #   matrices (2*d*d*2 bytes) plus the gathered rows in and the K, V rows out (3*n*d*2 bytes); with many tokens
+    #   (more than eight 128-row tiles) a step that reuses attention outputs projects only the refresh set's rows
+    #   through W_O (its slot then also holds the copy of the reused rows);
+    #   attention: 4*rows*S*d flop; RMSNorm: read + write of [T, d] bf16; selection: scores in, staleness counters
+    #   in and out, index list out.
+    many = shape.batch * ((shape.seq + 127) // 128) > 8
+    n_out = n if ((mode & 2) and many) else T
     work = {
         "q_gemm": ("tensor", 2.0 * T * d * d),
-        "out_gemm": ("tensor", 2.0 * T * d * d),
+        "out_gemm": ("tensor", 2.0 * n_out * d * d),
         "kv_gemm": ("hbm", 2.0 * d * d * 2 + 3.0 * n_kv * d * 2) if n_kv <= 215 else ("tensor", 4.0 * n_kv * d * d),
         "attention": ("tensor", 4.0 * n_o * shape.seq * d),   # n_o counts rows of all sequences
         "rmsnorm": ("hbm", 2.0 * T * d * 2),
-        "select_compact": ("hbm", 4.0 * T + 4.0 * n + (2.0 * n * d * 2 if (mode & 1) else 0.0)),
+        "select_compact": ("hbm", 12.0 * T + 4.0 * n),
     }
     rows = []
     for name, us in kernels.items():
