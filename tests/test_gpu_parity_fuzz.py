@@ -1,0 +1,55 @@
+"""Seeded random geometries through the tensor-core path against the fp64 oracle: odd sequence lengths and windows,
+every mode, refresh sets from empty to full.  The sizes walk across the launch rules of the kernels (split-K or not,
+128- or 256-wide gathered tiles, one or two query tiles per attention CTA, key split, gathered output projection,
+short or long selection)."""
+import numpy as np
+import pytest
+
+from paper_2605_08134_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dare():
+    from paper_2605_08134_b200 import build
+    build.build()
+    from paper_2605_08134_b200 import dare as d
+    return d
+
+
+CASES = [
+    # d_model, batch, seq, prompt
+    (256, 1, 57, 20),
+    (256, 3, 129, 1),
+    (512, 2, 700, 188),
+    (256, 1, 2300, 252),        # few (head, sequence) pairs, many key blocks: key split
+    (512, 5, 1031, 7),          # > 8 row tiles: gathered output projection, 256-wide gathered tiles
+    (1024, 8, 1153, 129),       # two query tiles per attention CTA, dense and row-sparse
+    (1024, 2, 384, 128),
+    (256, 6, 513, 100),
+]
+
+
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_random_steps(dare, case):
+    d_model, batch, seq, prompt = CASES[case]
+    rng = np.random.default_rng(1000 + case)
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=d_model, n_heads=d_model // 128, batch=batch, seq=seq, prompt=prompt)
+    w = wl.make_weights(shape, 300 + case)
+    hs = wl.HiddenStream(shape, 300 + case)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), int(rng.integers(0, 4)), 0.1, shape, first=True)
+    for step in range(4):
+        mode = int(rng.integers(0, 4))
+        frac = float(rng.choice([0.0, 0.03, 0.13, 0.4, 1.0]))
+        n = min(seq, int(round(frac * seq)))
+        ch = wl.uniform_positions(hs.rng, shape, n) if n > 0 else np.zeros((batch, seq), bool)
+        x = hs.advance(ch)
+        if rng.random() < 0.5:
+            parity.compare_step(g, o, x, mode, 0.1, shape)
+        else:
+            parity.compare_step(g, o, np.ascontiguousarray(x[:, prompt:]), mode, 0.1, shape, pos_begin=prompt)
+    g.close()
