@@ -32,10 +32,10 @@ struct StepGeom {
 };
 
 // Launch with programmatic stream serialization (the kernel calls griddepcontrol.wait before touching global data)
-// and, optionally, a thread-block cluster along z.
+// and, optionally, a thread-block cluster along x and z.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_z,
-                       Args&&... args) {
+cudaError_t launch_pdl_xz(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x,
+                          int cluster_z, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -46,9 +46,9 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[n].val.programmaticStreamSerializationAllowed = 1;
   ++n;
-  if (cluster_z > 1) {
+  if (cluster_x > 1 || cluster_z > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
-    attr[n].val.clusterDim.x = 1;
+    attr[n].val.clusterDim.x = cluster_x;
     attr[n].val.clusterDim.y = 1;
     attr[n].val.clusterDim.z = cluster_z;
     ++n;
@@ -56,6 +56,11 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cfg.attrs = attr;
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_z,
+                       Args&&... args) {
+  return launch_pdl_xz(kernel, grid, block, smem, st, 1, cluster_z, static_cast<Args&&>(args)...);
 }
 
 // ---- kernels common to both paths (common.cu) -------------------------------------------------------------

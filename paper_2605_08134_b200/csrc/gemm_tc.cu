@@ -35,11 +35,14 @@ namespace {
 constexpr int BM = 128, BK = 64;
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int HD = 128;                              // head width the rotary/score epilogues assume
-template <int BN>
+// PAIR: two CTAs (row tiles 2i, 2i + 1 of the same column tile and reduction slice) share one M = 256 MMA; each
+// keeps its own 128 rows of A and only half of the W tile's rows in shared memory: 32 KB instead of 48 KB per stage
+// and CTA come through the L2, which is what bounds the main loop of the projections.
+template <int BN, bool PAIR = false>
 struct Cfg {
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;     // this CTA's part of the W tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int STAGES = (PAIR || BN != 256) ? 6 : 4;
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int SMEM_TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
   static constexpr int PROW_BYTES = BN * 4;
@@ -103,16 +106,17 @@ __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParam
   }
 }
 
-template <int EPI, int BN>
+template <int EPI, int BN, bool PAIR>
 __global__ void __launch_bounds__(Warps<BN>::N * 32, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
-  constexpr int STAGES = Cfg<BN>::STAGES, STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
+  using C = Cfg<BN, PAIR>;
+  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
   constexpr int kWarps = Warps<BN>::N, RB = Warps<BN>::RB;
-  constexpr int PROW_BYTES = Cfg<BN>::PROW_BYTES, RECV_OFFSET = Cfg<BN>::RECV_OFFSET;
+  constexpr int PROW_BYTES = C::PROW_BYTES, RECV_OFFSET = C::RECV_OFFSET;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg<BN>::BAR_OFFSET);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + C::BAR_OFFSET);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* accum_bar = empty_bar + STAGES;
   uint64_t* recv_bar = accum_bar + 1;
@@ -121,12 +125,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // the warp index through a shuffle: the compiler then knows the role decisions and the descriptors derived from
   // it to be uniform over the warp
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  const int nt = blockIdx.x, mt = blockIdx.y;
+  // (a pair launch has the row tiles along x: the two CTAs of an MMA pair are neighbours in x)
+  const int nt = PAIR ? blockIdx.y : blockIdx.x, mt = PAIR ? blockIdx.x : blockIdx.y;
   const int splits = gridDim.z;                 // = cluster size along z
-  const int z = (int)cluster_ctarank();
+  // cluster = (PAIR ? 2 : 1, 1, splits): rank = place in the MMA pair + 2 * reduction slice
+  const int crank = (int)cluster_ctarank();
+  const int pr = PAIR ? (crank & 1) : 0;        // place in the MMA pair; place 0 issues the MMAs
+  const int z = PAIR ? (crank >> 1) : crank;    // reduction slice
+  const uint32_t lead = (uint32_t)(crank & ~1); // cluster rank of the pair's issuing CTA
+  auto rank_of_slice = [&](int zz) { return (uint32_t)(PAIR ? 2 * zz + pr : zz); };
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  const int lin = (z * gridDim.y + mt) * gridDim.x + nt;
+  const int lin = (z * (int)(PAIR ? gridDim.x : gridDim.y) + mt) * (int)(PAIR ? gridDim.y : gridDim.x) + nt;
   const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
@@ -150,7 +160,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // into the swizzled tile layout (the TMA producer then only brings the W tiles); each of them arrives on a stage
   // once its rows of that stage have landed.
   const bool gather = p.gather_src != nullptr;
-  const uint32_t tx_bytes = gather ? (uint32_t)Cfg<BN>::B_BYTES : (uint32_t)STAGE_BYTES;
+  const uint32_t tx_bytes = gather ? (uint32_t)C::B_BYTES : (uint32_t)STAGE_BYTES;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], gather ? 5 : 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(accum_bar, 1);
@@ -161,23 +171,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     prefetch_tmap(tm_b);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
-    tmem_relinquish();
+    if (PAIR) { tmem_alloc2(tmem_slot, BN); tmem_relinquish2(); }
+    else { tmem_alloc(tmem_slot, BN); tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  uint32_t tmem_base;
+  if (PAIR) {
+    // both CTAs of the pair have their barriers and their tensor memory before either touches the other's
+    cluster_sync_all();
+    tc_fence_after();
+    tmem_base = ld_cluster_u32(map_to_cta(smem_u32(tmem_slot), lead));
+  } else {
+    tc_fence_after();
+    tmem_base = *tmem_slot;
+  }
   // The weights do not depend on the previous kernel in the stream: the producer starts their first tiles now, so
   // that they stream in while that kernel drains.  Everything it produced is needed only after pdl_wait().
   const int n_early = likely ? (nkb < STAGES ? nkb : STAGES) : 0;
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
-      mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
       uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
+      if (PAIR) {
+        // the bytes of both CTAs are counted on the issuing CTA's barrier; each CTA brings its half of the W rows
+        if (pr == 0) mbar_arrive_expect_tx(&full_bar[i], 2 * STAGE_BYTES);
+        tma_load_2d_pair(b_dst, tm_b, (kb_begin + i) * BK, n0 + pr * (BN / 2), map_to_cta(smem_u32(&full_bar[i]), lead));
+        continue;
+      }
+      mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
       if (p.b_pair) {
         tma_load_2d(b_dst, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[i]);
-        tma_load_2d(b_dst + Cfg<BN>::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[i]);
+        tma_load_2d(b_dst + C::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[i]);
       } else {
         tma_load_2d(b_dst, tm_b, (kb_begin + i) * BK, n0, &full_bar[i]);
       }
@@ -199,9 +223,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     rows_valid = min(BM, n - t0);
     a_row = t0;
   } else {
-    const int b = mt / p.tiles_per_seq, tis = mt - b * p.tiles_per_seq;
+    // (a pair launch pads the row tiles to an even number: the tile past the end runs the main loop for its
+    // partner's sake, on the first tile's rows, and finishes no rows)
+    const bool exists = mt < p.m_tiles;
+    const int mte = exists ? mt : 0;
+    const int b = mte / p.tiles_per_seq, tis = mte - b * p.tiles_per_seq;
     t0 = b * p.seq_act + tis * BM;
-    rows_valid = min(BM, p.seq_act - tis * BM);
+    rows_valid = exists ? min(BM, p.seq_act - tis * BM) : 0;
     a_row = b * p.a_seq_stride + p.a_row0 + tis * BM;
     pos0 = p.g.pos_begin + tis * BM;
     crow0 = (size_t)b * p.g.max_seq + pos0;
@@ -220,8 +248,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // issues: the operands of the copies and MMAs are then warp-uniform values, which is what those instructions take.
   if (warp == 0) {
     if (!gather && elect_one()) {
-      for (int i = 0; i < n_early; ++i)          // the W halves of these stages are already on their way
-        tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
+      for (int i = 0; i < n_early; ++i) {        // the W halves of these stages are already on their way
+        if (PAIR)
+          tma_load_2d_pair(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, map_to_cta(smem_u32(&full_bar[i]), lead));
+        else
+          tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
+      }
     }
     __syncwarp();
     for (int i = n_early; i < nkb; ++i) {
@@ -229,35 +261,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
       if (elect_one()) {
         uint8_t* a_dst = smem + s * STAGE_BYTES;
-        mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-        if (!gather) tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
-        if (p.b_pair) {
-          tma_load_2d(a_dst + A_BYTES, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[s]);
-          tma_load_2d(a_dst + A_BYTES + Cfg<BN>::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[s]);
+        if (PAIR) {
+          const uint32_t fb = map_to_cta(smem_u32(&full_bar[s]), lead);
+          if (pr == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * STAGE_BYTES);
+          tma_load_2d_pair(a_dst, &tm_a, (kb_begin + i) * BK, a_row, fb);
+          tma_load_2d_pair(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0 + pr * (BN / 2), fb);
         } else {
-          tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
+          mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
+          if (!gather) tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
+          if (p.b_pair) {
+            tma_load_2d(a_dst + A_BYTES, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[s]);
+            tma_load_2d(a_dst + A_BYTES + C::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[s]);
+          } else {
+            tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
+          }
         }
       }
       __syncwarp();
     }
   } else if (warp == 1) {
-    constexpr uint32_t idesc = idesc_bf16(BM, BN);
-    for (int i = 0; i < nkb; ++i) {
-      const int s = i % STAGES;
-      mbar_wait(&full_bar[s], (i / STAGES) & 1, p.status);
-      tc_fence_after();
-      if (dbg && i == 0 && lane == 0) p.debug[2] = globaltimer_ns();
-      if (elect_one()) {
-        const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
-        const uint64_t a_desc = smem_desc_k_sw128(a_addr);
-        const uint64_t b_desc = smem_desc_k_sw128(a_addr + A_BYTES);
+    if (!PAIR || pr == 0) {
+      // (in a pair only the even-ranked CTA issues: one M = 256 MMA covers both CTAs' rows)
+      constexpr uint32_t idesc = idesc_bf16(PAIR ? 2 * BM : BM, BN);
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % STAGES;
+        mbar_wait(&full_bar[s], (i / STAGES) & 1, p.status);
+        tc_fence_after();
+        if (dbg && i == 0 && lane == 0) p.debug[2] = globaltimer_ns();
+        if (elect_one()) {
+          const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
+          const uint64_t a_desc = smem_desc_k_sw128(a_addr);
+          const uint64_t b_desc = smem_desc_k_sw128(a_addr + A_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
-          umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
-        umma_commit(&empty_bar[s]);
-        if (i == nkb - 1) umma_commit(accum_bar);      // by the thread that issued the MMAs it covers
+          for (int k = 0; k < BK / 16; ++k) {  // 16 k-elements = 32 bytes = 2 descriptor address units per MMA
+            if (PAIR) umma2_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
+            else umma_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
+          }
+          // the stage is free again, in both CTAs of a pair; after the last one the accumulators are complete
+          if (PAIR) {
+            umma2_commit(map_to_cta(smem_u32(&empty_bar[s]), lead));
+            umma2_commit(map_to_cta(smem_u32(&empty_bar[s]), lead + 1));
+            if (i == nkb - 1) {
+              umma2_commit(map_to_cta(smem_u32(accum_bar), lead));
+              umma2_commit(map_to_cta(smem_u32(accum_bar), lead + 1));
+            }
+          } else {
+            umma_commit(&empty_bar[s]);
+            if (i == nkb - 1) umma_commit(accum_bar);      // by the thread that issued the MMAs it covers
+          }
+        }
+        __syncwarp();
       }
-      __syncwarp();
     }
   } else {
     // While the main loop runs, pull the table rows the finishing pass of this CTA will read into the L2
@@ -349,8 +403,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if ((kWarps != 8 || warp < 4) && lane == 0) {
           const int rl0 = quarter * 32 - owner * rows_per_cta;
           const uint32_t src = smem_u32(smem + (size_t)(quarter * 32) * PROW_BYTES);
-          const uint32_t rdst = map_to_cta(smem_u32(smem + RECV_OFFSET + (size_t)rl0 * PROW_BYTES), (uint32_t)owner);
-          const uint32_t rbar = map_to_cta(smem_u32(recv_bar), (uint32_t)owner);
+          const uint32_t rdst = map_to_cta(smem_u32(smem + RECV_OFFSET + (size_t)rl0 * PROW_BYTES), rank_of_slice(owner));
+          const uint32_t rbar = map_to_cta(smem_u32(recv_bar), rank_of_slice(owner));
           bulk_copy_to_cta(rdst, src, 32 * PROW_BYTES, rbar);
         }
       }
@@ -500,38 +554,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
   tc_fence_before();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
-  if (splits > 1) cluster_sync_all(); else __syncthreads();
+  // (nor frees tensor memory its MMA partner may still read through)
+  if (splits > 1 || PAIR) cluster_sync_all(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
-  if (warp == 1) tmem_dealloc(tmem_base, BN);
+  if (warp == 1) {
+    if (PAIR) tmem_dealloc2(*tmem_slot, BN);
+    else tmem_dealloc(tmem_base, BN);
+  }
 }
 
-template <int EPI, int BN>
+template <int EPI, int BN, bool PAIR>
 static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
                               int n_tiles, int m_tiles, int splits, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = gemm_tc_kernel<EPI, BN>;
-  constexpr int SMEM_TOTAL = Cfg<BN>::SMEM_TOTAL;
+  auto kern = gemm_tc_kernel<EPI, BN, PAIR>;
+  constexpr int SMEM_TOTAL = Cfg<BN, PAIR>::SMEM_TOTAL;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pdl(kern, dim3(n_tiles, m_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, splits, a, b0, b1, p);
+  GemmParams q = p;
+  q.m_tiles = m_tiles;
+  if (PAIR)
+    return launch_pdl_xz(kern, dim3((m_tiles + 1) / 2 * 2, n_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, 2,
+                         splits, a, b0, b1, q);
+  return launch_pdl_xz(kern, dim3(n_tiles, m_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, 1, splits, a, b0, b1,
+                       q);
 }
 
+// pair != 0: the launch uses two-CTA MMAs (256-wide tiles, A through the tensor map); b0 / b1 must then be maps with
+// 128-row boxes.
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st) {
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
   if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
-  if (bn == 256) {
-    if (epi == EPI_Q) return launch_one<EPI_Q, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
-    if (epi == EPI_KV) return launch_one<EPI_KV, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
-    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
-    if (epi == EPI_F32) return launch_one<EPI_F32, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
-    return launch_one<EPI_OUT, 256>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+  if (pair) {
+    if (bn != 256 || p.gather_src != nullptr || p.count != nullptr || p.b_pair) return cudaErrorInvalidValue;
+    if (epi == EPI_Q) return launch_one<EPI_Q, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_KV) return launch_one<EPI_KV, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_OUT) return launch_one<EPI_OUT, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    return cudaErrorInvalidValue;
   }
-  if (bn == 128 && epi == EPI_KV) return launch_one<EPI_KV, 128>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+  if (bn == 256) {
+    if (epi == EPI_Q) return launch_one<EPI_Q, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_KV) return launch_one<EPI_KV, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_F32) return launch_one<EPI_F32, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    return launch_one<EPI_OUT, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+  }
+  if (bn == 128 && epi == EPI_KV) return launch_one<EPI_KV, 128, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
   return cudaErrorInvalidValue;
 }
 

@@ -9,11 +9,22 @@ namespace dare {
 struct TcState {
   CUtensorMap a_xn, a_oc;                  // A operands, box 64 x 128 rows
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 256 rows
-  CUtensorMap w_k128, w_v128;              // weights, box 64 x 128 rows
+  CUtensorMap w_k128, w_v128, w_q128, w_o128;   // weights, box 64 x 128 rows
   CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 128 rows (keys)
 };
 
 namespace {
+
+#ifndef DARE_PAIR_MMA
+#define DARE_PAIR_MMA 1
+#endif
+// Two-CTA MMAs (pairs of row tiles share their W tile: a third less operand traffic from the L2 per CTA) for the
+// launches of about one wave, whose main loops are bound by that traffic; launches of many waves measured slower
+// with them (they are bound by the tensor pipe under the power cap, and the pair adds two cluster barriers and
+// ties two SMs' pipelines together).
+bool use_pairs(int n_tiles, int m_tiles, int splits) {
+  return DARE_PAIR_MMA != 0 && m_tiles >= 2 && n_tiles * ((m_tiles + 1) / 2 * 2) * splits <= 160;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -68,7 +79,8 @@ dare_status_t tc_create(dare_layer* L) {
             make_map(&s->a_oc, L->buf.oc, Tm, d, 128) && make_map(&s->w_q, L->w.w_q, d, d, 256) &&
             make_map(&s->w_k, L->w.w_k, d, d, 256) && make_map(&s->w_v, L->w.w_v, d, d, 256) &&
             make_map(&s->w_o, L->w.w_o, d, d, 256) && make_map(&s->w_k128, L->w.w_k, d, d, 128) &&
-            make_map(&s->w_v128, L->w.w_v, d, d, 128) && make_map(&s->kc64, L->buf.kc, Tm, d, 128) &&
+            make_map(&s->w_v128, L->w.w_v, d, d, 128) && make_map(&s->w_q128, L->w.w_q, d, d, 128) &&
+            make_map(&s->w_o128, L->w.w_o, d, d, 128) && make_map(&s->kc64, L->buf.kc, Tm, d, 128) &&
             make_map(&s->vc64, L->buf.vc, Tm, d, 128);
   if (!ok) { delete s; return DARE_ERR_CUDA; }
   L->tc = s;
@@ -120,8 +132,12 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     p.debug = dbg;
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_Q_GEMM, st);
-    e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense,
-                       pick_splits(n_tiles * m_tiles_dense, kblocks), st); ++launches;
+    const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
+    if (use_pairs(n_tiles, m_tiles_dense, sp))
+      e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
+    else
+      e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, sp, st);
+    ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // lines 4-5 + Sec. 4
@@ -153,8 +169,12 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       }
     } else {
       prof_mark(L, SLOT_KV_GEMM, st);
-      e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense,
-                         pick_splits(n_tiles * m_tiles_dense, kblocks), st); ++launches;
+      const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
+      if (use_pairs(n_tiles, m_tiles_dense, sp))
+        e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, sp, st, 1);
+      else
+        e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, sp, st);
+      ++launches;
     }
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
@@ -190,8 +210,12 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       if (e != cudaSuccess) return DARE_ERR_CUDA;
       launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
     } else {
-      e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense,
-                         pick_splits(n_tiles * m_tiles_dense, kblocks), st); ++launches;
+      const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
+      if (use_pairs(n_tiles, m_tiles_dense, sp))
+        e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, sp, st, 1);
+      else
+        e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, sp, st);
+      ++launches;
       if (e != cudaSuccess) return DARE_ERR_CUDA;
       // the cache is complete once a dense projection has covered every cached row, and stays so while every
       // later step maintains it

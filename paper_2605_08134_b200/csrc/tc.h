@@ -11,6 +11,7 @@ enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2, EPI_SWIGLU = 3, EPI_F32 = 4 };
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
+  int m_tiles;           // row tiles of the launch (set by the launcher; a pair launch pads its grid to an even count)
   int m_total;           // dense: tokens of the step; gathered: capacity of the row list
   int seq_act;           // dense row mapping: rows per sequence ...
   int tiles_per_seq;     // ... and 128-row tiles per sequence
@@ -62,7 +63,7 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
 bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st);
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair = 0);
 
 
 }  // namespace dare
