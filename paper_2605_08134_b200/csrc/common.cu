@@ -1,4 +1,5 @@
 // Memory-bound kernels shared by both kernel paths: rotary table, RMSNorm, threshold + compaction, row gather.
+#include <type_traits>
 #include "dare_internal.h"
 #include "tc_ptx.cuh"
 
@@ -156,10 +157,94 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
   if (dbg && threadIdx.x == 0) atomicMax(&dbg[5], ptx::globaltimer_ns());   // latest CTA end
 }
 
+// Many rows (the step is then a stream through HBM): a CTA takes ROWS consecutive rows at once, all of their loads in
+// flight before the one block reduction they share, the data kept as packed bf16 between the two passes.
+// d <= 4096 (two 16-byte vectors per thread).
+template <int ROWS>
+__global__ void __launch_bounds__(256) rmsnorm_stream_kernel(const __nv_bfloat16* __restrict__ x,
+                                                             const float* __restrict__ gain,
+                                                             __nv_bfloat16* __restrict__ xn, int rows, int d, float eps) {
+  __shared__ float red[8][ROWS];
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
+  const int nvec = d / 8, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const size_t row0 = (size_t)blockIdx.x * ROWS;
+  uint4 raw[ROWS][2];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int vi = threadIdx.x + i * 256;
+      raw[r][i] = make_uint4(0u, 0u, 0u, 0u);
+      if (vi < nvec && row0 + r < (size_t)rows) raw[r][i] = *reinterpret_cast<const uint4*>(x + (row0 + r) * d + vi * 8);
+    }
+  }
+  float ss[ROWS];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    ss[r] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[r][i]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(h[e]);
+        ss[r] += f.x * f.x + f.y * f.y;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss[r] += __shfl_xor_sync(0xffffffffu, ss[r], o);
+    if (lane == 0) red[warp][r] = ss[r];
+  }
+  __syncthreads();
+  float gn[2][8];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int vi = threadIdx.x + i * 256;
+    if (vi < nvec) {
+#pragma unroll
+      for (int e = 0; e < 8; e += 4) {
+        const float4 t = *reinterpret_cast<const float4*>(gain + vi * 8 + e);
+        gn[i][e] = t.x; gn[i][e + 1] = t.y; gn[i][e + 2] = t.z; gn[i][e + 3] = t.w;
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w][r];
+    const float sc = rsqrtf(tot / (float)d + eps);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int vi = threadIdx.x + i * 256;
+      if (vi < nvec && row0 + r < (size_t)rows) {
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[r][i]);
+        uint4 o;
+        __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(h[e]);
+          oh[e] = __floats2bfloat162_rn(f.x * sc * gn[i][2 * e], f.y * sc * gn[i][2 * e + 1]);
+        }
+        *reinterpret_cast<uint4*>(xn + (row0 + r) * d + vi * 8) = o;
+      }
+    }
+  }
+}
+
 template <typename T>
 void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float eps, cudaStream_t st,
                     unsigned long long* dbg) {
   if (rows <= 0) return;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    constexpr int ROWS = 4;
+    if (rows > 2048 && d % 8 == 0 && d / 8 <= 512 && dbg == nullptr) {
+      launch_pdl(rmsnorm_stream_kernel<ROWS>, dim3((rows + ROWS - 1) / ROWS), dim3(256), 0, st, 1, x, gain, xn, rows, d,
+                 eps);
+      return;
+    }
+  }
   int nvec = d / Vec16<T>::N;
   int threads = nvec >= 512 ? 256 : (nvec >= 128 ? 128 : ((nvec + 31) / 32) * 32);
   if (threads > 256) threads = 256;
