@@ -1,7 +1,7 @@
 """Seeded random geometries through the tensor-core path against the fp64 oracle: odd sequence lengths and windows,
 every mode, refresh sets from empty to full.  The sizes walk across the launch rules of the kernels (split-K or not,
 128- or 256-wide gathered tiles, one or two query tiles per attention CTA, key split, gathered output projection,
-short or long selection)."""
+short or long selection, two-CTA MMAs with an even or odd number of row tiles)."""
 import numpy as np
 import pytest
 
@@ -29,6 +29,10 @@ CASES = [
     (1024, 8, 1153, 129),       # two query tiles per attention CTA, dense and row-sparse
     (1024, 2, 384, 128),
     (256, 6, 513, 100),
+    (256, 3, 100, 10),          # three row tiles: MMA pairs with a padding tile, split reduction
+    (512, 1, 384, 64),
+    (512, 1, 100, 10),
+    (1024, 2, 256, 64),
 ]
 
 
