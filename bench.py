@@ -238,6 +238,32 @@ def run_ours(args):
         lay.set_profiling(False)
     kernels = {k: 1e3 * sum(v) / len(v) for k, v in acc.items()}          # microseconds per launch
 
+    # ---- the same kernels inside the undisturbed chain: device timestamps (%globaltimer) written by the kernels
+    # themselves, from the return of a kernel's wait on its predecessor to the exit of its last CTA.  The events of
+    # the pass above break the programmatic launch overlap and add a few microseconds to every kernel; these do not.
+    in_chain = {}
+    if True:
+        try:
+            one_pass(2 * len(layers), mode)
+            for lay in layers:
+                lay.debug_timestamps(True)
+            one_pass(4 * len(layers), mode)
+            torch.cuda.synchronize()
+            acc2 = {}
+            for lay in layers:
+                ts = lay.debug_timestamps(False).astype(np.int64)
+                q, kv, at, out = ts[0], ts[1], ts[2], ts[3]
+                if min(q[1], kv[1], out[1], at[0]) <= 0:
+                    continue
+                for name, us in (("q_gemm", (q[6] - q[1]) / 1e3), ("kv_gemm", (kv[6] - kv[1]) / 1e3),
+                                 ("attention", (at[6] - max(at[0], kv[6])) / 1e3), ("out_gemm", (out[6] - out[1]) / 1e3)):
+                    if 0 < us < 1e6:
+                        acc2.setdefault(name, []).append(us)
+            in_chain = {k: sum(v) / len(v) for k, v in acc2.items()}
+        except Exception:                 # diagnostics only: the bench line stands without them
+            in_chain = {}
+        barrier()
+
     # ---- end to end through the host-buffer entry point (pinned host x and y, copies inside the timed region)
     prime(mode)
     xh = [torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).pin_memory() for a in (xa_np, xb_np)]
@@ -282,16 +308,24 @@ def run_ours(args):
                 ach, peak, unit = amount / (us * 1e-6) / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
             rows.append({"kernel": name, "us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": peak,
                          "unit": unit, "frac": round(ach / peak, 4)})
+            if name in in_chain:
+                scale = 1e9 if bound == "hbm" else 1e12
+                rows[-1]["in_chain"] = {"us": round(in_chain[name], 2),
+                                        "achieved": round(amount / (in_chain[name] * 1e-6) / scale, 1),
+                                        "frac": round(amount / (in_chain[name] * 1e-6) / scale / peak, 4)}
         else:
             rows.append({"kernel": name, "us": round(us, 2)})
     dom = max((r for r in rows if "bound" in r), key=lambda r: r["us"])
     # DRAM bytes per launch of that kernel from one ncu capture of this workload (profiles/ holds the summaries)
-    ncu_traffic = {"q_gemm": 38.4e6, "kv_gemm": 69.3e6, "out_gemm": 37.9e6}
+    ncu_traffic = {"q_gemm": 38.3e6, "kv_gemm": 68.7e6, "out_gemm": 37.8e6}
     roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
                 "unit": dom["unit"], "frac": dom["frac"],
                 "traffic": ncu_traffic.get(dom["kernel"]) if shape.name == wl.LLADA_LAYER.name else None,
                 "peak_source": f"of {peaks['source']} (sustained figure: the kernel is timed inside the step)",
-                "timing": "CUDA events recorded by the library around each kernel, second pass of K steps"}
+                "timing": "CUDA events recorded by the library around each kernel, second pass of K steps",
+                "in_chain": dom.get("in_chain"),
+                "in_chain_timing": "device timestamps inside the undisturbed programmatic-launch chain: return of the "
+                                   "kernel's wait on its predecessor -> exit of its last CTA"}
 
     # ---- CPU baseline: the oracle as it stands, bounded sample
     cpu = None if args.no_cpu_baseline else cpu_baseline(shape, xa_np, xb_np, layers[0], mode, budget_s=12.0)
