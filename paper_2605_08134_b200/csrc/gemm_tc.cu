@@ -194,8 +194,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
       if (PAIR) {
         // the bytes of both CTAs are counted on the issuing CTA's barrier; each CTA brings its half of the W rows
+        // (a tile of two matrices: the even CTA brings the rows of the first, the odd one those of the second)
         if (pr == 0) mbar_arrive_expect_tx(&full_bar[i], 2 * STAGE_BYTES);
-        tma_load_2d_pair(b_dst, tm_b, (kb_begin + i) * BK, n0 + pr * (BN / 2), map_to_cta(smem_u32(&full_bar[i]), lead));
+        tma_load_2d_pair(b_dst, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, (kb_begin + i) * BK,
+                         p.b_pair ? n0 : n0 + pr * (BN / 2), map_to_cta(smem_u32(&full_bar[i]), lead));
         continue;
       }
       mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
@@ -265,7 +267,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const uint32_t fb = map_to_cta(smem_u32(&full_bar[s]), lead);
           if (pr == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * STAGE_BYTES);
           tma_load_2d_pair(a_dst, &tm_a, (kb_begin + i) * BK, a_row, fb);
-          tma_load_2d_pair(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0 + pr * (BN / 2), fb);
+          tma_load_2d_pair(a_dst + A_BYTES, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, (kb_begin + i) * BK,
+                           p.b_pair ? n0 : n0 + pr * (BN / 2), fb);
         } else {
           mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
           if (!gather) tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
@@ -591,7 +594,9 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
   if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
   if (pair) {
-    if (bn != 256 || p.gather_src != nullptr || p.count != nullptr || p.b_pair) return cudaErrorInvalidValue;
+    if (bn != 256 || p.gather_src != nullptr || p.count != nullptr || (p.b_pair != 0) != (epi == EPI_SWIGLU))
+      return cudaErrorInvalidValue;
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_Q) return launch_one<EPI_Q, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_KV) return launch_one<EPI_KV, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_OUT) return launch_one<EPI_OUT, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);

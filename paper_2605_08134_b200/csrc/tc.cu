@@ -18,13 +18,7 @@ namespace {
 #ifndef DARE_PAIR_MMA
 #define DARE_PAIR_MMA 1
 #endif
-// Two-CTA MMAs (pairs of row tiles share their W tile: a third less operand traffic from the L2 per CTA) for the
-// launches of about one wave, whose main loops are bound by that traffic; launches of many waves measured slower
-// with them (they are bound by the tensor pipe under the power cap, and the pair adds two cluster barriers and
-// ties two SMs' pipelines together).
-bool use_pairs(int n_tiles, int m_tiles, int splits) {
-  return DARE_PAIR_MMA != 0 && m_tiles >= 2 && n_tiles * ((m_tiles + 1) / 2 * 2) * splits <= 160;
-}
+bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0 && pairs_pay(n_tiles, m_tiles, splits); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

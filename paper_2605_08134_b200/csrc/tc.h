@@ -62,6 +62,15 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
 // Row-major bf16 matrix [rows, cols] as a TMA tensor map with a box of 64 columns x box_rows rows, 128-byte swizzle.
 bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
+// Two-CTA MMAs (pairs of row tiles share their W tile: a third less operand traffic from the L2 per CTA) pay where
+// the main loop is bound by that traffic: launches of at most four row tiles, or of about one wave.  Launches of
+// many waves measured slower with them (they are bound by the tensor pipe under the power cap, and the pair adds two
+// cluster barriers and ties two SMs' pipelines together).
+inline bool pairs_pay(int n_tiles, int m_tiles, int splits) {
+  const int ctas = n_tiles * ((m_tiles + 1) / 2 * 2) * splits;
+  return m_tiles >= 2 && (ctas <= 160 || m_tiles <= 4);
+}
+
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                            const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair = 0);
 
