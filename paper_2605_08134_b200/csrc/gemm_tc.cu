@@ -20,7 +20,7 @@
 //   Q    drift score of the scoring head against the stored query (Sec. 3.1), store of the new query, rotary
 //        embedding, bf16 store
 //   K/V  rotary embedding of K, scatter of both rows into the caches at the refresh-set rows (Eq. 3)
-//   OUT  bf16 store of y, optionally plus a residual row
+//   OUT  bf16 store of y (OUT_RES: plus a residual row, read together with the row's tables)
 //   SWIGLU  silu(gate) * up of a tile that holds both projections of the same 128 outputs (MLP of a stack)
 //   F32  fp32 store (logits of a stack's LM head)
 #include "layer.h"
@@ -74,12 +74,13 @@ struct RowBatch {
   bool ok[RB];
   float4 cs[RB];          // (cos, sin) of the two rotary pairs this lane owns
   float2 qa[RB], qb[RB];  // stored query of the scoring head: elements 2*lane.. and 64 + 2*lane..
+  __nv_bfloat162 res[RB][2][2];   // residual row (output projection of a transformer block): this lane's pairs per head
 };
 
-template <int EPI, int RB, int kWarps>
+template <int EPI, int RB, int kWarps, int BN>
 __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParams& p, int rl0, int z, int rows_per_cta,
                                                int rows_valid, int t0, int pos0, size_t crow0, bool rotate,
-                                               bool score_tile, int lane) {
+                                               bool score_tile, int lane, int n0) {
 #pragma unroll
   for (int k = 0; k < RB; ++k) {
     const int rl = rl0 + kWarps * k;
@@ -102,6 +103,14 @@ __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParam
     if (EPI == EPI_Q && score_tile && p.has_prev) {
       rb.qa[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + 2 * lane);
       rb.qb[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + HD / 2 + 2 * lane);
+    }
+    if (EPI == EPI_OUT_RES) {
+      const __nv_bfloat16* rs = p.resid + (size_t)rb.tok[k] * p.ld_resid + n0;
+#pragma unroll
+      for (int hh = 0; hh < BN / HD; ++hh) {
+        rb.res[k][hh][0] = *reinterpret_cast<const __nv_bfloat162*>(rs + hh * HD + 2 * lane);
+        rb.res[k][hh][1] = *reinterpret_cast<const __nv_bfloat162*>(rs + hh * HD + HD / 2 + 2 * lane);
+      }
     }
   }
 }
@@ -328,7 +337,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
     // the table reads of this warp's first rows of the finishing pass: in flight for the whole main loop
-    load_row_batch<EPI, RB, kWarps>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+    load_row_batch<EPI, RB, kWarps, BN>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
     if (gather && warp < 6) {
       // One stage of the A tile = 128 rows x 128 bytes (64 k-elements).  A warp takes 32 rows; one of its copy
       // instructions covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row, so every
@@ -373,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   // The table reads of the first rows the producer and MMA warps will finish start now (those of the other warps
   // started before the main loop) and land during the exchange below.
-  if (warp < 2) load_row_batch<EPI, RB, kWarps>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+  if (warp < 2) load_row_batch<EPI, RB, kWarps, BN>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
 
   // ---- every CTA of the cluster has finished its main loop: the rings are free to receive partial rows
   tc_fence_before();
@@ -424,7 +433,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
 #pragma unroll 1
     for (int rl0 = warp; rl0 < rows_per_cta; rl0 += kWarps * RB) {
-      if (rl0 != warp) load_row_batch<EPI, RB, kWarps>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane);
+      if (rl0 != warp) load_row_batch<EPI, RB, kWarps, BN>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
       if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[34 + (rl0 - warp) / (kWarps * RB) * 2] = globaltimer_ns();
       // (1) combine the partial rows: lane <-> pairs (2*lane, 2*lane+1) of each head
       float2 vlo[RB][BN / HD], vhi[RB][BN / HD];
@@ -522,16 +531,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             *reinterpret_cast<float2*>(d32 + c_hi) = hi;
             continue;
           }
-          if (EPI == EPI_OUT && p.resid != nullptr) {
-            const __nv_bfloat16* rs = p.resid + (size_t)rb.tok[k] * p.ld_resid + n0;
-            const float2 ra = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(rs + c_lo));
-            const float2 rb2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(rs + c_hi));
+          if (EPI == EPI_OUT_RES) {                                  // (read with the row's tables, long before)
+            const float2 ra = __bfloat1622float2(rb.res[k][hh][0]), rb2 = __bfloat1622float2(rb.res[k][hh][1]);
             lo.x += ra.x; lo.y += ra.y; hi.x += rb2.x; hi.y += rb2.y;
           }
           const __nv_bfloat162 o_lo = __floats2bfloat162_rn(lo.x, lo.y), o_hi = __floats2bfloat162_rn(hi.x, hi.y);
           *reinterpret_cast<__nv_bfloat162*>(dst + c_lo) = o_lo;
           *reinterpret_cast<__nv_bfloat162*>(dst + c_hi) = o_hi;
-          if (EPI == EPI_OUT && p.out1 != nullptr) {       // second copy, by cache row: the projected-output cache
+          if ((EPI == EPI_OUT || EPI == EPI_OUT_RES) && p.out1 != nullptr) {       // second copy, by cache row: the projected-output cache
             __nv_bfloat16* dst2 = p.out1 + rb.crow[k] * p.ld_out + n0;
             *reinterpret_cast<__nv_bfloat162*>(dst2 + c_lo) = o_lo;
             *reinterpret_cast<__nv_bfloat162*>(dst2 + c_hi) = o_hi;
@@ -592,6 +599,7 @@ static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                            const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
+  if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
   if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
   if (pair) {
     if (bn != 256 || p.gather_src != nullptr || p.count != nullptr || (p.b_pair != 0) != (epi == EPI_SWIGLU))
@@ -600,6 +608,7 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
     if (epi == EPI_Q) return launch_one<EPI_Q, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_KV) return launch_one<EPI_KV, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_OUT) return launch_one<EPI_OUT, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_OUT_RES) return launch_one<EPI_OUT_RES, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     return cudaErrorInvalidValue;
   }
   if (bn == 256) {
@@ -607,6 +616,7 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
     if (epi == EPI_KV) return launch_one<EPI_KV, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     if (epi == EPI_F32) return launch_one<EPI_F32, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_OUT_RES) return launch_one<EPI_OUT_RES, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
     return launch_one<EPI_OUT, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
   }
   if (bn == 128 && epi == EPI_KV) return launch_one<EPI_KV, 128, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st);

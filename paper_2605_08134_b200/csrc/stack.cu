@@ -70,55 +70,71 @@ __global__ void cand_kernel(const int* __restrict__ tokens, int batch, int seq_t
 }
 
 // Per candidate row of the logits: argmax (lowest index on ties, the mask id excluded) and its softmax probability.
+// One pass over the row: every thread keeps a running maximum (with its index) and the sum of exp(v - maximum),
+// rescaled when the maximum moves; the triples are then merged over the warp and the CTA.
+struct RowStat {
+  float m, s;
+  int arg;
+};
+__device__ __forceinline__ void stat_add(RowStat& a, float v, int j) {
+  if (v > a.m) {
+    a.s = a.s * __expf(a.m - v) + 1.f;      // (exp(-inf) = 0 covers the first element)
+    a.m = v; a.arg = j;
+  } else {
+    a.s += __expf(v - a.m);
+  }
+}
+__device__ __forceinline__ void stat_merge(RowStat& a, float om, float os, int oa) {
+  const bool take = om > a.m || (om == a.m && oa < a.arg);
+  const float M = fmaxf(a.m, om);
+  const float sa = a.m == -INFINITY ? 0.f : a.s * __expf(a.m - M), sb = om == -INFINITY ? 0.f : os * __expf(om - M);
+  a.s = sa + sb; a.m = M;
+  if (take) a.arg = oa;
+}
 __global__ void __launch_bounds__(1024) rowstats_kernel(const float* __restrict__ logits, const int* __restrict__ count,
                                                         int vocab, int mask_id, int* __restrict__ tok,
                                                         float* __restrict__ prob) {
-  __shared__ float s_max[32];
+  __shared__ float s_max[32], s_sum[32];
   __shared__ int s_arg[32];
-  __shared__ float s_sum[32];
   const int r = blockIdx.x;
   if (r >= *count) return;
   const float* row = logits + (size_t)r * vocab;
-  float mx = -INFINITY;
-  int arg = 0x7fffffff;
-  for (int j = threadIdx.x; j < vocab; j += blockDim.x) {
-    if (j == mask_id) continue;
-    const float v = row[j];
-    if (v > mx || (v == mx && j < arg)) { mx = v; arg = j; }
+  RowStat a{-INFINITY, 0.f, 0x7fffffff};
+  if ((vocab & 3) == 0) {                                   // rows then start on 16-byte boundaries
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    for (int j4 = threadIdx.x; j4 < vocab / 4; j4 += blockDim.x) {
+      const float4 v = row4[j4];
+      const int j = 4 * j4;
+      if (j != mask_id) stat_add(a, v.x, j);
+      if (j + 1 != mask_id) stat_add(a, v.y, j + 1);
+      if (j + 2 != mask_id) stat_add(a, v.z, j + 2);
+      if (j + 3 != mask_id) stat_add(a, v.w, j + 3);
+    }
+  } else {
+    for (int j = threadIdx.x; j < vocab; j += blockDim.x)
+      if (j != mask_id) stat_add(a, row[j], j);
   }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, mx, o);
-    const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
-    if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+    const float om = __shfl_xor_sync(0xffffffffu, a.m, o), os = __shfl_xor_sync(0xffffffffu, a.s, o);
+    const int oa = __shfl_xor_sync(0xffffffffu, a.arg, o);
+    stat_merge(a, om, os, oa);
   }
-  if (lane == 0) { s_max[warp] = mx; s_arg[warp] = arg; }
+  if (lane == 0) { s_max[warp] = a.m; s_sum[warp] = a.s; s_arg[warp] = a.arg; }
   __syncthreads();
   if (warp == 0) {
-    mx = s_max[lane]; arg = s_arg[lane];
+    a.m = s_max[lane]; a.s = s_sum[lane]; a.arg = s_arg[lane];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      const float om = __shfl_xor_sync(0xffffffffu, mx, o);
-      const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
-      if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+      const float om = __shfl_xor_sync(0xffffffffu, a.m, o), os = __shfl_xor_sync(0xffffffffu, a.s, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, a.arg, o);
+      stat_merge(a, om, os, oa);
     }
-    if (lane == 0) { s_max[0] = mx; s_arg[0] = arg; }
-  }
-  __syncthreads();
-  mx = s_max[0];
-  float sum = 0.f;
-  for (int j = threadIdx.x; j < vocab; j += blockDim.x)
-    if (j != mask_id) sum += __expf(row[j] - mx);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  if (lane == 0) s_sum[warp] = sum;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float tot = 0.f;
-    for (int w = 0; w < 32; ++w) tot += s_sum[w];
-    tok[r] = s_arg[0];
-    prob[r] = 1.f / tot;
+    if (lane == 0) {
+      tok[r] = a.arg;
+      prob[r] = 1.f / a.s;                                  // exp(max - max) / sum
+    }
   }
 }
 

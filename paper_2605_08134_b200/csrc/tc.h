@@ -7,7 +7,8 @@
 
 namespace dare {
 
-enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2, EPI_SWIGLU = 3, EPI_F32 = 4 };
+enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2, EPI_SWIGLU = 3, EPI_F32 = 4,
+       EPI_OUT_RES = 5 };   // EPI_OUT plus a residual row (chosen by the launcher when GemmParams::resid is set)
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
