@@ -512,6 +512,8 @@ def run_stack(args):
     out = {"metric": "generated_tokens_per_s", "unit": "tokens/s", "data": "synthetic", "dtype": "bf16",
            "config": {"workload": shape.name, "layers": shape.n_layers, "d_model": d, "d_ff": f, "vocab": V,
                       "prompt": P, "generated": shape.gen_len, "block": lay.block, "batch": B, "threshold": TAU}}
+    n_gen = min(args.gen, shape.gen_len) if args.gen > 0 else shape.gen_len
+    out["config"]["generated"] = n_gen
     for name in ("both", "dense"):
         best = None
         for rep in range(2):
@@ -520,13 +522,13 @@ def run_stack(args):
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             refreshed = 0
-            for step in range(shape.gen_len):
+            for step in range(n_gen):
                 stack.decode_step(toks, P, step // lay.block, step == 0, MODES[name], taus)
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
             best = dt if best is None else min(best, dt)
-        assert not bool((toks == shape.mask_id).any())
-        out[name] = {"tokens_per_s": round(shape.gen_len * B / best, 1), "ms_per_token": round(best / shape.gen_len * 1e3, 3)}
+        assert n_gen < shape.gen_len or not bool((toks == shape.mask_id).any())
+        out[name] = {"tokens_per_s": round(n_gen * B / best, 1), "ms_per_token": round(best / n_gen * 1e3, 3)}
     sel = [stack.layer(l).last_selection(B, lay.seq - P)["count"] for l in range(shape.n_layers)]
     out["value"] = out["both"]["tokens_per_s"]
     out["speedup_of_reuse_path"] = round(out["both"]["tokens_per_s"] / out["dense"]["tokens_per_s"], 3)
@@ -628,6 +630,7 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
     ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
     ap.add_argument("--stack", action="store_true", help="full 32-layer stack generation (config 4) instead")
+    ap.add_argument("--gen", type=int, default=0, help="with --stack: stop after this many generated tokens (profiling)")
     ap.add_argument("--sweep", action="store_true", help="long-context crossover sweep (config 5) instead")
     ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
     args = ap.parse_args()
