@@ -847,14 +847,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem::TOTAL);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::TOTAL);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> attr_one{0}, attr_pair{0};
+  if (cudaError_t e = ensure_dyn_smem(attn_tc_kernel, AttnSmem::TOTAL, attr_one); e != cudaSuccess) return e;
+  if (cudaError_t e = ensure_dyn_smem(attn_pair_kernel, PairSmem::TOTAL, attr_pair); e != cudaSuccess) return e;
   const int tps = (p.g.seq_act + BQ - 1) / BQ;
   // CTAs expected to have work: every row tile (dense) or one row tile per sequence (row-sparse, small refresh set)
   const int expected = p.g.n_heads * p.g.batch * (p.idx ? 1 : tps);

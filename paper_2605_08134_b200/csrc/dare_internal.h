@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libdare (not part of the C ABI).
 #pragma once
 
+#include <atomic>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -30,6 +31,20 @@ struct StepGeom {
   __host__ __device__ int cache_row(int t) const { return (t / seq_act) * max_seq + pos_begin + (t % seq_act); }
   __host__ __device__ int position(int t) const { return pos_begin + (t % seq_act); }
 };
+
+// Raises a kernel's dynamic shared-memory limit once per device: the attribute belongs to the device's context, and a
+// process may hold layers on several devices.  `done` is the caller's bit mask of devices already served.
+template <typename K>
+inline cudaError_t ensure_dyn_smem(K kernel, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
 
 // Launch with programmatic stream serialization (the kernel calls griddepcontrol.wait before touching global data)
 // and, optionally, a thread-block cluster along x and z.

@@ -577,14 +577,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 template <int EPI, int BN, bool PAIR>
 static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
                               int n_tiles, int m_tiles, int splits, cudaStream_t st) {
-  static bool attr_set = false;
+  static std::atomic<unsigned long long> attr_done{0};
   auto kern = gemm_tc_kernel<EPI, BN, PAIR>;
   constexpr int SMEM_TOTAL = Cfg<BN, PAIR>::SMEM_TOTAL;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  if (cudaError_t e = ensure_dyn_smem(kern, SMEM_TOTAL, attr_done); e != cudaSuccess) return e;
   GemmParams q = p;
   q.m_tiles = m_tiles;
   if (PAIR)
