@@ -19,6 +19,10 @@ namespace {
 #define DARE_PAIR_MMA 1
 #endif
 bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0 && pairs_pay(n_tiles, m_tiles, splits); }
+#ifndef DARE_PERSIST
+#define DARE_PERSIST 1
+#endif
+bool use_persist(int n_tiles, int m_tiles, int splits) { return DARE_PERSIST != 0 && persist_pays(n_tiles, m_tiles, splits); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -127,7 +131,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_Q_GEMM, st);
     const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-    if (use_pairs(n_tiles, m_tiles_dense, sp))
+    if (use_persist(n_tiles, m_tiles_dense, sp))
+      e = launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st);
+    else if (use_pairs(n_tiles, m_tiles_dense, sp))
       e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
     else
       e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, sp, st);
@@ -164,7 +170,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     } else {
       prof_mark(L, SLOT_KV_GEMM, st);
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-      if (use_pairs(n_tiles, m_tiles_dense, sp))
+      if (use_persist(n_tiles, m_tiles_dense, sp))
+        e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, st);
+      else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else
         e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, sp, st);
@@ -205,7 +213,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
     } else {
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-      if (use_pairs(n_tiles, m_tiles_dense, sp))
+      if (use_persist(n_tiles, m_tiles_dense, sp))
+        e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, st);
+      else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, sp, st);
