@@ -12,7 +12,12 @@
 //              the row segments are stored; the accumulator is handed back after the last read of tensor memory
 // In the one-tile-per-CTA kernel of gemm_tc.cu a tile costs set-up + pipeline fill + finishing pass + the gap to the
 // next CTA on top of its main loop (about 30 % at these sizes, measured); here the main loops follow one another.
-// Dense row mapping only (no index list), no reduction split, epilogues Q, K/V, OUT, OUT_RES.
+// Gathered launches (the rows of the refresh set, Alg. 1 line 6 / the gathered output projection) add
+//   warps 6-9  A-operand producers: the rows named by the index list are fetched 16 bytes at a time with cp.async into
+//              the swizzled tile layout (eight consecutive lanes on one row: whole 128-byte lines), each warp
+//              arriving on a stage's barrier once its 32 rows of that stage have landed
+// and read the number of row tiles from the device-side count, so no CTA is spent on tiles past the refresh set.
+// No reduction split, epilogues Q, K/V, OUT, OUT_RES.
 #include "layer.h"
 #include "tc.h"
 #include "tc_ptx.cuh"
@@ -30,19 +35,26 @@ constexpr int ACC_OFFSET = STG_OFFSET + 4 * STG_WARP_BYTES;   // partial score s
 constexpr int BAR_OFFSET = ACC_OFFSET + BM * 12;
 static_assert(BAR_OFFSET + 256 + 1024 <= 227 * 1024, "shared memory of one CTA");
 constexpr int SMEM_TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
-constexpr int kThreads = 6 * 32;
+constexpr int kWarpsDense = 6, kWarpsGather = 10;
 
 struct TileGeom {
   int nt, mt, n0, is_b1;
   int t0, rows_valid, a_row, pos0;
   size_t crow0;
 };
-__device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int n_tiles) {
+// n_rows: rows of a gathered launch (the device-side count), unused otherwise
+__device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int n_tiles, bool gather, int n_rows) {
   TileGeom t;
   t.nt = tile % n_tiles;
   t.mt = tile / n_tiles;
   t.is_b1 = t.nt >= p.n_split;
   t.n0 = (t.is_b1 ? t.nt - p.n_split : t.nt) * BN;
+  if (gather) {                      // rows t0 .. of the index list; position and cache row come from the tokens
+    t.t0 = t.mt * BM;
+    t.rows_valid = min(BM, n_rows - t.t0);
+    t.a_row = 0; t.pos0 = 0; t.crow0 = 0;
+    return t;
+  }
   const int b = t.mt / p.tiles_per_seq, tis = t.mt - b * p.tiles_per_seq;
   t.t0 = b * p.seq_act + tis * BM;
   t.rows_valid = min(BM, p.seq_act - tis * BM);
@@ -53,11 +65,11 @@ __device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int
 }
 }  // namespace
 
-template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int EPI, bool GATHER>
+__global__ void __launch_bounds__((GATHER ? kWarpsGather : kWarpsDense) * 32, 1)
 gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                     const __grid_constant__ CUtensorMap tm_b1, const GemmParams p, const int n_tiles,
-                    const int total_tiles) {
+                    const int total_tiles_dense) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + BAR_OFFSET);
@@ -71,7 +83,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 5 : 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
     fence_mbar_init();
     prefetch_tmap(&tm_a);
@@ -89,19 +101,21 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   const int KB = p.K / BK;
+  const int n_rows = GATHER ? min(*p.count, p.m_total) : 0;
+  const int total_tiles = GATHER ? ((n_rows + BM - 1) / BM) * n_tiles : total_tiles_dense;
   if (warp == 0) {
     // ---- producer
     uint32_t it = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const TileGeom t = tile_geom(p, tile, n_tiles);
+      const TileGeom t = tile_geom(p, tile, n_tiles, GATHER, n_rows);
       const CUtensorMap* tm_b = t.is_b1 ? &tm_b1 : &tm_b0;
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int s = it % STAGES;
         mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, p.status);
         if (elect_one()) {
           uint8_t* dst = smem + s * STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[s], (uint32_t)STAGE_BYTES);
-          tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
+          mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(GATHER ? B_BYTES : STAGE_BYTES));
+          if (!GATHER) tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
           tma_load_2d(dst + A_BYTES, tm_b, kb * BK, t.n0, &full_bar[s]);
         }
         __syncwarp();
@@ -131,6 +145,45 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         __syncwarp();
       }
     }
+  } else if (GATHER && warp >= 6) {
+    // ---- A-operand producers of a gathered launch.  One stage of the A tile = 128 rows x 128 bytes; a warp takes 32
+    // rows; one copy instruction covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row.
+    const int gq = warp - 6;
+    constexpr int LAG = STAGES - 2;                              // copy groups in flight per thread
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, it += KB) {
+      const TileGeom t = tile_geom(p, tile, n_tiles, true, n_rows);
+      const int r_own = gq * 32 + lane;                          // the row whose token this lane looks up
+      const int tok_own = r_own < t.rows_valid ? p.idx[t.t0 + r_own] : -1;
+      const uint8_t* src_k[8];
+      uint32_t dst_k[8], bytes_k[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int rw = k * 4 + (lane >> 3), r = gq * 32 + rw, u = lane & 7;
+        const int tok = __shfl_sync(0xffffffffu, tok_own, rw);
+        const int srow = tok < 0 ? 0 : (p.gather_cache_rows ? p.g.cache_row(tok) : tok);
+        src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)srow * p.K * 2 + u * 16;
+        bytes_k[k] = tok >= 0 ? 16u : 0u;                        // rows past the refresh set are zero-filled
+        dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
+      }
+      for (int i = 0; i < KB + LAG; ++i) {
+        if (i < KB) {
+          const uint32_t g = it + i;
+          const int s = g % STAGES;
+          mbar_wait(&empty_bar[s], ((g / STAGES) & 1) ^ 1, p.status);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)i * (BK * 2), bytes_k[k]);
+        }
+        cp_async_commit();                                       // (empty groups at the tail keep the lag uniform)
+        if (i >= LAG) {
+          cp_async_wait<LAG>();                                  // this thread's copies of block i - LAG have landed
+          fence_proxy_async_smem();                              // ... and are visible to the tensor core's reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full_bar[(it + i - LAG) % STAGES]);
+        }
+      }
+    }
   } else {
     // ---- finishing warps: quarter q of the TMEM lanes = rows 32q .. 32q + 31 of every tile
     const int q = warp & 3;
@@ -140,11 +193,17 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     const int half_id = lane >> 4, l16 = lane & 15;
     uint32_t tcount = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
-      const TileGeom t = tile_geom(p, tile, n_tiles);
+      const TileGeom t = tile_geom(p, tile, n_tiles, GATHER, n_rows);
       const uint32_t buf = tcount & 1;
       mbar_wait(&acc_full[buf], (tcount >> 1) & 1, p.status);
       tc_fence_after();
       const uint32_t t_lane = tmem_base + buf * BN + ((uint32_t)(q * 32) << 16);
+      // gathered rows: lane L holds the token of the warp's row L (-1 past the refresh set), lane-to-lane below
+      int tok_own = -1, tok_first = 0;
+      if (GATHER) {
+        if (q * 32 + lane < t.rows_valid) tok_own = p.idx[t.t0 + q * 32 + lane];
+        tok_first = p.idx[t.t0];                         // a row that exists, for the table reads of rows that do not
+      }
       const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !t.is_b1);
       const int head0 = t.n0 / HD;
       const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
@@ -181,24 +240,35 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
           float2 qa[4], qb[4];
           __nv_bfloat162 ra[4], rb[4];
           bool ok[4];
+          int tok_k[4];
+          size_t crow_k[4];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int rr = 2 * (i0 + k) + half_id, r = q * 32 + rr;
             ok[k] = r < t.rows_valid;
             const int rc = ok[k] ? r : 0;                // rows past the end read row 0's tables and are dropped
+            int pos = t.pos0 + rc, tokr = t.t0 + rc;
+            size_t crowr = t.crow0 + rc;
+            if (GATHER) {
+              const int tk = __shfl_sync(0xffffffffu, tok_own, rr);
+              tokr = ok[k] ? tk : tok_first;
+              pos = p.g.position(tokr);
+              crowr = (size_t)p.g.cache_row(tokr);
+            }
+            tok_k[k] = tokr; crow_k[k] = crowr;
             const uint8_t* row = stg + rr * STG_ROW_BYTES;
             const uint32_t off = (uint32_t)((((l16 >> 1) ^ (rr & 7)) << 4) | ((l16 & 1) << 3));
             lo[k] = *reinterpret_cast<const float2*>(row + off);
             hi[k] = *reinterpret_cast<const float2*>(row + 128 + off);
             if (rotate)
-              cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)(t.pos0 + rc) * (HD / 2) + half * 32 + 2 * l16);
+              cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)pos * (HD / 2) + half * 32 + 2 * l16);
             if (EPI == EPI_Q && score_chunk && p.has_prev) {
-              const float* qp = p.q_prev + (t.crow0 + rc) * HD + half * 32 + 2 * l16;
+              const float* qp = p.q_prev + crowr * HD + half * 32 + 2 * l16;
               qa[k] = *reinterpret_cast<const float2*>(qp);
               qb[k] = *reinterpret_cast<const float2*>(qp + HD / 2);
             }
             if (EPI == EPI_OUT_RES) {
-              const __nv_bfloat16* rs = p.resid + (size_t)(t.t0 + rc) * p.ld_resid + t.n0 + c_lo + 2 * l16;
+              const __nv_bfloat16* rs = p.resid + (size_t)tokr * p.ld_resid + t.n0 + c_lo + 2 * l16;
               ra[k] = *reinterpret_cast<const __nv_bfloat162*>(rs);
               rb[k] = *reinterpret_cast<const __nv_bfloat162*>(rs + HD / 2);
             }
@@ -206,8 +276,8 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int rr = 2 * (i0 + k) + half_id, r = q * 32 + rr;
-            const int tok = t.t0 + r;
-            const size_t crow = t.crow0 + r;
+            const int tok = tok_k[k];
+            const size_t crow = crow_k[k];
             float2 vlo = lo[k], vhi = hi[k];
             if (EPI == EPI_Q && score_chunk) {
               // Sec. 3.1 on the un-rotated query of the scoring head: 1 - cos(current, stored); this quarter of the
@@ -253,7 +323,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
               const float2 fa = __bfloat1622float2(ra[k]), fb = __bfloat1622float2(rb[k]);
               vlo.x += fa.x; vlo.y += fa.y; vhi.x += fb.x; vhi.y += fb.y;
             }
-            const size_t orow = p.out_is_cache == 1 ? crow : (size_t)tok;
+            const size_t orow = p.out_is_cache == 1 ? crow : (p.out_is_cache == 2 ? (size_t)(t.t0 + r) : (size_t)tok);
             const __nv_bfloat162 o_lo = __floats2bfloat162_rn(vlo.x, vlo.y), o_hi = __floats2bfloat162_rn(vhi.x, vhi.y);
             __nv_bfloat16* dst = out + orow * p.ld_out + t.n0 + c_lo + 2 * l16;
             *reinterpret_cast<__nv_bfloat162*>(dst) = o_lo;
@@ -275,11 +345,11 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
-template <int EPI>
+template <int EPI, bool GATHER>
 static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
                                   int n_tiles, int m_tiles, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  auto kern = gemm_persist_kernel<EPI>;
+  auto kern = gemm_persist_kernel<EPI, GATHER>;
   if (cudaError_t e = ensure_dyn_smem(kern, SMEM_TOTAL, attr_done); e != cudaSuccess) return e;
   int dev = 0, sms = 0;
   if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
@@ -287,20 +357,28 @@ static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, c
   const int total = n_tiles * m_tiles;
   GemmParams q = p;
   q.m_tiles = m_tiles;
-  return launch_pdl(kern, dim3(total < sms ? total : sms), dim3(kThreads), SMEM_TOTAL, st, 1, a, b0, b1, q, n_tiles, total);
+  return launch_pdl(kern, dim3(total < sms ? total : sms), dim3((GATHER ? kWarpsGather : kWarpsDense) * 32), SMEM_TOTAL, st,
+                    1, a, b0, b1, q, n_tiles, total);
 }
 
-// Dense rows, 256-wide tiles, no reduction split; b0 / b1 are maps with 256-row boxes.
+// 256-wide tiles, no reduction split; b0 / b1 are maps with 256-row boxes.  Gathered launches (idx, count and
+// gather_src set; m_tiles = capacity of the row list in tiles) fetch their A rows by index.
 cudaError_t launch_gemm_persist(int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                                 const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
-  if (p.idx != nullptr || p.count != nullptr || p.gather_src != nullptr || p.b_pair || p.K % BK != 0)
-    return cudaErrorInvalidValue;
+  if (p.b_pair || p.K % BK != 0) return cudaErrorInvalidValue;
+  const bool gather = p.gather_src != nullptr;
+  if (gather != (p.idx != nullptr) || gather != (p.count != nullptr)) return cudaErrorInvalidValue;
   if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
-  if (epi == EPI_Q) return launch_persist<EPI_Q>(a, b0, b1, p, n_tiles, m_tiles, st);
-  if (epi == EPI_KV) return launch_persist<EPI_KV>(a, b0, b1, p, n_tiles, m_tiles, st);
-  if (epi == EPI_OUT) return launch_persist<EPI_OUT>(a, b0, b1, p, n_tiles, m_tiles, st);
-  if (epi == EPI_OUT_RES) return launch_persist<EPI_OUT_RES>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if (gather) {
+    if (epi == EPI_KV) return launch_persist<EPI_KV, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    if (epi == EPI_OUT) return launch_persist<EPI_OUT, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    return cudaErrorInvalidValue;
+  }
+  if (epi == EPI_Q) return launch_persist<EPI_Q, false>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if (epi == EPI_KV) return launch_persist<EPI_KV, false>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if (epi == EPI_OUT) return launch_persist<EPI_OUT, false>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if (epi == EPI_OUT_RES) return launch_persist<EPI_OUT_RES, false>(a, b0, b1, p, n_tiles, m_tiles, st);
   return cudaErrorInvalidValue;
 }
 

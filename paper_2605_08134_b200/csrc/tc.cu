@@ -19,6 +19,9 @@ namespace {
 #define DARE_PAIR_MMA 1
 #endif
 bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0 && pairs_pay(n_tiles, m_tiles, splits); }
+#ifndef DARE_PERSIST_GATHER
+#define DARE_PERSIST_GATHER 1
+#endif
 #ifndef DARE_PERSIST
 #define DARE_PERSIST 1
 #endif
@@ -165,7 +168,11 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
                            pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
-        e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st); ++launches;
+        if (DARE_PERSIST_GATHER && use_persist(n_tiles, m_tiles, 1))
+          e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, st);
+        else
+          e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st);
+        ++launches;
       }
     } else {
       prof_mark(L, SLOT_KV_GEMM, st);
@@ -208,7 +215,11 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     prof_mark(L, SLOT_OUT_GEMM, st);
     if (y_sparse) {
       p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.oc; p.gather_cache_rows = 1;
-      e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, 1, st); ++launches;
+      if (DARE_PERSIST_GATHER && use_persist(n_tiles, (T_ + 127) / 128, 1))
+        e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, st);
+      else
+        e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, 1, st);
+      ++launches;
       if (e != cudaSuccess) return DARE_ERR_CUDA;
       launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
     } else {
