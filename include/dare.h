@@ -173,8 +173,11 @@ const char* dare_kernel_slot_name(int slot);
 /* Diagnostics: when enabled, block (0,0) of each tensor-core kernel of a step writes %globaltimer values (ns) at its
  * phase boundaries into 64 slots of the workspace: slots [8k, 8k+8) belong to kernel k of the step in the order
  * Q projection, K/V projection, attention, output projection; within a kernel: start, set-up done, first operand
- * tile landed, main loop done, epilogue done, ~(earliest block start), latest block end, blocks that ran.  After the
- * 64 slots come 1024 records (SM id, start, end) of the blocks of the Q projection, by linear block index.
+ * tile landed, main loop done, epilogue done, latest block start (attention with two query tiles per CTA only),
+ * latest block end, blocks that ran (a running total over the steps since recording was switched on).  The
+ * persistent projection kernel records start, set-up done, latest end and the count only.  After the 64 slots come
+ * 1024 records (start, accumulator complete, end) of the blocks of the one-tile-per-CTA Q projection, by linear
+ * block index.
  * `out_host` (may be NULL, else room for 64 + 3*1024 values) receives the buffer of the last step (the call
  * synchronises the stream); `enable` switches recording for later steps. */
 dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint64_t* out_host, void* cuda_stream);

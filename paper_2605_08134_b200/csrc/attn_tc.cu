@@ -589,6 +589,14 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     pdl_wait();
     if (p.batch_off[b] + tile * kPairRows >= p.batch_off[b + 1]) return;
   }
+  // diagnostics: [0] first CTA's start, [1] its set-up done, [3] its key loop done, [4] its end; over the CTAs with
+  // work: [5] latest start, [6] latest end, [7] their number
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  unsigned long long t_start = 0;
+  if (p.debug != nullptr && threadIdx.x == 0) {
+    t_start = globaltimer_ns();
+    if (dbg) p.debug[0] = t_start;
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&k_empty[i], 2); mbar_init(&v_empty[i], 2);
@@ -675,6 +683,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   if (active) {
   // stream = query tile: warps 2/3 issue for tile 0/1, softmax warps 4-7 / 8-11; warp 0 brings the key blocks
@@ -754,6 +763,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int j = 0; j < n_blocks; ++j) {
       mbar_wait(&s_full[st], j & 1, p.status);
       tc_fence_after();
+      if (dbg && j == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
       const int n_keys = min(BKV, g.kv_len - j * BKV);
       float v[128];
       tmem_ld_32x32_nowait(tmem_s + lane_addr, v);
@@ -818,6 +828,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       mbar_wait(&o_full[st], (n_blocks - 1) & 1, p.status);
       tc_fence_after();
     }
+    if (dbg && threadIdx.x == 128) p.debug[3] = globaltimer_ns();
     // ---- normalise and store this row (the tensor-memory loads are warp-wide; rows past the tile's end only skip
     // the store)
     {
@@ -842,6 +853,13 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   }  // active
   tc_fence_before();
   __syncthreads();
+  if (p.debug != nullptr && threadIdx.x == 0 && active) {
+    const unsigned long long t_end = globaltimer_ns();
+    if (dbg) p.debug[4] = t_end;
+    atomicMax(&p.debug[5], t_start);
+    atomicMax(&p.debug[6], t_end);
+    atomicAdd(&p.debug[7], 1ull);
+  }
   if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
 }
 
