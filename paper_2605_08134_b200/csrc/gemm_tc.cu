@@ -337,13 +337,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
     // the table reads of this warp's first rows of the finishing pass: in flight for the whole main loop
+    // (a gathering warp asks for its rows' tokens before the table reads below stall on theirs: one round trip, not two)
+    const int r_own = quarter * 32 + lane;                     // the row whose token this lane looks up
+    int tok_own = -1;
+    if (gather && warp < 6 && r_own < rows_valid) tok_own = p.idx[t0 + r_own];
     load_row_batch<EPI, RB, kWarps, BN>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
     if (gather && warp < 6) {
       // One stage of the A tile = 128 rows x 128 bytes (64 k-elements).  A warp takes 32 rows; one of its copy
       // instructions covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row, so every
       // request is a whole 128-byte line.
-      const int r_own = quarter * 32 + lane;                   // the row whose token this lane looks up
-      const int tok_own = r_own < rows_valid ? p.idx[t0 + r_own] : -1;
       const uint8_t* src_k[8];
       uint32_t dst_k[8], bytes_k[8];
 #pragma unroll
