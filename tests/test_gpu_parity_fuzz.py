@@ -33,6 +33,7 @@ CASES = [
     (512, 1, 384, 64),
     (512, 1, 100, 10),
     (1024, 2, 256, 64),
+    (512, 16, 1153, 100),       # 160 row tiles at a short reduction: every projection in the persistent kernel
 ]
 
 
