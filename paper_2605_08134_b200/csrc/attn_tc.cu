@@ -85,7 +85,10 @@ constexpr uint32_t kTmemCols = 512;
 #ifndef DARE_ATTN_PAIR_MIN_SPARSE
 #define DARE_ATTN_PAIR_MIN_SPARSE 1024    // row-sparse launches from this window length on
 #endif
-constexpr float kRescaleStep = 8.f;     // log2 of the growth of the running maximum that triggers a rescale of O
+#ifndef DARE_RESCALE_STEP
+#define DARE_RESCALE_STEP 8.f
+#endif
+constexpr float kRescaleStep = DARE_RESCALE_STEP;     // log2 of the growth of the running maximum that triggers a rescale of O
 
 }  // namespace
 
@@ -536,6 +539,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // brought into shared memory once for both tiles, which halves what a CTA pulls from the L2 per flop (that traffic,
 // 64 KB per key block and tile, is what the kernel above runs into when every SM does it at once).  No merge at the
 // end: a stream owns its rows.
+// Tensor memory per stream: two score buffers of 64 columns and the 128-column O accumulator.  The unit of the
+// pipeline is a half block of 64 keys: S(h) goes to buffer h & 1, and the issuer keeps S(h + 1) in flight while the
+// softmax warps are on S(h) (tcgen05.ld, maximum, exp2, P(h) as bf16 back into the first 32 columns of the buffer),
+// then issues P(h) V and, behind it in issue order, S(h + 2) into the buffer P(h) was read from.  With one score
+// buffer per stream the softmax warps idled through their own stream's two products of every block (measured: the
+// special-function unit is only 13 % of the kernel's time; the chain S -> softmax -> P V -> S was the rest).
+// The softmax warps can therefore be up to two P V products ahead of the tensor core; they wait for a product only
+// to rescale O or to read it out, on one of two barriers per stream (product h signals barrier h & 1) so that a
+// parity wait never has to tell more than two consecutive phases apart.
 namespace {
 struct PairSmem {
   static constexpr int Q_BYTES = BQ * HD * 2;
@@ -548,6 +560,7 @@ struct PairSmem {
 };
 static_assert(PairSmem::TOTAL <= 232448, "shared memory");
 constexpr int kPairRows = 2 * BQ;
+constexpr int kHalf = BKV / 2;     // keys per score buffer
 }  // namespace
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -561,10 +574,10 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   uint64_t* k_empty = bars + 2;     // [2]: one arrival per stream
   uint64_t* v_full = bars + 4;      // [2]
   uint64_t* v_empty = bars + 6;     // [2]: one arrival per stream
-  uint64_t* s_full = bars + 8;      // [2 streams]
-  uint64_t* p_full = bars + 10;     // [2 streams]
-  uint64_t* o_full = bars + 12;     // [2 streams]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+  uint64_t* s_full = bars + 8;      // [2 streams][2 score buffers]
+  uint64_t* p_full = bars + 12;     // [2 streams][2 score buffers]
+  uint64_t* o_full = bars + 16;     // [2 streams][2]: product h signals o_full[stream][h & 1]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const StepGeom& g = p.g;
@@ -600,8 +613,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&k_empty[i], 2); mbar_init(&v_empty[i], 2);
-      mbar_init(&s_full[i], 1); mbar_init(&o_full[i], 1);
-      mbar_init(&p_full[i], kSoftmaxThreads / 64);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&s_full[2 * i + b], 1); mbar_init(&p_full[2 * i + b], kSoftmaxThreads / 64); mbar_init(&o_full[2 * i + b], 1);
+      }
     }
     fence_mbar_init();
     prefetch_tmap(&tm_k);
@@ -626,6 +640,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     rows_all = min(kPairRows, g.seq_act - tile * kPairRows);
   }
   const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  const int n_half = (g.kv_len + kHalf - 1) / kHalf;   // half blocks: the unit of the score / softmax / P V pipeline
   const int kv_row0 = b * g.max_seq;
   auto load_kv = [&](int i) {        // one thread: key block i into ring slot i & 1
     const int slot = i & 1, row = kv_row0 + i * BKV;
@@ -702,7 +717,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       __syncwarp();
     }
   } else if (warp == 2 || warp == 3) {
-    constexpr uint32_t idesc_qk = idesc_bf16(BQ, BKV, false);
+    constexpr uint32_t idesc_qk = idesc_bf16(BQ, kHalf, false);
     constexpr uint32_t idesc_pv = idesc_bf16(BQ, HD, true);
     const uint64_t q_desc = smem_desc_k_sw128(smem_u32(smem + S::Q_OFF + st * S::Q_BYTES));
     const uint64_t k_desc0 = smem_desc_k_sw128(smem_u32(smem + S::K_OFF));
@@ -720,37 +735,41 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         __syncwarp();
       }
     } else {
-      auto issue_qk = [&](int i) {
-        const int slot = i & 1;
-        mbar_wait(&k_full[slot], (i >> 1) & 1, p.status);
+      // Half blocks of 64 keys, h = 0 .. n_half - 1, scores of half h into buffer h & 1: S(h + 1) is computed while
+      // the softmax warps are on S(h), so they go from one half to the next without waiting for the tensor core.
+      auto issue_qk = [&](int hf) {
+        const int i = hf >> 1, slot = i & 1, hb = hf & 1;
+        if (hb == 0) mbar_wait(&k_full[slot], (i >> 1) & 1, p.status);   // (the second half: same block, already here)
         tc_fence_after();
         if (elect_one()) {
-          const uint64_t k_desc = k_desc0 + (uint64_t)(slot * (S::KV_BYTES >> 4));
+          const uint64_t k_desc = k_desc0 + (uint64_t)(slot * (S::KV_BYTES >> 4)) + (uint64_t)((hb * kHalf * 128) >> 4);
 #pragma unroll
           for (int kk = 0; kk < HD / 16; ++kk)
-            umma_ss(tmem_s, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
+            umma_ss(tmem_s + hb * kHalf, q_desc + (((kk >> 2) * (BQ * 128) + (kk & 3) * 32) >> 4),
                     k_desc + (((kk >> 2) * (BKV * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk != 0 ? 1u : 0u);
-          umma_commit(&s_full[st]);
-          umma_commit(&k_empty[slot]);
+          umma_commit(&s_full[2 * st + hb]);
+          if (hb == 1 || hf == n_half - 1) umma_commit(&k_empty[slot]);   // the block's keys are done with
         }
         __syncwarp();
       };
-      if (n_blocks > 0) issue_qk(0);
-      for (int i = 0; i < n_blocks; ++i) {
-        const int slot = i & 1;
-        mbar_wait(&p_full[st], i & 1, p.status);      // P(i) has replaced S(i) in tensor memory
-        mbar_wait(&v_full[slot], (i >> 1) & 1, p.status);
+      if (n_half > 0) issue_qk(0);
+      if (n_half > 1) issue_qk(1);
+      for (int hf = 0; hf < n_half; ++hf) {
+        const int i = hf >> 1, slot = i & 1, hb = hf & 1;
+        mbar_wait(&p_full[2 * st + hb], (hf >> 1) & 1, p.status);   // P(hf) has replaced S(hf) in tensor memory
+        if (hb == 0) mbar_wait(&v_full[slot], (i >> 1) & 1, p.status);
         tc_fence_after();
         if (elect_one()) {
           const uint64_t v_desc = v_desc0 + (uint64_t)(slot * (S::KV_BYTES >> 4));
 #pragma unroll
-          for (int ks = 0; ks < BKV / 16; ++ks)
-            umma_ts(tmem_o, tmem_s + ks * 8, v_desc + ((ks * (16 * 128)) >> 4), idesc_pv, (i | ks) != 0 ? 1u : 0u);
-          umma_commit(&o_full[st]);
-          umma_commit(&v_empty[slot]);
+          for (int k4 = 0; k4 < kHalf / 16; ++k4)
+            umma_ts(tmem_o, tmem_s + hb * kHalf + k4 * 8, v_desc + (((hb * (kHalf / 16) + k4) * (16 * 128)) >> 4), idesc_pv,
+                    (hf | k4) != 0 ? 1u : 0u);
+          umma_commit(&o_full[2 * st + hb]);
+          if (hb == 1 || hf == n_half - 1) umma_commit(&v_empty[slot]);
         }
         __syncwarp();
-        if (i + 1 < n_blocks) issue_qk(i + 1);        // in issue order behind the product that reads P(i)
+        if (hf + 2 < n_half) issue_qk(hf + 2);          // in issue order behind the product that reads P(hf)
       }
     }
   } else if (warp >= 4 && st_active) {
@@ -760,39 +779,42 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)HD) * 1.4426950408889634f;
     float m = -INFINITY, l = 0.f;
-    for (int j = 0; j < n_blocks; ++j) {
-      mbar_wait(&s_full[st], j & 1, p.status);
+    for (int hf = 0; hf < n_half; ++hf) {
+      const uint32_t sbuf = tmem_s + (hf & 1) * kHalf + lane_addr;      // scores of half block hf, then its P
+      mbar_wait(&s_full[2 * st + (hf & 1)], (hf >> 1) & 1, p.status);
       tc_fence_after();
-      if (dbg && j == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
-      const int n_keys = min(BKV, g.kv_len - j * BKV);
-      float v[128];
-      tmem_ld_32x32_nowait(tmem_s + lane_addr, v);
-      tmem_ld_32x32_nowait(tmem_s + lane_addr + 32, v + 32);
-      tmem_ld_32x32_nowait(tmem_s + lane_addr + 64, v + 64);
-      tmem_ld_32x32_nowait(tmem_s + lane_addr + 96, v + 96);
+
+      if (dbg && hf == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
+      const int n_keys = min(kHalf, g.kv_len - hf * kHalf);
+      float v[kHalf];
+      tmem_ld_32x32_nowait(sbuf, v);
+      tmem_ld_32x32_nowait(sbuf + 32, v + 32);
       tmem_ld_wait();
-      if (n_keys < BKV) {
+      if (n_keys < kHalf) {
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < kHalf; ++i)
           if (i >= n_keys) v[i] = -INFINITY;
       }
       float mx4[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(v[k], v[4 + k]);
 #pragma unroll
-      for (int i = 8; i < 128; i += 8) {
+      for (int i = 8; i < kHalf; i += 8) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) mx4[k] = fmax3(mx4[k], v[i + k], v[i + 4 + k]);
       }
       const float m_new = fmax3(m, fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      if (j == 0) {
+      if (hf == 0) {
         m = m_new;
       } else {
         const bool grow = (m_new - m) * c > kRescaleStep;
         if (__any_sync(0xffffffffu, grow)) {
           const float alpha = grow ? fast_exp2((m - m_new) * c) : 1.f;
           if (grow) { m = m_new; l *= alpha; }
-          mbar_wait(&o_full[st], (j - 1) & 1, p.status);
+          // P(hf - 1) V has been added.  (The softmax warps may be two products ahead of the tensor core, and a
+          // parity wait tells apart only two consecutive phases: hence one barrier per parity of hf, each of which
+          // these warps are at most one phase behind.)
+          mbar_wait(&o_full[2 * st + ((hf - 1) & 1)], ((hf - 1) >> 1) & 1, p.status);
           tc_fence_after();
 #pragma unroll 1
           for (int ch = 0; ch < 4; ++ch) {
@@ -806,9 +828,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       }
       const float2 c2 = make_float2(c, c), nmc2 = make_float2(-m * c, -m * c);
       float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-      float pk[64];
+      float pk[kHalf / 2];
 #pragma unroll
-      for (int i = 0; i < 128; i += 2) {
+      for (int i = 0; i < kHalf; i += 2) {
         float2 e = __ffma2_rn(make_float2(v[i], v[i + 1]), c2, nmc2);
         e.x = fast_exp2(e.x);
         e.y = fast_exp2(e.y);
@@ -816,18 +838,16 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
         pk[i >> 1] = __uint_as_float(*reinterpret_cast<uint32_t*>(&h2));
       }
-      tmem_st_32x32_nowait(tmem_s + lane_addr, pk);
-      tmem_st_32x32_nowait(tmem_s + lane_addr + 32, pk + 32);
+      tmem_st_32x32_nowait(sbuf, pk);
       tmem_st_wait();
       l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[st]);
+      if (lane == 0) mbar_arrive(&p_full[2 * st + (hf & 1)]);
     }
-    if (n_blocks > 0) {
-      mbar_wait(&o_full[st], (n_blocks - 1) & 1, p.status);
-      tc_fence_after();
-    }
+    for (int hh = max(0, n_half - 2); hh < n_half; ++hh)       // the last two products
+      mbar_wait(&o_full[2 * st + (hh & 1)], (hh >> 1) & 1, p.status);
+    tc_fence_after();
     if (dbg && threadIdx.x == 128) p.debug[3] = globaltimer_ns();
     // ---- normalise and store this row (the tensor-memory loads are warp-wide; rows past the tile's end only skip
     // the store)

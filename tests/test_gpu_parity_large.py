@@ -99,3 +99,32 @@ def test_config5_long_context_one_sequence(dare, frac, pattern, mode):
     parity.assert_close("o_cache", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
     assert g.status() == 0
     g.close()
+
+
+def test_long_context_attention_repeats_bit_identically(dare):
+    """Batch 4 x 4096, two steps (dense, then K/V reuse at 50 % clustered) on three fresh handles: the caches must be
+    bit-identical from run to run.  The softmax warps of the two-tile attention kernel run up to two P V products
+    ahead of the tensor core there; a wait that mistook one phase of a barrier for another showed up as outputs that
+    varied between runs."""
+    import torch
+    shape = wl.LLADA_LONG
+    w_t, _ = _weights_gpu(shape, 55, torch)
+
+    def run():
+        hs = wl.HiddenStream(shape)
+        g = dare.Layer(shape, w_t)
+        g.step(parity.to_device(hs.first(), shape), 1, 0.1)
+        c0 = g.read_caches(shape.batch, shape.seq)
+        ch = wl.clustered_positions(hs.rng, shape, 9, shape.seq // 2, 0)
+        g.step(parity.to_device(hs.advance(ch), shape), 1, 0.1)
+        c1 = g.read_caches(shape.batch, shape.seq)
+        assert g.status() == 0
+        g.close()
+        return c0, c1
+
+    a0, a1 = run()
+    for _ in range(2):
+        b0, b1 = run()
+        for name in ("k", "v", "o"):
+            np.testing.assert_array_equal(a0[name], b0[name])
+            np.testing.assert_array_equal(a1[name], b1[name])
