@@ -238,7 +238,7 @@ void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float
                     unsigned long long* dbg) {
   if (rows <= 0) return;
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-    constexpr int ROWS = 4;
+    constexpr int ROWS = 2;        // measured at 16384 rows of 4096: 56 us (1 row per CTA: 65, 4: 65, 8: 93)
     if (rows > 2048 && d % 8 == 0 && d / 8 <= 512 && dbg == nullptr) {
       launch_pdl(rmsnorm_stream_kernel<ROWS>, dim3((rows + ROWS - 1) / ROWS), dim3(256), 0, st, 1, x, gain, xn, rows, d,
                  eps);
