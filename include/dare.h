@@ -127,6 +127,16 @@ dare_status_t dare_layer_step(dare_layer_t* layer, const void* x, int batch, int
 dare_status_t dare_layer_step_host(dare_layer_t* layer, const void* x_host, int batch, int seq_act, int pos_begin,
                                    int mode, float threshold, void* y_host, void* cuda_stream);
 
+/* The same, enqueue only: the copy in runs on a copy stream of the layer as soon as the staging buffer is free (the
+ * previous step of this layer has consumed it), the step on `cuda_stream` behind it, the copy out on a second copy
+ * stream behind the step; nothing else on `cuda_stream` waits for the copy out.  Steps of several layers issued this
+ * way overlap one layer's copies with another's kernels (full-duplex PCIe).  x_host must stay valid and y_host is
+ * defined only after dare_layer_wait_host(layer), which blocks the calling thread until the layer's last copy out
+ * has landed.  The copy streams and events are created on first use and live as long as the handle. */
+dare_status_t dare_layer_step_host_async(dare_layer_t* layer, const void* x_host, int batch, int seq_act, int pos_begin,
+                                         int mode, float threshold, void* y_host, void* cuda_stream);
+dare_status_t dare_layer_wait_host(dare_layer_t* layer);
+
 /* Forgets every cached activation: the next step is dense and must start at position 0.  Host-only. */
 dare_status_t dare_layer_reset(dare_layer_t* layer);
 

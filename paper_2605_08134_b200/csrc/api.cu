@@ -240,6 +240,7 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->prof_n = 0;
   L->prof_ev_ready = false;
   L->debug_on = false;
+  L->host_async_ready = false;
   memset(&L->last_geom, 0, sizeof(L->last_geom));
   carve(cfg, use_tc, (char*)workspace, &L->buf);
   L->workspace = workspace;
@@ -291,6 +292,46 @@ dare_status_t dare_layer_step_host(dare_layer_t* L, const void* x_host, int batc
   return DARE_OK;
 }
 
+dare_status_t dare_layer_step_host_async(dare_layer_t* L, const void* x_host, int batch, int seq_act, int pos_begin,
+                                         int mode, float threshold, void* y_host, void* cuda_stream) {
+  dare_status_t s = validate_step(L, x_host, batch, seq_act, pos_begin, mode, threshold, y_host);
+  if (s != DARE_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (!L->host_async_ready) {
+    CUDA_TRY(cudaStreamCreateWithFlags(&L->copy_in, cudaStreamNonBlocking));
+    CUDA_TRY(cudaStreamCreateWithFlags(&L->copy_out, cudaStreamNonBlocking));
+    CUDA_TRY(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&L->ev_consumed, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
+    // (never-recorded events: waiting on them returns at once, which is right for the first step)
+    L->host_async_ready = true;
+  }
+  const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
+  const size_t bytes = (size_t)batch * seq_act * L->cfg.d_model * e;
+  // copy in: once the layer's previous step has read the staging buffer
+  CUDA_TRY(cudaStreamWaitEvent(L->copy_in, L->ev_consumed, 0));
+  CUDA_TRY(cudaMemcpyAsync(L->buf.x_stage, x_host, bytes, cudaMemcpyHostToDevice, L->copy_in));
+  CUDA_TRY(cudaEventRecord(L->ev_in, L->copy_in));
+  // the step: behind the copy in, and behind the previous copy out of the output staging buffer
+  CUDA_TRY(cudaStreamWaitEvent(st, L->ev_in, 0));
+  CUDA_TRY(cudaStreamWaitEvent(st, L->ev_out, 0));
+  s = enqueue_step(L, L->buf.x_stage, batch, seq_act, pos_begin, mode, threshold, L->buf.y_stage, st);
+  if (s != DARE_OK) return s;
+  CUDA_TRY(cudaEventRecord(L->ev_consumed, st));
+  // copy out: behind the step, on its own stream
+  CUDA_TRY(cudaStreamWaitEvent(L->copy_out, L->ev_consumed, 0));
+  CUDA_TRY(cudaMemcpyAsync(y_host, L->buf.y_stage, bytes, cudaMemcpyDeviceToHost, L->copy_out));
+  CUDA_TRY(cudaEventRecord(L->ev_out, L->copy_out));
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_wait_host(dare_layer_t* L) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (L->host_async_ready) CUDA_TRY(cudaEventSynchronize(L->ev_out));
+  return DARE_OK;
+}
+
 dare_status_t dare_layer_reset(dare_layer_t* L) {
   dare_status_t s = check_handle(L);
   if (s != DARE_OK) return s;
@@ -307,6 +348,12 @@ dare_status_t dare_layer_destroy(dare_layer_t* L) {
   if (L->use_tc) tc_destroy(L);
   if (L->prof_ev_ready)
     for (int i = 0; i <= kMaxMarks; ++i) cudaEventDestroy(L->prof_ev[i]);
+  if (L->host_async_ready) {
+    cudaStreamSynchronize(L->copy_in);
+    cudaStreamSynchronize(L->copy_out);
+    cudaEventDestroy(L->ev_in); cudaEventDestroy(L->ev_consumed); cudaEventDestroy(L->ev_out);
+    cudaStreamDestroy(L->copy_in); cudaStreamDestroy(L->copy_out);
+  }
   L->magic = 0;
   delete L;
   return DARE_OK;

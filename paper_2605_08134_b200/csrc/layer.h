@@ -58,6 +58,10 @@ struct dare_layer {
   cudaEvent_t prof_ev[dare::kMaxMarks + 1];
   bool prof_ev_ready;
   bool debug_on;
+  // asynchronous host-buffer steps: copy streams and the events that order staging-buffer reuse (created on first use)
+  bool host_async_ready;
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_in, ev_consumed, ev_out;
 };
 
 namespace dare {

@@ -64,6 +64,8 @@ def _load():
         "dare_layer_create": (C.c_int, [C.POINTER(LayerConfig), C.POINTER(LayerWeights), vp, sz, C.POINTER(vp)]),
         "dare_layer_step": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
         "dare_layer_step_host": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
+        "dare_layer_step_host_async": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
+        "dare_layer_wait_host": (C.c_int, [vp]),
         "dare_layer_reset": (C.c_int, [vp]),
         "dare_layer_destroy": (C.c_int, [vp]),
         "dare_layer_status": (C.c_int, [vp, vp]),
@@ -134,6 +136,15 @@ def dare_layer_step(handle, x_ptr, batch, seq_act, pos_begin, mode, threshold, y
 
 def dare_layer_step_host(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr, stream=0) -> int:
     return _lib.dare_layer_step_host(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr, stream)
+
+
+def dare_layer_step_host_async(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr, stream=0) -> int:
+    return _lib.dare_layer_step_host_async(handle, x_host_ptr, batch, seq_act, pos_begin, mode, threshold, y_host_ptr,
+                                           stream)
+
+
+def dare_layer_wait_host(handle) -> int:
+    return _lib.dare_layer_wait_host(handle)
 
 
 def dare_layer_reset(handle) -> int:
@@ -315,6 +326,18 @@ class Layer:
         if st != OK:
             raise DareError(st, "dare_layer_step_host")
         return y_host
+
+    def step_host_async(self, x_host, mode, threshold, y_host, pos_begin=0):
+        """Enqueue only: y_host is defined after wait_host(); x_host must stay valid until then."""
+        st = dare_layer_step_host_async(self.handle, x_host.data_ptr(), x_host.shape[0], x_host.shape[1], pos_begin, mode,
+                                        threshold, y_host.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_step_host_async")
+
+    def wait_host(self):
+        st = dare_layer_wait_host(self.handle)
+        if st != OK:
+            raise DareError(st, "dare_layer_wait_host")
 
     def reset(self):
         st = dare_layer_reset(self.handle)

@@ -169,3 +169,31 @@ def test_step_host_matches_device_step(dare):
         torch.cuda.synchronize()
         assert torch.equal(ya.cpu(), yh)
     a.close(); b.close()
+
+
+def test_step_host_async_pipeline_matches_device_steps(dare):
+    """Four layers stepped through the enqueue-only host-buffer entry point, three rounds without waiting in between
+    (copies of one layer overlap kernels of another; a layer's staging buffers are reused from round to round), against
+    the same steps with device buffers: bit-identical outputs."""
+    import torch
+    shape = wl.TINY_F32
+    w, x0, x1, _ = wl.two_step_case(shape, 26)
+    n = 4
+    ref = [dare.Layer(shape, w) for _ in range(n)]
+    pipe = [dare.Layer(shape, w) for _ in range(n)]
+    xs = [x0, x1, x0]
+    xh = [[torch.from_numpy(np.ascontiguousarray(x + 0.01 * i)).pin_memory() for x in xs] for i in range(n)]
+    yh = [[torch.empty_like(xh[i][r]).pin_memory() for r in range(len(xs))] for i in range(n)]
+    for r in range(len(xs)):
+        for i in range(n):
+            pipe[i].step_host_async(xh[i][r], 3, 0.1, yh[i][r])
+    for i in range(n):
+        pipe[i].wait_host()
+    for r in range(len(xs)):
+        for i in range(n):
+            ya = ref[i].step(xh[i][r].cuda(), 3, 0.1)
+            torch.cuda.synchronize()
+            assert torch.equal(ya.cpu(), yh[i][r]), (r, i)
+    for l in ref + pipe:
+        assert l.status() == 0
+        l.close()
