@@ -599,6 +599,15 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
   if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
   if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
+  if (pair && bn == 128) {
+    // narrow pair tiles (256 rows x 128 columns per pair; b0 / b1 with 64-row boxes): twice the CTAs of the wide ones
+    // for launches of two row tiles, whose main loops are bound by what one SM can pull from the L2
+    if (p.gather_src != nullptr || p.count != nullptr || p.b_pair) return cudaErrorInvalidValue;
+    if (epi == EPI_Q) return launch_one<EPI_Q, 128, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_OUT) return launch_one<EPI_OUT, 128, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    if (epi == EPI_OUT_RES) return launch_one<EPI_OUT_RES, 128, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st);
+    return cudaErrorInvalidValue;
+  }
   if (pair) {
     if (bn != 256 || p.gather_src != nullptr || p.count != nullptr || (p.b_pair != 0) != (epi == EPI_SWIGLU))
       return cudaErrorInvalidValue;

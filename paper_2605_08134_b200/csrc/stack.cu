@@ -26,7 +26,7 @@ constexpr int kMaxCand = 128;       // candidates per decoding step: batch * blo
 
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
-struct BlockMaps { CUtensorMap w_gate, w_up, w_down, w_down128; };   // w_down: 256-row boxes, the others 128
+struct BlockMaps { CUtensorMap w_gate, w_up, w_down, w_down128, w_down64; };   // w_down: 256-row boxes, w_down64: 64, the others 128
 
 // x[t, :] = emb[tokens[b, pos_begin + i], :]   (t = b*seq_act + i)
 __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ tokens, int seq_total, int seq_act,
@@ -283,9 +283,14 @@ dare_status_t forward(dare_stack* S, const int* tokens, int batch, int seq_total
       const int n_tiles = d / 256;
       const int sp = pick_splits(n_tiles * m_tiles, f / 64);
       const bool pair = pairs_pay(n_tiles, m_tiles, sp);
-      const CUtensorMap& wd = pair ? S->maps[l].w_down128 : S->maps[l].w_down;
-      if (launch_gemm_tc(EPI_OUT, 256, S->a_act, wd, wd, p, n_tiles, m_tiles, sp, st, pair ? 1 : 0) != cudaSuccess)
-        return DARE_ERR_CUDA;
+      if (narrow_pairs_pay(d, m_tiles, f / 64)) {
+        if (launch_gemm_tc(EPI_OUT, 128, S->a_act, S->maps[l].w_down64, S->maps[l].w_down64, p, d / 128, m_tiles, 2, st,
+                           1) != cudaSuccess) return DARE_ERR_CUDA;
+      } else {
+        const CUtensorMap& wd = pair ? S->maps[l].w_down128 : S->maps[l].w_down;
+        if (launch_gemm_tc(EPI_OUT, 256, S->a_act, wd, wd, p, n_tiles, m_tiles, sp, st, pair ? 1 : 0) != cudaSuccess)
+          return DARE_ERR_CUDA;
+      }
     }
   }
   launch_rmsnorm<bf16>(B.xa, S->final_gain, B.hidden, T_, d, lc.rms_eps, st);
@@ -343,7 +348,8 @@ dare_status_t dare_stack_create(const dare_stack_config_t* cfg, const dare_stack
     S->blocks.push_back(bw);
     BlockMaps m;
     if (!make_map(&m.w_gate, bw.w_gate, f, d, 128) || !make_map(&m.w_up, bw.w_up, f, d, 128) ||
-        !make_map(&m.w_down, bw.w_down, d, f, 256) || !make_map(&m.w_down128, bw.w_down, d, f, 128))
+        !make_map(&m.w_down, bw.w_down, d, f, 256) || !make_map(&m.w_down128, bw.w_down, d, f, 128) ||
+        !make_map(&m.w_down64, bw.w_down, d, f, 64))
       st = DARE_ERR_CUDA;
     S->maps.push_back(m);
   }

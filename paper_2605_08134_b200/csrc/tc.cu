@@ -10,6 +10,7 @@ struct TcState {
   CUtensorMap a_xn, a_oc;                  // A operands, box 64 x 128 rows
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 256 rows
   CUtensorMap w_k128, w_v128, w_q128, w_o128;   // weights, box 64 x 128 rows
+  CUtensorMap w_q64, w_o64;                // weights, box 64 x 64 rows (narrow pair tiles)
   CUtensorMap kc64, vc64;                  // K/V caches as attention operands, box 64 x 128 rows (keys)
 };
 
@@ -19,6 +20,9 @@ namespace {
 #define DARE_PAIR_MMA 1
 #endif
 bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0 && pairs_pay(n_tiles, m_tiles, splits); }
+#ifndef DARE_NARROW_PAIRS
+#define DARE_NARROW_PAIRS 1
+#endif
 #ifndef DARE_PERSIST_GATHER
 #define DARE_PERSIST_GATHER 1
 #endif
@@ -81,7 +85,8 @@ dare_status_t tc_create(dare_layer* L) {
             make_map(&s->w_k, L->w.w_k, d, d, 256) && make_map(&s->w_v, L->w.w_v, d, d, 256) &&
             make_map(&s->w_o, L->w.w_o, d, d, 256) && make_map(&s->w_k128, L->w.w_k, d, d, 128) &&
             make_map(&s->w_v128, L->w.w_v, d, d, 128) && make_map(&s->w_q128, L->w.w_q, d, d, 128) &&
-            make_map(&s->w_o128, L->w.w_o, d, d, 128) && make_map(&s->kc64, L->buf.kc, Tm, d, 128) &&
+            make_map(&s->w_o128, L->w.w_o, d, d, 128) && make_map(&s->w_q64, L->w.w_q, d, d, 64) &&
+            make_map(&s->w_o64, L->w.w_o, d, d, 64) && make_map(&s->kc64, L->buf.kc, Tm, d, 128) &&
             make_map(&s->vc64, L->buf.vc, Tm, d, 128);
   if (!ok) { delete s; return DARE_ERR_CUDA; }
   L->tc = s;
@@ -134,7 +139,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_Q_GEMM, st);
     const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-    if (use_persist(n_tiles, m_tiles_dense, sp))
+    if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
+      e = launch_gemm_tc(EPI_Q, 128, S.a_xn, S.w_q64, S.w_q64, p, d / 128, m_tiles_dense, 2, st, 1);
+    else if (use_persist(n_tiles, m_tiles_dense, sp))
       e = launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st);
     else if (use_pairs(n_tiles, m_tiles_dense, sp))
       e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
@@ -224,7 +231,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
     } else {
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-      if (use_persist(n_tiles, m_tiles_dense, sp))
+      if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
+        e = launch_gemm_tc(EPI_OUT, 128, S.a_oc, S.w_o64, S.w_o64, p, d / 128, m_tiles_dense, 2, st, 1);
+      else if (use_persist(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, st);
       else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, sp, st, 1);

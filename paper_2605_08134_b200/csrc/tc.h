@@ -72,6 +72,12 @@ inline bool pairs_pay(int n_tiles, int m_tiles, int splits) {
   return m_tiles >= 2 && (ctas <= 160 || m_tiles <= 4);
 }
 
+// ... and with exactly two row tiles (a window of up to 256 rows) the narrow pair tiles (256 x 128 per pair, reduction
+// split in two) put twice as many CTAs on the launch: d/128 column tiles x 2 x 2 CTAs, if that still is one wave.
+inline bool narrow_pairs_pay(int d_out, int m_tiles, int kblocks) {
+  return m_tiles == 2 && kblocks >= 4 && (d_out / 128) * 2 * 2 <= 160;
+}
+
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                            const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair = 0);
 

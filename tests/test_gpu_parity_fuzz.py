@@ -34,6 +34,8 @@ CASES = [
     (512, 1, 100, 10),
     (1024, 2, 256, 64),
     (512, 16, 1153, 100),       # 160 row tiles at a short reduction: every projection in the persistent kernel
+    (1024, 1, 250, 60),         # two row tiles: narrow MMA-pair tiles (one sequence, ragged)
+    (512, 2, 128, 32),          # ... one row tile per sequence
 ]
 
 
