@@ -36,6 +36,9 @@ CASES = [
     (512, 16, 1153, 100),       # 160 row tiles at a short reduction: every projection in the persistent kernel
     (1024, 1, 250, 60),         # two row tiles: narrow MMA-pair tiles (one sequence, ragged)
     (512, 2, 128, 32),          # ... one row tile per sequence
+    (4096, 1, 250, 100),        # the full layer width at two, two and three row tiles: narrow pairs, padding tile
+    (4096, 2, 128, 16),
+    (4096, 3, 120, 20),
 ]
 
 
