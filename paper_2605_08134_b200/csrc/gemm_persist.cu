@@ -17,6 +17,13 @@
 //              the swizzled tile layout (eight consecutive lanes on one row: whole 128-byte lines), each warp
 //              arriving on a stage's barrier once its 32 rows of that stage have landed
 // and read the number of row tiles from the device-side count, so no CTA is spent on tiles past the refresh set.
+// PAIR (dense launches): the CTAs of a cluster of two take row tiles 2i and 2i + 1 of the same column tile as one
+// M = 256 tcgen05.mma.cta_group::2 issued by the even CTA; each keeps its own 128 rows of A and 128 of the W tile's
+// 256 rows (32 KB per stage, six stages), which takes a third off what an SM pulls from the L2 per flop: the
+// one-CTA form runs its main loop at 667 cycles per 64 k-elements against 512 of tensor work, bound by that
+// traffic (ncu: tensor pipe 87 % active).  Both CTAs' TMA loads complete on the even CTA's barriers, stages and
+// accumulators are released to both by one commit each, and the finishing warps of both CTAs hand an accumulator
+// back by arriving on the even CTA's barrier.
 // No reduction split, epilogues Q, K/V, OUT, OUT_RES.
 #include "layer.h"
 #include "tc.h"
@@ -27,9 +34,16 @@ namespace dare {
 using namespace ptx;
 
 namespace {
-constexpr int BM = 128, BN = 256, BK = 64, HD = 128, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int STG_OFFSET = STAGES * STAGE_BYTES;     // finishing warps' staging: 4 x (32 rows x 64 fp32)
+constexpr int BM = 128, BN = 256, BK = 64, HD = 128;
+constexpr int A_BYTES = BM * BK * 2;
+template <bool PAIR>
+struct Ring {
+  static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;    // this CTA's part of the W tile
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = PAIR ? 6 : 4;
+};
+constexpr int STG_OFFSET = Ring<false>::STAGES * Ring<false>::STAGE_BYTES;   // finishing warps' staging: 4 x (32 rows x 64 fp32)
+static_assert(Ring<true>::STAGES * Ring<true>::STAGE_BYTES == STG_OFFSET, "both rings end where the staging begins");
 constexpr int STG_ROW_BYTES = 64 * 4, STG_WARP_BYTES = 32 * STG_ROW_BYTES;
 constexpr int ACC_OFFSET = STG_OFFSET + 4 * STG_WARP_BYTES;   // partial score sums: [128 rows][3] fp32
 constexpr int BAR_OFFSET = ACC_OFFSET + BM * 12;
@@ -65,11 +79,13 @@ __device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int
 }
 }  // namespace
 
-template <int EPI, bool GATHER>
+template <int EPI, bool GATHER, bool PAIR>
 __global__ void __launch_bounds__((GATHER ? kWarpsGather : kWarpsDense) * 32, 1)
 gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                     const __grid_constant__ CUtensorMap tm_b1, const GemmParams p, const int n_tiles,
                     const int total_tiles_dense) {
+  static_assert(!(GATHER && PAIR), "gathered launches use single-CTA tiles");
+  constexpr int STAGES = Ring<PAIR>::STAGES, STAGE_BYTES = Ring<PAIR>::STAGE_BYTES, B_BYTES = Ring<PAIR>::B_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + BAR_OFFSET);
@@ -81,20 +97,34 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const bool dbg = p.debug != nullptr && blockIdx.x == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
+  // PAIR: place in the MMA pair (cluster of two along x); place 0 issues the MMAs and owns the barriers that count
+  const int pr = PAIR ? (int)cluster_ctarank() : 0;
+  // the walk over the launch's work: single tiles, or pairs of row tiles taken by the two CTAs of a cluster
+  const int walker = PAIR ? (int)blockIdx.x / 2 : (int)blockIdx.x, n_walkers = PAIR ? (int)gridDim.x / 2 : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 5 : 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], PAIR ? 8 : 4); }
     fence_mbar_init();
     prefetch_tmap(&tm_a);
     prefetch_tmap(&tm_b0);
     prefetch_tmap(&tm_b1);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  if (warp == 1) {
+    if (PAIR) { tmem_alloc2(tmem_slot, 512); tmem_relinquish2(); }
+    else { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  }
   tc_fence_before();
   __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  uint32_t tmem_base;
+  if (PAIR) {
+    cluster_sync_all();              // both CTAs have their barriers and tensor memory before either touches the other's
+    tc_fence_after();
+    tmem_base = ld_cluster_u32(map_to_cta(smem_u32(tmem_slot), 0));
+  } else {
+    tc_fence_after();
+    tmem_base = *tmem_slot;
+  }
   // A (and everything the finishing pass reads) may be the previous kernel's output
   pdl_wait();
   pdl_launch_dependents();
@@ -102,30 +132,49 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
   const int KB = p.K / BK;
   const int n_rows = GATHER ? min(*p.count, p.m_total) : 0;
-  const int total_tiles = GATHER ? ((n_rows + BM - 1) / BM) * n_tiles : total_tiles_dense;
+  // (PAIR: units = column tiles x pairs of row tiles; this CTA's row tile of unit u is 2 * (u / n_tiles) + pr, and
+  // a row tile past the end of an odd count runs the main loop for its partner's sake and finishes no rows)
+  const int total_tiles = GATHER ? ((n_rows + BM - 1) / BM) * n_tiles
+                                 : (PAIR ? n_tiles * ((p.m_tiles + 1) / 2) : total_tiles_dense);
+  auto tile_of = [&](int u) {
+    if (!PAIR) return tile_geom(p, u, n_tiles, GATHER, n_rows);
+    const int nt = u % n_tiles, mt = 2 * (u / n_tiles) + pr;
+    TileGeom t = tile_geom(p, (mt < p.m_tiles ? mt : mt - 1) * n_tiles + nt, n_tiles, false, 0);
+    if (mt >= p.m_tiles) t.rows_valid = 0;
+    return t;
+  };
   if (warp == 0) {
     // ---- producer
     uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const TileGeom t = tile_geom(p, tile, n_tiles, GATHER, n_rows);
+    for (int tile = walker; tile < total_tiles; tile += n_walkers) {
+      const TileGeom t = tile_of(tile);
       const CUtensorMap* tm_b = t.is_b1 ? &tm_b1 : &tm_b0;
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int s = it % STAGES;
         mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, p.status);
         if (elect_one()) {
           uint8_t* dst = smem + s * STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(GATHER ? B_BYTES : STAGE_BYTES));
-          if (!GATHER) tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
-          tma_load_2d(dst + A_BYTES, tm_b, kb * BK, t.n0, &full_bar[s]);
+          if (PAIR) {
+            // the bytes of both CTAs are counted on the even CTA's barrier; each brings its rows of A and its half
+            // of the W tile's rows
+            const uint32_t fb = map_to_cta(smem_u32(&full_bar[s]), 0);
+            if (pr == 0) mbar_arrive_expect_tx(&full_bar[s], 2u * STAGE_BYTES);
+            tma_load_2d_pair(dst, &tm_a, kb * BK, t.a_row, fb);
+            tma_load_2d_pair(dst + A_BYTES, tm_b, kb * BK, t.n0 + pr * (BN / 2), fb);
+          } else {
+            mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(GATHER ? B_BYTES : STAGE_BYTES));
+            if (!GATHER) tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
+            tma_load_2d(dst + A_BYTES, tm_b, kb * BK, t.n0, &full_bar[s]);
+          }
         }
         __syncwarp();
       }
     }
-  } else if (warp == 1) {
-    // ---- MMA issuer
-    constexpr uint32_t idesc = idesc_bf16(BM, BN);
+  } else if (warp == 1 && pr == 0) {
+    // ---- MMA issuer (of a pair: the even CTA's)
+    constexpr uint32_t idesc = idesc_bf16(PAIR ? 2 * BM : BM, BN);
     uint32_t it = 0, tcount = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
+    for (int tile = walker; tile < total_tiles; tile += n_walkers, ++tcount) {
       const uint32_t buf = tcount & 1;
       mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, p.status);     // (passes at once the first two times)
       tc_fence_after();
@@ -138,20 +187,34 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
           const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
           const uint64_t a_desc = smem_desc_k_sw128(a_addr), b_desc = smem_desc_k_sw128(a_addr + A_BYTES);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) umma_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit(&empty_bar[s]);
-          if (kb == KB - 1) umma_commit(&acc_full[buf]);
+          for (int k = 0; k < BK / 16; ++k) {
+            if (PAIR) umma2_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else umma_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          if (PAIR) {                      // the stage is free again, and the accumulator complete, in both CTAs
+            umma2_commit(map_to_cta(smem_u32(&empty_bar[s]), 0));
+            umma2_commit(map_to_cta(smem_u32(&empty_bar[s]), 1));
+            if (kb == KB - 1) {
+              umma2_commit(map_to_cta(smem_u32(&acc_full[buf]), 0));
+              umma2_commit(map_to_cta(smem_u32(&acc_full[buf]), 1));
+            }
+          } else {
+            umma_commit(&empty_bar[s]);
+            if (kb == KB - 1) umma_commit(&acc_full[buf]);
+          }
         }
         __syncwarp();
       }
     }
+  } else if (warp == 1) {
+    // (the odd CTA of a pair issues nothing)
   } else if (GATHER && warp >= 6) {
     // ---- A-operand producers of a gathered launch.  One stage of the A tile = 128 rows x 128 bytes; a warp takes 32
     // rows; one copy instruction covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row.
     const int gq = warp - 6;
     constexpr int LAG = STAGES - 2;                              // copy groups in flight per thread
     uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, it += KB) {
+    for (int tile = walker; tile < total_tiles; tile += n_walkers, it += KB) {
       const TileGeom t = tile_geom(p, tile, n_tiles, true, n_rows);
       const int r_own = gq * 32 + lane;                          // the row whose token this lane looks up
       const int tok_own = r_own < t.rows_valid ? p.idx[t.t0 + r_own] : -1;
@@ -192,8 +255,8 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     const uint32_t stg_w = smem_u32(stg) + (uint32_t)lane * STG_ROW_BYTES;    // this thread's row when it writes
     const int half_id = lane >> 4, l16 = lane & 15;
     uint32_t tcount = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
-      const TileGeom t = tile_geom(p, tile, n_tiles, GATHER, n_rows);
+    for (int tile = walker; tile < total_tiles; tile += n_walkers, ++tcount) {
+      const TileGeom t = tile_of(tile);
       const uint32_t buf = tcount & 1;
       mbar_wait(&acc_full[buf], (tcount >> 1) & 1, p.status);
       tc_fence_after();
@@ -228,7 +291,10 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         if (chunk == 3) {                                // the accumulator is free for the tile after next
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&acc_empty[buf]);
+          if (lane == 0) {
+            if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));   // (the issuing CTA's barrier)
+            else mbar_arrive(&acc_empty[buf]);
+          }
         }
         __syncwarp();
         const bool score_chunk = score_tile && head0 + hh == p.g.score_head;
@@ -340,16 +406,20 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
   }
   tc_fence_before();
-  __syncthreads();
+  // (a pair: nobody frees tensor memory or leaves while its partner's MMAs or barrier arrivals may still refer to it)
+  if (PAIR) cluster_sync_all(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
-  if (warp == 1) tmem_dealloc(tmem_base, 512);
+  if (warp == 1) {
+    if (PAIR) tmem_dealloc2(*tmem_slot, 512);
+    else tmem_dealloc(tmem_base, 512);
+  }
 }
 
-template <int EPI, bool GATHER>
+template <int EPI, bool GATHER, bool PAIR = false>
 static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
                                   int n_tiles, int m_tiles, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  auto kern = gemm_persist_kernel<EPI, GATHER>;
+  auto kern = gemm_persist_kernel<EPI, GATHER, PAIR>;
   if (cudaError_t e = ensure_dyn_smem(kern, SMEM_TOTAL, attr_done); e != cudaSuccess) return e;
   int dev = 0, sms = 0;
   if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
@@ -357,6 +427,10 @@ static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, c
   const int total = n_tiles * m_tiles;
   GemmParams q = p;
   q.m_tiles = m_tiles;
+  if (PAIR) {
+    const int units = n_tiles * ((m_tiles + 1) / 2), clusters = units < sms / 2 ? units : sms / 2;
+    return launch_pdl_xz(kern, dim3(2 * clusters), dim3(kWarpsDense * 32), SMEM_TOTAL, st, 2, 1, a, b0, b1, q, n_tiles, total);
+  }
   return launch_pdl(kern, dim3(total < sms ? total : sms), dim3((GATHER ? kWarpsGather : kWarpsDense) * 32), SMEM_TOTAL, st,
                     1, a, b0, b1, q, n_tiles, total);
 }
@@ -364,15 +438,23 @@ static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, c
 // 256-wide tiles, no reduction split; b0 / b1 are maps with 256-row boxes.  Gathered launches (idx, count and
 // gather_src set; m_tiles = capacity of the row list in tiles) fetch their A rows by index.
 cudaError_t launch_gemm_persist(int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                                const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st) {
+                                const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st, int pair) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
   if (p.b_pair || p.K % BK != 0) return cudaErrorInvalidValue;
   const bool gather = p.gather_src != nullptr;
   if (gather != (p.idx != nullptr) || gather != (p.count != nullptr)) return cudaErrorInvalidValue;
   if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
   if (gather) {
+    if (pair) return cudaErrorInvalidValue;
     if (epi == EPI_KV) return launch_persist<EPI_KV, true>(a, b0, b1, p, n_tiles, m_tiles, st);
     if (epi == EPI_OUT) return launch_persist<EPI_OUT, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    return cudaErrorInvalidValue;
+  }
+  if (pair) {            // two-CTA MMAs: b0 / b1 are maps with 128-row boxes
+    if (epi == EPI_Q) return launch_persist<EPI_Q, false, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    if (epi == EPI_KV) return launch_persist<EPI_KV, false, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    if (epi == EPI_OUT) return launch_persist<EPI_OUT, false, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    if (epi == EPI_OUT_RES) return launch_persist<EPI_OUT_RES, false, true>(a, b0, b1, p, n_tiles, m_tiles, st);
     return cudaErrorInvalidValue;
   }
   if (epi == EPI_Q) return launch_persist<EPI_Q, false>(a, b0, b1, p, n_tiles, m_tiles, st);

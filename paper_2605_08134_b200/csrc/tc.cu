@@ -23,6 +23,9 @@ bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0
 #ifndef DARE_NARROW_PAIRS
 #define DARE_NARROW_PAIRS 1
 #endif
+#ifndef DARE_PERSIST_PAIR
+#define DARE_PERSIST_PAIR 1
+#endif
 #ifndef DARE_PERSIST_GATHER
 #define DARE_PERSIST_GATHER 1
 #endif
@@ -142,7 +145,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
       e = launch_gemm_tc(EPI_Q, 128, S.a_xn, S.w_q64, S.w_q64, p, d / 128, m_tiles_dense, 2, st, 1);
     else if (use_persist(n_tiles, m_tiles_dense, sp))
-      e = launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st);
+      e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_Q, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, st, 1)
+                               : launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st));
     else if (use_pairs(n_tiles, m_tiles_dense, sp))
       e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
     else
@@ -185,7 +189,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       prof_mark(L, SLOT_KV_GEMM, st);
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
       if (use_persist(n_tiles, m_tiles_dense, sp))
-        e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, st);
+        e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_KV, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, st, 1)
+                               : launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, st));
       else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else
@@ -234,7 +239,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
         e = launch_gemm_tc(EPI_OUT, 128, S.a_oc, S.w_o64, S.w_o64, p, d / 128, m_tiles_dense, 2, st, 1);
       else if (use_persist(n_tiles, m_tiles_dense, sp))
-        e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, st);
+        e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, st, 1)
+                               : launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, st));
       else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else

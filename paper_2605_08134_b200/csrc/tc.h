@@ -84,8 +84,9 @@ cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensor
 
 // Persistent form for launches of many row tiles (dense rows, 256-wide tiles, no reduction split, epilogues Q, K/V,
 // OUT): one CTA per SM walks the tiles, finishing pass overlapped with the next tile's main loop.
+// pair != 0 (dense launches only): two-CTA MMAs over pairs of row tiles, b0 / b1 with 128-row boxes.
 cudaError_t launch_gemm_persist(int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                                const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st);
+                                const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st, int pair = 0);
 // ... pays from about two waves of tiles on.
 inline bool persist_pays(int n_tiles, int m_tiles, int splits) { return splits == 1 && n_tiles * m_tiles >= 296; }
 
