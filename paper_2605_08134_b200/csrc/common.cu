@@ -441,6 +441,35 @@ void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, 
   int grid = max_rows < 148 * 8 ? max_rows : 148 * 8;
   gather_rows_kernel<T><<<grid, 256, 0, st>>>(src, idx, count, dst, max_rows, d);
 }
+// The same for the rows of a step's refresh set, by flat token index or (by_cache_row) by cache row: a stream of
+// n * d elements, chained with programmatic dependent launch.
+template <typename T>
+__global__ void __launch_bounds__(256) gather_step_rows_kernel(const T* __restrict__ src, const int* __restrict__ idx,
+                                                               const int* __restrict__ count, T* __restrict__ dst,
+                                                               StepGeom g, int by_cache_row) {
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
+  const int n = min(*count, g.tokens());
+  constexpr int N = 16 / sizeof(T);
+  const int nvec = g.d / N;
+  for (int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += gridDim.x * (blockDim.x >> 5)) {
+    const int tok = idx[r];
+    const size_t srow = by_cache_row ? (size_t)g.cache_row(tok) : (size_t)tok;
+    const uint4* s = reinterpret_cast<const uint4*>(src + srow * g.d);
+    uint4* o = reinterpret_cast<uint4*>(dst + (size_t)r * g.d);
+    for (int v = threadIdx.x & 31; v < nvec; v += 32) o[v] = s[v];
+  }
+}
+template <typename T>
+void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
+                             cudaStream_t st) {
+  const int T_ = g.tokens();
+  if (T_ <= 0) return;
+  const int grid = (T_ + 7) / 8 < 148 * 8 ? (T_ + 7) / 8 : 148 * 8;
+  launch_pdl(gather_step_rows_kernel<T>, dim3(grid), dim3(256), 0, st, 1, src, idx, count, dst, g, by_cache_row ? 1 : 0);
+}
+template void launch_gather_step_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*,
+                                                     const StepGeom&, bool, cudaStream_t);
 template void launch_gather_rows<float>(const float*, const int*, const int*, float*, int, int, cudaStream_t);
 template void launch_gather_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*, int, int,
                                                 cudaStream_t);

@@ -92,6 +92,10 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
                    int* batch_off, int* delta, cudaStream_t st);
 template <typename T>
 void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
+// dst[r, :] = src[idx[r] (or its cache row), :] for the rows of a step's refresh set
+template <typename T>
+void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
+                             cudaStream_t st);
 
 // ---- stand-alone score / compaction for large token counts (select_large.cu)
 int select_large_tiles(long long n);

@@ -12,12 +12,13 @@
 //              the row segments are stored; the accumulator is handed back after the last read of tensor memory
 // In the one-tile-per-CTA kernel of gemm_tc.cu a tile costs set-up + pipeline fill + finishing pass + the gap to the
 // next CTA on top of its main loop (about 30 % at these sizes, measured); here the main loops follow one another.
-// Gathered launches (the rows of the refresh set, Alg. 1 line 6 / the gathered output projection) add
-//   warps 6-9  A-operand producers: the rows named by the index list are fetched 16 bytes at a time with cp.async into
-//              the swizzled tile layout (eight consecutive lanes on one row: whole 128-byte lines), each warp
-//              arriving on a stage's barrier once its 32 rows of that stage have landed
-// and read the number of row tiles from the device-side count, so no CTA is spent on tiles past the refresh set.
-// PAIR (dense launches): the CTAs of a cluster of two take row tiles 2i and 2i + 1 of the same column tile as one
+// Listed launches (the rows of a refresh set, Alg. 1 line 6 / the gathered output projection, given by an index list
+// with a device-side count): A is a compact copy of the listed rows, made by a copy kernel before the launch (row r of
+// the list = row r of the copy), so that every operand comes through TMA; the number of row tiles is read from the
+// count, so no CTA is spent on tiles past the refresh set; the finishing pass takes positions and cache rows from the
+// tokens.  Such a launch is issued in both forms below (one-CTA and two-CTA tiles), and the one the count does not
+// favour leaves at once.
+// PAIR: the CTAs of a cluster of two take row tiles 2i and 2i + 1 of the same column tile as one
 // M = 256 tcgen05.mma.cta_group::2 issued by the even CTA; each keeps its own 128 rows of A and 128 of the W tile's
 // 256 rows (32 KB per stage, six stages), which takes a third off what an SM pulls from the L2 per flop: the
 // one-CTA form runs its main loop at 667 cycles per 64 k-elements against 512 of tensor work, bound by that
@@ -49,7 +50,7 @@ constexpr int ACC_OFFSET = STG_OFFSET + 4 * STG_WARP_BYTES;   // partial score s
 constexpr int BAR_OFFSET = ACC_OFFSET + BM * 12;
 static_assert(BAR_OFFSET + 256 + 1024 <= 227 * 1024, "shared memory of one CTA");
 constexpr int SMEM_TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
-constexpr int kWarpsDense = 6, kWarpsGather = 10;
+constexpr int kWarps = 6;
 
 struct TileGeom {
   int nt, mt, n0, is_b1;
@@ -66,7 +67,7 @@ __device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int
   if (gather) {                      // rows t0 .. of the index list; position and cache row come from the tokens
     t.t0 = t.mt * BM;
     t.rows_valid = min(BM, n_rows - t.t0);
-    t.a_row = 0; t.pos0 = 0; t.crow0 = 0;
+    t.a_row = t.t0; t.pos0 = 0; t.crow0 = 0;     // (a_row: the row of a compact copy of the listed rows)
     return t;
   }
   const int b = t.mt / p.tiles_per_seq, tis = t.mt - b * p.tiles_per_seq;
@@ -79,12 +80,13 @@ __device__ __forceinline__ TileGeom tile_geom(const GemmParams& p, int tile, int
 }
 }  // namespace
 
+// GATHER: the rows of the launch are listed by an index list with a device-side count (row geometry and finishing
+// pass by token); A maps a compact copy of them.
 template <int EPI, bool GATHER, bool PAIR>
-__global__ void __launch_bounds__((GATHER ? kWarpsGather : kWarpsDense) * 32, 1)
+__global__ void __launch_bounds__(kWarps * 32, 1)
 gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                     const __grid_constant__ CUtensorMap tm_b1, const GemmParams p, const int n_tiles,
                     const int total_tiles_dense) {
-  static_assert(!(GATHER && PAIR), "gathered launches use single-CTA tiles");
   constexpr int STAGES = Ring<PAIR>::STAGES, STAGE_BYTES = Ring<PAIR>::STAGE_BYTES, B_BYTES = Ring<PAIR>::B_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -103,7 +105,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   const int walker = PAIR ? (int)blockIdx.x / 2 : (int)blockIdx.x, n_walkers = PAIR ? (int)gridDim.x / 2 : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 5 : 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], PAIR ? 8 : 4); }
     fence_mbar_init();
     prefetch_tmap(&tm_a);
@@ -134,11 +136,19 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   const int n_rows = GATHER ? min(*p.count, p.m_total) : 0;
   // (PAIR: units = column tiles x pairs of row tiles; this CTA's row tile of unit u is 2 * (u / n_tiles) + pr, and
   // a row tile past the end of an odd count runs the main loop for its partner's sake and finishes no rows)
-  const int total_tiles = GATHER ? ((n_rows + BM - 1) / BM) * n_tiles
-                                 : (PAIR ? n_tiles * ((p.m_tiles + 1) / 2) : total_tiles_dense);
+  const int m_tiles_live = GATHER ? (n_rows + BM - 1) / BM : p.m_tiles;
+  int total_tiles = PAIR ? n_tiles * ((m_tiles_live + 1) / 2) : (GATHER ? m_tiles_live * n_tiles : total_tiles_dense);
+  // A listed launch whose size only the device knows is issued in both forms; each looks at the count and one of them
+  // leaves at once: pairs pay when there are enough units to keep every cluster busy for two rounds or more.
+  if (GATHER && p.unit_gate > 0 && (n_tiles * ((m_tiles_live + 1) / 2) >= p.unit_gate) != PAIR) total_tiles = 0;
   auto tile_of = [&](int u) {
     if (!PAIR) return tile_geom(p, u, n_tiles, GATHER, n_rows);
     const int nt = u % n_tiles, mt = 2 * (u / n_tiles) + pr;
+    if (GATHER) {                      // (the tile past an odd count has no rows: nothing stored)
+      TileGeom t = tile_geom(p, mt * n_tiles + nt, n_tiles, true, n_rows);
+      t.rows_valid = max(t.rows_valid, 0);
+      return t;
+    }
     TileGeom t = tile_geom(p, (mt < p.m_tiles ? mt : mt - 1) * n_tiles + nt, n_tiles, false, 0);
     if (mt >= p.m_tiles) t.rows_valid = 0;
     return t;
@@ -162,8 +172,8 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             tma_load_2d_pair(dst, &tm_a, kb * BK, t.a_row, fb);
             tma_load_2d_pair(dst + A_BYTES, tm_b, kb * BK, t.n0 + pr * (BN / 2), fb);
           } else {
-            mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(GATHER ? B_BYTES : STAGE_BYTES));
-            if (!GATHER) tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
+            mbar_arrive_expect_tx(&full_bar[s], (uint32_t)STAGE_BYTES);
+            tma_load_2d(dst, &tm_a, kb * BK, t.a_row, &full_bar[s]);
             tma_load_2d(dst + A_BYTES, tm_b, kb * BK, t.n0, &full_bar[s]);
           }
         }
@@ -208,45 +218,6 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
   } else if (warp == 1) {
     // (the odd CTA of a pair issues nothing)
-  } else if (GATHER && warp >= 6) {
-    // ---- A-operand producers of a gathered launch.  One stage of the A tile = 128 rows x 128 bytes; a warp takes 32
-    // rows; one copy instruction covers four rows, eight consecutive lanes fetching the eight 16-byte units of a row.
-    const int gq = warp - 6;
-    constexpr int LAG = STAGES - 2;                              // copy groups in flight per thread
-    uint32_t it = 0;
-    for (int tile = walker; tile < total_tiles; tile += n_walkers, it += KB) {
-      const TileGeom t = tile_geom(p, tile, n_tiles, true, n_rows);
-      const int r_own = gq * 32 + lane;                          // the row whose token this lane looks up
-      const int tok_own = r_own < t.rows_valid ? p.idx[t.t0 + r_own] : -1;
-      const uint8_t* src_k[8];
-      uint32_t dst_k[8], bytes_k[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int rw = k * 4 + (lane >> 3), r = gq * 32 + rw, u = lane & 7;
-        const int tok = __shfl_sync(0xffffffffu, tok_own, rw);
-        const int srow = tok < 0 ? 0 : (p.gather_cache_rows ? p.g.cache_row(tok) : tok);
-        src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)srow * p.K * 2 + u * 16;
-        bytes_k[k] = tok >= 0 ? 16u : 0u;                        // rows past the refresh set are zero-filled
-        dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
-      }
-      for (int i = 0; i < KB + LAG; ++i) {
-        if (i < KB) {
-          const uint32_t g = it + i;
-          const int s = g % STAGES;
-          mbar_wait(&empty_bar[s], ((g / STAGES) & 1) ^ 1, p.status);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)i * (BK * 2), bytes_k[k]);
-        }
-        cp_async_commit();                                       // (empty groups at the tail keep the lag uniform)
-        if (i >= LAG) {
-          cp_async_wait<LAG>();                                  // this thread's copies of block i - LAG have landed
-          fence_proxy_async_smem();                              // ... and are visible to the tensor core's reads
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&full_bar[(it + i - LAG) % STAGES]);
-        }
-      }
-    }
   } else {
     // ---- finishing warps: quarter q of the TMEM lanes = rows 32q .. 32q + 31 of every tile
     const int q = warp & 3;
@@ -265,7 +236,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       int tok_own = -1, tok_first = 0;
       if (GATHER) {
         if (q * 32 + lane < t.rows_valid) tok_own = p.idx[t.t0 + q * 32 + lane];
-        tok_first = p.idx[t.t0];                         // a row that exists, for the table reads of rows that do not
+        tok_first = t.rows_valid > 0 ? p.idx[t.t0] : 0;  // a row that exists, for the table reads of rows that do not
       }
       const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !t.is_b1);
       const int head0 = t.n0 / HD;
@@ -429,25 +400,31 @@ static cudaError_t launch_persist(const CUtensorMap& a, const CUtensorMap& b0, c
   q.m_tiles = m_tiles;
   if (PAIR) {
     const int units = n_tiles * ((m_tiles + 1) / 2), clusters = units < sms / 2 ? units : sms / 2;
-    return launch_pdl_xz(kern, dim3(2 * clusters), dim3(kWarpsDense * 32), SMEM_TOTAL, st, 2, 1, a, b0, b1, q, n_tiles, total);
+    return launch_pdl_xz(kern, dim3(2 * clusters), dim3(kWarps * 32), SMEM_TOTAL, st, 2, 1, a, b0, b1, q, n_tiles, total);
   }
-  return launch_pdl(kern, dim3(total < sms ? total : sms), dim3((GATHER ? kWarpsGather : kWarpsDense) * 32), SMEM_TOTAL, st,
+  return launch_pdl(kern, dim3(total < sms ? total : sms), dim3(kWarps * 32), SMEM_TOTAL, st,
                     1, a, b0, b1, q, n_tiles, total);
 }
 
-// 256-wide tiles, no reduction split; b0 / b1 are maps with 256-row boxes.  Gathered launches (idx, count and
-// gather_src set; m_tiles = capacity of the row list in tiles) fetch their A rows by index.
+// 256-wide tiles, no reduction split; b0 / b1 are maps with 256-row boxes (128-row boxes with pair != 0).  Listed
+// launches (idx and count set, gather_src not; m_tiles = capacity of the row list in tiles): `a` maps a compact copy of
+// the listed rows (row r of the list = row r of the copy).
 cudaError_t launch_gemm_persist(int epi, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                                 const GemmParams& p, int n_tiles, int m_tiles, cudaStream_t st, int pair) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
   if (p.b_pair || p.K % BK != 0) return cudaErrorInvalidValue;
-  const bool gather = p.gather_src != nullptr;
-  if (gather != (p.idx != nullptr) || gather != (p.count != nullptr)) return cudaErrorInvalidValue;
+  const bool listed = p.idx != nullptr, gather = p.gather_src != nullptr;
+  if (listed != (p.count != nullptr) || (gather && !listed)) return cudaErrorInvalidValue;
   if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
-  if (gather) {
-    if (pair) return cudaErrorInvalidValue;
-    if (epi == EPI_KV) return launch_persist<EPI_KV, true>(a, b0, b1, p, n_tiles, m_tiles, st);
-    if (epi == EPI_OUT) return launch_persist<EPI_OUT, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+  if (gather) return cudaErrorInvalidValue;       // (rows fetched by index inside the kernel: gemm_tc.cu)
+  if (listed) {          // A = compact copy of the listed rows
+    if (pair) {
+      if (epi == EPI_KV) return launch_persist<EPI_KV, true, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+      if (epi == EPI_OUT) return launch_persist<EPI_OUT, true, true>(a, b0, b1, p, n_tiles, m_tiles, st);
+    } else {
+      if (epi == EPI_KV) return launch_persist<EPI_KV, true, false>(a, b0, b1, p, n_tiles, m_tiles, st);
+      if (epi == EPI_OUT) return launch_persist<EPI_OUT, true, false>(a, b0, b1, p, n_tiles, m_tiles, st);
+    }
     return cudaErrorInvalidValue;
   }
   if (pair) {            // two-CTA MMAs: b0 / b1 are maps with 128-row boxes

@@ -8,6 +8,7 @@ namespace dare {
 
 struct TcState {
   CUtensorMap a_xn, a_oc;                  // A operands, box 64 x 128 rows
+  CUtensorMap a_xg;                        // compact copy of a refresh set's rows (the input staging buffer, idle after RMSNorm)
   CUtensorMap w_q, w_k, w_v, w_o;          // weights, box 64 x 256 rows
   CUtensorMap w_k128, w_v128, w_q128, w_o128;   // weights, box 64 x 128 rows
   CUtensorMap w_q64, w_o64;                // weights, box 64 x 64 rows (narrow pair tiles)
@@ -26,8 +27,10 @@ bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0
 #ifndef DARE_PERSIST_PAIR
 #define DARE_PERSIST_PAIR 1
 #endif
-#ifndef DARE_PERSIST_GATHER
-#define DARE_PERSIST_GATHER 1
+// units (column tile x pair of row tiles) from which the two-CTA form of a listed launch runs: two rounds of the 74 clusters
+constexpr int kPairUnitGate = 148;
+#ifndef DARE_PERSIST_LIST
+#define DARE_PERSIST_LIST 1
 #endif
 #ifndef DARE_PERSIST
 #define DARE_PERSIST 1
@@ -83,7 +86,7 @@ dare_status_t tc_create(dare_layer* L) {
   TcState* s = new (std::nothrow) TcState();
   if (!s) return DARE_ERR_INVALID_ARG;
   const uint64_t Tm = (uint64_t)L->cfg.max_batch * L->cfg.max_seq, d = L->cfg.d_model;
-  bool ok = make_map(&s->a_xn, L->buf.xn, Tm, d, 128) &&
+  bool ok = make_map(&s->a_xn, L->buf.xn, Tm, d, 128) && make_map(&s->a_xg, L->buf.x_stage, Tm, d, 128) &&
             make_map(&s->a_oc, L->buf.oc, Tm, d, 128) && make_map(&s->w_q, L->w.w_q, d, d, 256) &&
             make_map(&s->w_k, L->w.w_k, d, d, 256) && make_map(&s->w_v, L->w.w_v, d, d, 256) &&
             make_map(&s->w_o, L->w.w_o, d, d, 256) && make_map(&s->w_k128, L->w.w_k, d, d, 128) &&
@@ -110,6 +113,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   const bool has_prev = L->has_prev;
   const bool kv_sparse = has_prev && (mode & DARE_MODE_KV);
   const bool o_sparse = has_prev && (mode & DARE_MODE_O);
+  // the input staging buffer doubles as the compact copy of a refresh set's rows once x has been normalised; not
+  // when x is still needed later (the residual of a transformer block reads it in the output projection)
+  const bool compact_ok = !add_input || x != B.x_stage;
   const int tiles_per_seq = (g.seq_act + 127) / 128;
   const int m_tiles_dense = g.batch * tiles_per_seq;
   const int kblocks = d / 64;
@@ -119,7 +125,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   GemmParams base;
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
-  base.gather_src = nullptr; base.gather_cache_rows = 0;
+  base.gather_src = nullptr; base.gather_cache_rows = 0; base.unit_gate = 0;
   base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
   base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
@@ -179,9 +185,15 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
                            pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
-        if (DARE_PERSIST_GATHER && use_persist(n_tiles, m_tiles, 1))
-          e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, st);
-        else
+        if (DARE_PERSIST_LIST && use_persist(n_tiles, m_tiles, 1) && compact_ok) {
+          // a compact copy of the refresh set's rows first (a stream of n x d elements), then the projection with
+          // every operand through TMA and two-CTA MMAs
+          launch_gather_step_rows((const bf16*)B.xn, B.idx, B.count, (bf16*)B.x_stage, g, false, st); ++launches;
+          p.gather_src = nullptr;
+          p.unit_gate = kPairUnitGate;
+          e = launch_gemm_persist(EPI_KV, S.a_xg, S.w_k128, S.w_v128, p, n_tiles, m_tiles, st, 1); ++launches;
+          if (e == cudaSuccess) e = launch_gemm_persist(EPI_KV, S.a_xg, S.w_k, S.w_v, p, n_tiles, m_tiles, st, 0);
+        } else
           e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st);
         ++launches;
       }
@@ -227,9 +239,13 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     prof_mark(L, SLOT_OUT_GEMM, st);
     if (y_sparse) {
       p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.oc; p.gather_cache_rows = 1;
-      if (DARE_PERSIST_GATHER && use_persist(n_tiles, (T_ + 127) / 128, 1))
-        e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, st);
-      else
+      if (DARE_PERSIST_LIST && use_persist(n_tiles, (T_ + 127) / 128, 1) && compact_ok) {
+        launch_gather_step_rows((const bf16*)B.oc, B.idx, B.count, (bf16*)B.x_stage, g, true, st); ++launches;
+        p.gather_src = nullptr;
+        p.unit_gate = kPairUnitGate;
+        e = launch_gemm_persist(EPI_OUT, S.a_xg, S.w_o128, S.w_o128, p, n_tiles, (T_ + 127) / 128, st, 1); ++launches;
+        if (e == cudaSuccess) e = launch_gemm_persist(EPI_OUT, S.a_xg, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, st, 0);
+      } else
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, 1, st);
       ++launches;
       if (e != cudaSuccess) return DARE_ERR_CUDA;

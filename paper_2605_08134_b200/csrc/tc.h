@@ -23,6 +23,9 @@ struct GemmParams {
   const __nv_bfloat16* gather_src;  // gathered: the matrix [*, K] whose rows idx[] the kernel fetches itself as its A
                                     // operand (Alg. 1 line 6); nullptr: A comes through the tensor map
   int gather_cache_rows; // gather_src is addressed by cache row (the O cache) instead of by flat token index
+  int unit_gate;         // persistent listed launches issued as a pair of kernels: the two-CTA form runs when the count
+                         // gives it at least this many (column tile, row-tile pair) units, the one-CTA form otherwise;
+                         // 0: no gate
   StepGeom g;
   int n_split;           // n-tiles [0, n_split) use W0/out0, the rest W1/out1
   __nv_bfloat16* out0;
