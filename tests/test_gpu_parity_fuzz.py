@@ -63,3 +63,40 @@ def test_random_steps(dare, case):
         else:
             parity.compare_step(g, o, np.ascontiguousarray(x[:, prompt:]), mode, 0.1, shape, pos_begin=prompt)
     g.close()
+
+
+BIG = [(512, 5, 3892, 1075), (1024, 5, 3196, 3030), (4096, 2, 2159, 564)]
+
+
+@pytest.mark.parametrize("case", range(len(BIG)))
+def test_large_geometries_repeat_bit_identically(dare, case):
+    """Shapes of several thousand rows (persistent projections in their one- and two-CTA forms, listed launches, two query
+    tiles per attention CTA): two fresh handles through the same four steps give bit-identical outputs and caches."""
+    import torch
+    d_model, batch, seq, prompt = BIG[case]
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=d_model, n_heads=d_model // 128, batch=batch, seq=seq, prompt=prompt)
+    w = wl.make_weights(shape, 800 + case)
+    hs = wl.HiddenStream(shape, 800 + case)
+    rng = np.random.default_rng(6000 + case)
+    steps = [(hs.first(), int(rng.integers(0, 4)), 0)]
+    for _ in range(3):
+        mode = int(rng.integers(0, 4))
+        n = max(1, int(round(float(rng.choice([0.03, 0.13, 0.4, 1.0])) * seq)))
+        x = hs.advance(wl.uniform_positions(hs.rng, shape, n))
+        if rng.random() < 0.4:
+            steps.append((np.ascontiguousarray(x[:, prompt:]), mode, prompt))
+        else:
+            steps.append((x, mode, 0))
+    outs = []
+    for _ in range(2):
+        g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+        ys = [g.step(parity.to_device(x, shape), mode, 0.1, pos_begin=pb).clone() for x, mode, pb in steps]
+        torch.cuda.synchronize()
+        caches = g.read_caches(batch, seq)
+        assert g.status() == 0
+        g.close()
+        outs.append((ys, caches))
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    for name in ("k", "v", "o"):
+        np.testing.assert_array_equal(outs[0][1][name], outs[1][1][name])
