@@ -164,6 +164,9 @@ dare_status_t enqueue_step(dare_layer_t* L, const void* x, int batch, int seq_ac
     s = step_simt<float>(L, (const float*)x, g, mode, tau, (float*)y, st);
   }
   if (s != DARE_OK) return s;
+  // (a step may use the input staging buffer as scratch; once the asynchronous host-buffer entry point is in use, its
+  // next copy in waits for this step, whichever entry point issued it)
+  if (L->host_async_ready && cudaEventRecord(L->ev_consumed, st) != cudaSuccess) return DARE_ERR_CUDA;
   if (!L->has_prev) { L->kv_len = seq_act; L->batch = batch; }
   L->has_prev = true;
   L->last_geom = g;
@@ -284,6 +287,7 @@ dare_status_t dare_layer_step_host(dare_layer_t* L, const void* x_host, int batc
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
   const size_t bytes = (size_t)batch * seq_act * L->cfg.d_model * e;
+  if (L->host_async_ready) CUDA_TRY(cudaStreamWaitEvent(st, L->ev_out, 0));   // (an earlier asynchronous copy out)
   CUDA_TRY(cudaMemcpyAsync(L->buf.x_stage, x_host, bytes, cudaMemcpyHostToDevice, st));
   s = enqueue_step(L, L->buf.x_stage, batch, seq_act, pos_begin, mode, threshold, L->buf.y_stage, st);
   if (s != DARE_OK) return s;
@@ -305,6 +309,9 @@ dare_status_t dare_layer_step_host_async(dare_layer_t* L, const void* x_host, in
     CUDA_TRY(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
     // (never-recorded events: waiting on them returns at once, which is right for the first step)
     L->host_async_ready = true;
+    // steps issued before through the other entry points may still be using the staging buffers
+    CUDA_TRY(cudaEventRecord(L->ev_consumed, st));
+    CUDA_TRY(cudaEventRecord(L->ev_out, st));
   }
   const size_t e = L->cfg.dtype == DARE_BF16 ? 2 : 4;
   const size_t bytes = (size_t)batch * seq_act * L->cfg.d_model * e;
@@ -315,9 +322,8 @@ dare_status_t dare_layer_step_host_async(dare_layer_t* L, const void* x_host, in
   // the step: behind the copy in, and behind the previous copy out of the output staging buffer
   CUDA_TRY(cudaStreamWaitEvent(st, L->ev_in, 0));
   CUDA_TRY(cudaStreamWaitEvent(st, L->ev_out, 0));
-  s = enqueue_step(L, L->buf.x_stage, batch, seq_act, pos_begin, mode, threshold, L->buf.y_stage, st);
+  s = enqueue_step(L, L->buf.x_stage, batch, seq_act, pos_begin, mode, threshold, L->buf.y_stage, st);   // records ev_consumed
   if (s != DARE_OK) return s;
-  CUDA_TRY(cudaEventRecord(L->ev_consumed, st));
   // copy out: behind the step, on its own stream
   CUDA_TRY(cudaStreamWaitEvent(L->copy_out, L->ev_consumed, 0));
   CUDA_TRY(cudaMemcpyAsync(y_host, L->buf.y_stage, bytes, cudaMemcpyDeviceToHost, L->copy_out));
