@@ -269,6 +269,36 @@ def run_ours(args):
             in_chain = {}
         barrier()
 
+    # ---- the same steps replayed from a CUDA graph (two steps of every layer instance captured once): what a caller
+    # gains by taking the launches off the host.  Diagnostics only; `value` stays the stream-launched number.
+    graph_ms_per_step = None
+    try:
+        prime(mode)
+        one_pass(max(args.warmup, 3), mode)
+        torch.cuda.synchronize()
+        n_cap = 2 * len(layers)
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(device)
+        with torch.cuda.graph(graph, stream=side):
+            one_pass(n_cap, mode)
+        reps = max(1, args.steps // n_cap)
+        for _ in range(3):
+            graph.replay()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        graph_ms_per_step = distrib.max_over_ranks(ev0.elapsed_time(ev1), dist, device) / (reps * n_cap)
+        sel = layers[0].last_selection(shape.batch, shape.seq)
+        assert sel["count"] == expect and all(l.status() == 0 for l in layers)
+        del graph
+    except Exception as e:                # diagnostics only
+        print(f"graph replay not measured: {e!r}", file=sys.stderr)
+        graph_ms_per_step = None
+    barrier()
+
     # ---- end to end through the host-buffer entry point (pinned host x and y, copies inside the timed region)
     prime(mode)
     xh = [torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).pin_memory() for a in (xa_np, xb_np)]
@@ -361,6 +391,9 @@ def run_ours(args):
                 "api": "dare_layer_step_host_async + dare_layer_wait_host (copies overlapped across layer instances)",
                 "synchronous_call": {"api": "dare_layer_step_host", "ms_per_step": round(e2e_sync_ms_per_step, 5),
                                      "value": round(world * T / (e2e_sync_ms_per_step * 1e-3), 1)}},
+        "graph_replay": None if graph_ms_per_step is None else
+                        {"ms_per_step": round(graph_ms_per_step, 5),
+                         "what": "the same steps captured once into a CUDA graph (programmatic launch edges kept) and replayed"},
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": roofline,
@@ -528,6 +561,7 @@ def run_stack(args):
                       "prompt": P, "generated": shape.gen_len, "block": lay.block, "batch": B, "threshold": TAU}}
     n_gen = min(args.gen, shape.gen_len) if args.gen > 0 else shape.gen_len
     out["config"]["generated"] = n_gen
+    final_toks = {}
     for name in ("both", "dense"):
         best = None
         for rep in range(2):
@@ -543,6 +577,37 @@ def run_stack(args):
             best = dt if best is None else min(best, dt)
         assert n_gen < shape.gen_len or not bool((toks == shape.mask_id).any())
         out[name] = {"tokens_per_s": round(n_gen * B / best, 1), "ms_per_token": round(best / n_gen * 1e3, 3)}
+        final_toks[name] = toks
+    # ---- the same generation with the decode step of every block captured once into a CUDA graph and replayed for
+    # the block's tokens (the step takes no decision on the host, so one capture serves a whole block); the first step
+    # of the generation (all positions, dense) is enqueued directly.  The host loop never synchronises.
+    try:
+        best, res = None, tuple(torch.empty(B, dtype=dt_, device=dev) for dt_ in (torch.int32, torch.int32, torch.float32))
+        side = torch.cuda.Stream(dev)
+        for rep in range(2):
+            toks_g = torch.from_numpy(np.concatenate([prompt, np.full((B, shape.gen_len), shape.mask_id, np.int32)], 1)).to(dev)
+            stack.reset()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            stack.decode_step_enqueue(toks_g, P, 0, True, MODES["both"], taus, out=res)
+            step = 1
+            while step < n_gen:
+                blk_i = step // lay.block
+                n_here = min(n_gen, (blk_i + 1) * lay.block) - step
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    stack.decode_step_enqueue(toks_g, P, blk_i, False, MODES["both"], taus, out=res)
+                for _ in range(n_here):
+                    graph.replay()
+                step += n_here
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        assert bool((toks_g == final_toks["both"]).all()), "graph replay generated other tokens than the direct launches"
+        out["both_graph"] = {"tokens_per_s": round(n_gen * B / best, 1), "ms_per_token": round(best / n_gen * 1e3, 3),
+                             "what": "one CUDA graph per 32-token block, captured inside the timed region"}
+    except Exception as e:                # diagnostics only
+        print(f"graph replay not measured: {e!r}", file=sys.stderr)
     sel = [stack.layer(l).last_selection(B, lay.seq - P)["count"] for l in range(shape.n_layers)]
     out["value"] = out["both"]["tokens_per_s"]
     out["speedup_of_reuse_path"] = round(out["both"]["tokens_per_s"] / out["dense"]["tokens_per_s"], 3)

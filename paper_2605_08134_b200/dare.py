@@ -509,6 +509,24 @@ class Stack:
         torch.cuda.synchronize(self.device)       # the forced arrays are host memory read by an async copy
         return pos.cpu().numpy(), tok.cpu().numpy(), prob.cpu().numpy()
 
+    def decode_step_enqueue(self, tokens, prompt_len, block_index, first, mode, taus, out=None):
+        """Enqueue-only form of decode_step (no forced choice, no synchronisation, nothing allocated when `out` is
+        given): usable inside a CUDA-graph capture.  -> (pos, tok, prob) device tensors [batch]."""
+        import numpy as np
+        torch = self.torch
+        B = tokens.shape[0]
+        taus = np.ascontiguousarray(taus, np.float32)
+        if out is None:
+            out = (torch.empty(B, dtype=torch.int32, device=self.device),
+                   torch.empty(B, dtype=torch.int32, device=self.device),
+                   torch.empty(B, dtype=torch.float32, device=self.device))
+        st = dare_stack_decode_step(self.handle, tokens.data_ptr(), B, tokens.shape[1], prompt_len, block_index,
+                                    1 if first else 0, mode, taus.ctypes.data, None, None,
+                                    out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_stack_decode_step")
+        return out
+
     def set_capture(self, layer_index, x_buf=None, h_buf=None):
         st = dare_stack_set_capture(self.handle, layer_index, x_buf.data_ptr() if x_buf is not None else None,
                                     h_buf.data_ptr() if h_buf is not None else None)

@@ -257,3 +257,43 @@ def test_tensor_path_is_deterministic(dare, geom):
         assert torch.equal(a, b)
     for k in ("k", "v", "o", "q_prev"):
         np.testing.assert_array_equal(outs[0][1][k], outs[1][1][k])
+
+
+@pytest.mark.parametrize("mode", ["both", "kv", "o", "dense"])
+def test_step_replays_from_a_cuda_graph(dare, mode):
+    """A reuse step captured once into a CUDA graph (programmatic launch edges included) and replayed with new inputs
+    in the same buffers gives, replay after replay, bit for bit what the same steps give when enqueued one by one: the
+    step takes every data-dependent decision on the device and makes no call that a capture forbids."""
+    import torch
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=512, n_heads=4, batch=2, seq=320, prompt=160)
+    w = wl.make_weights(shape, 31)
+    hs = wl.HiddenStream(shape, 31)
+    eager = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    graphed = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    xs = [hs.first()] + [hs.advance(wl.uniform_positions(hs.rng, shape, n)) for n in (40, 0, 150, 320, 17)]
+    xd = [parity.to_device(x, shape) for x in xs]
+    m = MODES[mode]
+    x_buf, y_buf = torch.empty_like(xd[0]), torch.empty_like(xd[0])
+    # first step (dense, fills the caches) and one reuse step outside the graph: the captured step then meets the
+    # same host-side state on every replay
+    for l in (eager, graphed):
+        l.step(xd[0], m, 0.1)
+        l.step(xd[1], m, 0.1)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=side):
+        graphed.step(x_buf, m, 0.1, y=y_buf)
+    for t in range(2, len(xd)):
+        x_buf.copy_(xd[t])
+        graph.replay()
+        ye = eager.step(xd[t], m, 0.1)
+        torch.cuda.synchronize()
+        assert torch.equal(ye, y_buf), (mode, t)
+        if mode != "dense":
+            se, sg = eager.last_selection(2, 320), graphed.last_selection(2, 320)
+            np.testing.assert_array_equal(se["idx"], sg["idx"])
+            np.testing.assert_array_equal(se["delta"], sg["delta"])
+    for l in (eager, graphed):
+        assert l.status() == 0
+        l.close()

@@ -207,3 +207,48 @@ def test_full_size_stack_teacher_forced_layer_checks(dare):
     for l in (0, 13, 31):
         assert g.layer(l).status() == 0
     g.close()
+
+
+def test_decode_steps_replay_from_cuda_graphs(dare):
+    """The decode step takes no decision on the host: one capture per block, replayed for the block's tokens, generates
+    the same tokens as the same steps enqueued one by one."""
+    import torch
+    shape = small_stack()
+    lay = shape.layer
+    B, P = 2, lay.prompt
+    w = wl.make_stack_weights(shape)
+    taus = [0.1] * shape.n_layers
+    prompt = wl.random_prompt(shape, B)
+    start = np.concatenate([prompt, np.full((B, shape.gen_len), shape.mask_id, np.int32)], axis=1)
+    n_steps = shape.gen_len // 2                       # per sequence one token per step: half of the generation
+
+    direct = dare.Stack(shape, w, B)
+    toks_d = torch.from_numpy(start.copy()).cuda()
+    picks_d = []
+    for step in range(n_steps):
+        picks_d.append(direct.decode_step(toks_d, P, step // lay.block, step == 0, 3, taus))
+
+    graphed = dare.Stack(shape, w, B)
+    toks_g = torch.from_numpy(start.copy()).cuda()
+    res = tuple(torch.empty(B, dtype=t, device="cuda") for t in (torch.int32, torch.int32, torch.float32))
+    graphed.decode_step_enqueue(toks_g, P, 0, True, 3, taus, out=res)
+    graphed.decode_step_enqueue(toks_g, P, 0, False, 3, taus, out=res)     # every kernel of a window step has run once
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    step = 2
+    while step < n_steps:
+        blk = step // lay.block
+        n_here = min(n_steps, (blk + 1) * lay.block) - step
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            graphed.decode_step_enqueue(toks_g, P, blk, False, 3, taus, out=res)
+        for i in range(n_here):
+            graph.replay()
+            torch.cuda.synchronize()
+            pos, tok, prob = (r.cpu().numpy() for r in res)
+            np.testing.assert_array_equal(pos, picks_d[step + i][0])
+            np.testing.assert_array_equal(tok, picks_d[step + i][1])
+            np.testing.assert_array_equal(prob, picks_d[step + i][2])
+        step += n_here
+    assert torch.equal(toks_g, toks_d)
+    direct.close(); graphed.close()
