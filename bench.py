@@ -514,19 +514,29 @@ def run_micro(args):
                            "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3)})
     del a, b
     n = 1 << 24
-    s = torch.rand(n, device=dev)
-    s = torch.where(s < 0.87, s * 1e-5, s)
+    # four score arrays in rotation (256 MB, twice the L2): every call reads its scores from HBM
+    bufs = []
+    for i in range(4):
+        s = torch.rand(n, device=dev)
+        bufs.append(torch.where(s < 0.87, s * 1e-5, s))
     idx = torch.empty(n, dtype=torch.int32, device=dev)
     cnt = torch.zeros(1, dtype=torch.int32, device=dev)
     nb = dare.dare_select_compact_scratch_bytes(n)
     scratch = torch.empty(nb, dtype=torch.uint8, device=dev)
-    t = time_it(lambda: dare.dare_select_compact(s.data_ptr(), n, 0.1, idx.data_ptr(), cnt.data_ptr(),
-                                                 scratch.data_ptr(), nb, st))
+    turn = [0]
+
+    def compact():
+        s = bufs[turn[0] & 3]
+        turn[0] += 1
+        dare.dare_select_compact(s.data_ptr(), n, 0.1, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(), nb, st)
+
+    t = time_it(compact)
     k = int(cnt.item())
-    algo = 4.0 * n + 4.0 * k            # scores in, index list out (the kernels read the scores twice)
+    algo = 4.0 * n + 4.0 * k            # scores in, index list out
     out["kernels"].append({"kernel": "select_compact", "tokens": n, "refreshed": k, "us": round(t * 1e6, 1),
                            "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3),
-                           "dram_bytes_moved": 8.0 * n + 4.0 * k})
+                           "l2": "four score arrays in rotation (256 MB)",
+                           "bytes_moved": 4.0 * n + 2.0 * (n / 8.0) + 4.0 * k})   # + decision bits out and back in
     print(json.dumps(out))
 
 

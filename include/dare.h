@@ -201,7 +201,7 @@ dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint6
  * dare_select_compact: Eq. 2 and its complement over `n_tokens` float32 scores: idx receives the ascending list of
  * tokens with !(s <= threshold) (room for n_tokens entries), *count their number.  `scratch` is
  * dare_select_compact_scratch_bytes(n_tokens) bytes of device memory owned by the caller (per-tile counts and
- * offsets); n_tokens <= 2^30; NaN threshold is rejected. */
+ * offsets, and one decision bit per score: about n_tokens / 8 bytes); n_tokens <= 2^30; NaN threshold is rejected. */
 dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t rows, int head_dim, float* scores,
                                 void* cuda_stream);
 size_t dare_select_compact_scratch_bytes(int64_t n_tokens);
@@ -211,8 +211,8 @@ dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float t
 /* dare_select_compact for callers that may not allocate (the paper has no counterpart: this is a service of the
  * library, not a step of the method).  An inference server that gives all device memory to its own arena at start-up,
  * or a latency-critical loop that cannot take the device-wide synchronisation of a cudaMalloc, has no scratch buffer
- * to pass; here the per-tile counts and offsets live in a 32 KB array inside the library image (present on every GPU
- * that loads the library until the process exits).  Same inputs, outputs and results as dare_select_compact.
+ * to pass; here the per-tile counts and offsets and the decision bits live in a 2 MB array inside the library image
+ * (present on every GPU that loads the library until the process exits).  Same inputs, outputs and results as dare_select_compact.
  *   - n_tokens <= dare_select_compact_static_max_tokens() (= 16,777,216); more returns DARE_ERR_SHAPE.
  *   - The call allocates nothing and frees nothing, on the device or through any library.
  *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress with that device

@@ -572,7 +572,8 @@ dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t
 
 size_t dare_select_compact_scratch_bytes(int64_t n_tokens) {
   if (n_tokens < 0 || n_tokens > (int64_t)1 << 30) return 0;
-  return align_up((size_t)select_large_tiles(n_tokens) * sizeof(int)) * 2 + kAlign;
+  return align_up((size_t)select_large_tiles(n_tokens) * sizeof(int)) * 2 + align_up(select_large_flag_bytes(n_tokens)) +
+         kAlign;
 }
 
 dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float threshold, int32_t* idx, int32_t* count,
@@ -585,7 +586,9 @@ dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float t
   const size_t half = align_up((size_t)select_large_tiles(n_tokens) * sizeof(int));
   int* counts = (int*)scratch;
   int* offsets = (int*)((char*)scratch + half);
-  CUDA_TRY(launch_select_large(scores, n_tokens, threshold, idx, count, counts, offsets, (cudaStream_t)cuda_stream));
+  unsigned short* flags = (unsigned short*)((char*)scratch + 2 * half);
+  CUDA_TRY(launch_select_large(scores, n_tokens, threshold, idx, count, counts, offsets, flags,
+                               (cudaStream_t)cuda_stream));
   return DARE_OK;
 }
 

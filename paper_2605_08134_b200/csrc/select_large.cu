@@ -1,20 +1,23 @@
 // Stand-alone drift score and threshold/compaction for token counts far beyond one layer step (millions of rows):
 // the same arithmetic as inside the layer step, organised for HBM bandwidth.
 //   drift score (Sec. 3.1): one warp per row, 16-byte loads of both query rows, shuffle reduction
-//   compaction (Eq. 2, complement): three passes over tiles of 4096 scores
-//     (1) per-tile count of refreshed tokens  -> scratch
+//   compaction (Eq. 2, complement): three passes over tiles of 16384 scores; the scores are read once
+//     (1) per-tile count of refreshed tokens and the decisions themselves, one bit per score -> scratch
 //     (2) exclusive scan of the tile counts (one CTA) -> scratch, total -> *count
-//     (3) per-tile ballot/popcount compaction written at the tile's offset: ascending index list
-// No CTA waits for another; the order of the list does not depend on scheduling.
+//     (3) per-tile compaction from the decision bits, written at the tile's offset: ascending index list
+// No CTA waits for another; the order of the list does not depend on scheduling.  Passes 2 and 3 are launched
+// programmatically dependent: their launch latency hides behind the pass before.
 #include <math.h>
 #include <mutex>
 
 #include "dare_internal.h"
+#include "tc_ptx.cuh"
 
 namespace dare {
 
 namespace {
-constexpr int kTile = 4096;          // scores per CTA (1024 threads x 4)
+constexpr int kThreads = 1024, kVecs = 4;
+constexpr int kTile = kThreads * kVecs * 4;     // 16384 scores per CTA: four 16-byte vectors per thread
 
 __global__ void __launch_bounds__(256) drift_score_kernel(const float* __restrict__ a, const float* __restrict__ b,
                                                           long long rows, int hd, float* __restrict__ scores) {
@@ -44,40 +47,60 @@ __global__ void __launch_bounds__(256) drift_score_kernel(const float* __restric
   }
 }
 
-// refreshed <=> !(s <= tau): a NaN score refreshes
-__device__ __forceinline__ int tile_flags(const float* __restrict__ scores, long long n, long long base, float tau,
-                                          bool (&sel)[4]) {
-  int c = 0;
-  const long long i0 = base + (long long)threadIdx.x * 4;
-  if (i0 + 3 < n) {
-    const float4 v = *reinterpret_cast<const float4*>(scores + i0);
-    sel[0] = !(v.x <= tau); sel[1] = !(v.y <= tau); sel[2] = !(v.z <= tau); sel[3] = !(v.w <= tau);
-  } else {
+// refreshed <=> !(s <= tau): a NaN score refreshes.
+// Thread t of a tile owns the four 16-byte vectors k = 0..3 at scores[base + (k * 1024 + t) * 4 ...]: every load
+// instruction of a warp covers 512 contiguous bytes, and all four are in flight before the first is used.  Its 16
+// decisions are one 16-bit word, bit 4k + j <-> element j of vector k.
+__device__ __forceinline__ unsigned tile_flags(const float* __restrict__ scores, long long n, long long base, float tau) {
+  float4 v[kVecs];
+  bool full[kVecs];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) sel[k] = (i0 + k < n) ? !(scores[i0 + k] <= tau) : false;
+  for (int k = 0; k < kVecs; ++k) {
+    const long long i0 = base + ((long long)k * kThreads + threadIdx.x) * 4;
+    full[k] = i0 + 3 < n;
+    v[k] = make_float4(0.f, 0.f, 0.f, 0.f);                 // 0 <= tau or not, a missing element is masked out below
+    if (full[k]) {
+      v[k] = __ldcs(reinterpret_cast<const float4*>(scores + i0));
+    } else {
+      if (i0 < n) v[k].x = scores[i0];
+      if (i0 + 1 < n) v[k].y = scores[i0 + 1];
+      if (i0 + 2 < n) v[k].z = scores[i0 + 2];
+    }
   }
+  unsigned bits = 0;
 #pragma unroll
-  for (int k = 0; k < 4; ++k) c += sel[k] ? 1 : 0;
-  return c;
+  for (int k = 0; k < kVecs; ++k) {
+    const long long i0 = base + ((long long)k * kThreads + threadIdx.x) * 4;
+    unsigned b = (!(v[k].x <= tau) ? 1u : 0u) | (!(v[k].y <= tau) ? 2u : 0u) | (!(v[k].z <= tau) ? 4u : 0u) |
+                 (!(v[k].w <= tau) ? 8u : 0u);
+    if (!full[k]) {
+      const long long left = n - i0;                        // elements of this vector that exist: <= 3, maybe <= 0
+      b &= left <= 0 ? 0u : ((1u << (int)left) - 1u);
+    }
+    bits |= b << (4 * k);
+  }
+  return bits;
 }
 
-// exclusive prefix of `v` over the 1024 threads of the CTA; *total = sum
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+// exclusive prefix of `v` over the 1024 threads of the CTA; *total = sum.  T: int, or four 16-bit counts packed into
+// 64 bits (no field of a sum over one tile can carry: it is at most 4096).
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T* warp_sums, T* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
+  T inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+    const T n = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += n;
   }
   if (lane == 31) warp_sums[warp] = inc;
   __syncthreads();
   if (warp == 0) {
-    const int w = warp_sums[lane];
-    int winc = w;
+    const T w = warp_sums[lane];
+    T winc = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, winc, o);
+      const T n = __shfl_up_sync(0xffffffffu, winc, o);
       if (lane >= o) winc += n;
     }
     warp_sums[lane] = winc - w;
@@ -87,25 +110,34 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
   return warp_sums[warp] + inc - v;
 }
 
-__global__ void __launch_bounds__(1024) tile_count_kernel(const float* __restrict__ scores, long long n, float tau,
-                                                          int* __restrict__ tile_counts) {
-  __shared__ int warp_sums[32];
+// pass 1: the only pass that reads the scores.  Leaves every thread's 16 decisions and the tile's count.
+__global__ void __launch_bounds__(kThreads) tile_flag_kernel(const float* __restrict__ scores, long long n, float tau,
+                                                             int* __restrict__ tile_counts,
+                                                             unsigned short* __restrict__ flags) {
   __shared__ int total;
-  bool sel[4];
-  const int c = tile_flags(scores, n, (long long)blockIdx.x * kTile, tau, sel);
-  block_exclusive_scan(c, warp_sums, &total);
+  ptx::pdl_launch_dependents();            // the scan's CTA may take its place now; it waits for this grid to complete
+  if (threadIdx.x == 0) total = 0;
+  __syncthreads();
+  const unsigned bits = tile_flags(scores, n, (long long)blockIdx.x * kTile, tau);
+  flags[(size_t)blockIdx.x * kThreads + threadIdx.x] = (unsigned short)bits;
+  const int c = __reduce_add_sync(0xffffffffu, __popc(bits));
+  if ((threadIdx.x & 31) == 0) atomicAdd(&total, c);
+  __syncthreads();
   if (threadIdx.x == 0) tile_counts[blockIdx.x] = total;
 }
 
-__global__ void __launch_bounds__(1024) tile_scan_kernel(const int* __restrict__ tile_counts, int n_tiles,
-                                                         int* __restrict__ tile_offsets, int* __restrict__ count) {
+// pass 2: exclusive scan of the tile counts, one CTA
+__global__ void __launch_bounds__(kThreads) tile_scan_kernel(const int* __restrict__ tile_counts, int n_tiles,
+                                                             int* __restrict__ tile_offsets, int* __restrict__ count) {
   __shared__ int warp_sums[32];
   __shared__ int total;
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
   int base = 0;
-  for (int start = 0; start < n_tiles; start += 1024) {
+  for (int start = 0; start < n_tiles; start += kThreads) {
     const int i = start + threadIdx.x;
     const int v = i < n_tiles ? tile_counts[i] : 0;
-    const int ex = block_exclusive_scan(v, warp_sums, &total);
+    const int ex = block_exclusive_scan<int>(v, warp_sums, &total);
     if (i < n_tiles) tile_offsets[i] = base + ex;
     base += total;
     __syncthreads();
@@ -113,23 +145,39 @@ __global__ void __launch_bounds__(1024) tile_scan_kernel(const int* __restrict__
   if (threadIdx.x == 0) *count = base;
 }
 
-__global__ void __launch_bounds__(1024) tile_scatter_kernel(const float* __restrict__ scores, long long n, float tau,
-                                                            const int* __restrict__ tile_offsets,
-                                                            int* __restrict__ idx) {
-  __shared__ int warp_sums[32];
-  __shared__ int total;
-  bool sel[4];
-  const long long base = (long long)blockIdx.x * kTile;
-  const int c = tile_flags(scores, n, base, tau, sel);
-  int out = tile_offsets[blockIdx.x] + block_exclusive_scan(c, warp_sums, &total);
+// pass 3: from the decisions alone (2 bytes per thread instead of 64 bytes of scores).  The list is ascending, so a
+// tile's order is vector k first, then thread, then element: one scan of the four per-vector counts packed into one
+// 64-bit word gives every thread its place among the threads for each k; the totals of the lower k come before.
+__global__ void __launch_bounds__(kThreads) tile_scatter_kernel(const unsigned short* __restrict__ flags,
+                                                                const int* __restrict__ tile_offsets,
+                                                                int* __restrict__ idx) {
+  __shared__ unsigned long long warp_sums[32];
+  __shared__ unsigned long long total;
+  const unsigned bits = flags[(size_t)blockIdx.x * kThreads + threadIdx.x];      // written two kernels back
+  unsigned long long packed = 0;
 #pragma unroll
-  for (int k = 0; k < 4; ++k)
-    if (sel[k]) idx[out++] = (int)(base + (long long)threadIdx.x * 4 + k);
+  for (int k = 0; k < kVecs; ++k) packed |= (unsigned long long)__popc((bits >> (4 * k)) & 0xfu) << (16 * k);
+  const unsigned long long ex = block_exclusive_scan<unsigned long long>(packed, warp_sums, &total);
+  ptx::pdl_wait();                                                               // the tile offsets: one kernel back
+  const long long base = (long long)blockIdx.x * kTile;
+  int out = tile_offsets[blockIdx.x];
+  const unsigned long long tot = total;
+#pragma unroll
+  for (int k = 0; k < kVecs; ++k) {
+    int o = out + (int)((ex >> (16 * k)) & 0xffffu);
+    const unsigned b = (bits >> (4 * k)) & 0xfu;
+    const int i0 = (int)(base + ((long long)k * kThreads + threadIdx.x) * 4);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (b & (1u << j)) idx[o++] = i0 + j;
+    out += (int)((tot >> (16 * k)) & 0xffffu);
+  }
 }
 
 }  // namespace
 
 int select_large_tiles(long long n) { return (int)((n + kTile - 1) / kTile); }
+size_t select_large_flag_bytes(long long n) { return (size_t)select_large_tiles(n) * kThreads * sizeof(unsigned short); }
 
 cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, int hd, float* scores,
                                 cudaStream_t st) {
@@ -140,14 +188,18 @@ cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, 
   return cudaGetLastError();
 }
 
-// tile_counts and tile_offsets: device arrays of select_large_tiles(n) ints each
+// tile_counts and tile_offsets: device arrays of select_large_tiles(n) ints each; flags: 1024 16-bit words per tile
 cudaError_t launch_select_large(const float* scores, long long n, float tau, int* idx, int* count, int* tile_counts,
-                                int* tile_offsets, cudaStream_t st) {
+                                int* tile_offsets, unsigned short* flags, cudaStream_t st) {
   const int tiles = select_large_tiles(n);
   if (tiles == 0) return cudaMemsetAsync(count, 0, sizeof(int), st);
-  tile_count_kernel<<<tiles, 1024, 0, st>>>(scores, n, tau, tile_counts);
-  tile_scan_kernel<<<1, 1024, 0, st>>>(tile_counts, tiles, tile_offsets, count);
-  tile_scatter_kernel<<<tiles, 1024, 0, st>>>(scores, n, tau, tile_offsets, idx);
+  tile_flag_kernel<<<tiles, kThreads, 0, st>>>(scores, n, tau, tile_counts, flags);
+  cudaError_t e = launch_pdl(tile_scan_kernel, dim3(1), dim3(kThreads), 0, st, 1, (const int*)tile_counts, tiles,
+                             tile_offsets, count);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(tile_scatter_kernel, dim3(tiles), dim3(kThreads), 0, st, 1, (const unsigned short*)flags,
+                 (const int*)tile_offsets, idx);
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 
@@ -158,9 +210,10 @@ cudaError_t launch_select_large(const float* scores, long long n, float tau, int
 //
 // Some hosts of this library hand all of the device's memory to one arena at start-up and forbid every later
 // cudaMalloc (an inference server with a fixed memory plan), or sit in a latency-critical loop where the device-wide
-// synchronisation an allocation implies is not acceptable.  For them the per-tile counts and offsets of the three-pass
-// compaction live in a small array that is part of the library image: 2 x 4096 ints = 32 KB of device memory on every
-// GPU that loads the library, held until the process exits.  That bounds the call at 4096 tiles = 16,777,216 scores.
+// synchronisation an allocation implies is not acceptable.  For them the per-tile counts and offsets and the decision
+// bits of the three-pass compaction live in arrays that are part of the library image: 2 x 1024 ints + 1024 x 1024
+// 16-bit words = 2 MB + 8 KB of device memory on every GPU that loads the library, held until the process exits.
+// That bounds the call at 1024 tiles = 16,777,216 scores.
 //
 // In host code the name `g_select_scratch` is only a stand-in for the symbol; the address a kernel may use comes from
 // cudaGetSymbolAddress, asked once per device with that device current (the first call on a device does this; make
@@ -169,8 +222,9 @@ cudaError_t launch_select_large(const float* scores, long long n, float tau, int
 // needs clearing), and two calls that overlap on the GPU (different streams) race on it.
 namespace dare {
 namespace {
-constexpr int kStaticTiles = 4096;
-static __device__ __align__(256) int g_select_scratch[2 * kStaticTiles];
+constexpr int kStaticTiles = 1024;
+// [0, 2 * tiles) ints: counts, offsets; behind them the decision words
+static __device__ __align__(256) int g_select_scratch[2 * kStaticTiles + kStaticTiles * kThreads / 2];
 constexpr int kMaxDevices = 64;
 int* g_select_scratch_addr[kMaxDevices] = {};
 std::mutex g_select_scratch_mutex;
@@ -204,7 +258,9 @@ extern "C" dare_status_t dare_select_compact_static(const float* scores, int64_t
   int* scratch = nullptr;
   if (dare::static_scratch_for_current_device(&scratch) != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
   cudaError_t e = dare::launch_select_large(scores, n_tokens, threshold, idx, count, scratch,
-                                            scratch + dare::kStaticTiles, (cudaStream_t)cuda_stream);
+                                            scratch + dare::kStaticTiles,
+                                            reinterpret_cast<unsigned short*>(scratch + 2 * dare::kStaticTiles),
+                                            (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
   return DARE_OK;
 }
