@@ -26,7 +26,7 @@ def _scores(n, seed):
     return s
 
 
-@pytest.mark.parametrize("n", [0, 1, 2, 3, 5, 4095, 4096, 4097, 16383, 16384, 16385, 16387, 100_003, 1 << 20, (1 << 22) + 12345])
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 5, 4095, 4096, 4097, 16383, 16384, 16385, 16387, 100_003, 1 << 20, (1 << 22) + 12345, (1 << 24) + 20_000])
 def test_select_compact_matches_the_predicate(dare, n):
     import torch
     s = _scores(n, n % 97)
