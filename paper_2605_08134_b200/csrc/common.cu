@@ -264,17 +264,40 @@ template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, 
 // and a scan over the warp totals give each thread its place; the staleness counters of Sec. 4 and the start of
 // every sequence's slice of the list come out of the same pass.  One CTA walks the chunks, which keeps the list
 // ordered without any inter-CTA hand-off (T <= a few 10^4 per layer step).
+// With more than one chunk the launch has one CTA per chunk, and none waits for another: a CTA first counts the
+// refreshed tokens of the chunks before its own from their scores (a few 16-byte loads per thread, from the L2), which
+// is where its part of the list starts.
 constexpr int kSelPerThread = 4;
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
                                                       int* __restrict__ batch_off, int* __restrict__ delta) {
   __shared__ int warp_tot[32];
+  __shared__ int before_chunk;
+  if (threadIdx.x == 0) before_chunk = 0;
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kChunk = 1024 * kSelPerThread;
+  const int chunk0 = (int)blockIdx.x * kChunk;            // this CTA's chunk: tokens [chunk0, chunk0 + kChunk)
   int base = 0;
-  for (int start = 0; start < T; start += 1024 * kSelPerThread) {
+  if (blockIdx.x > 0) {
+    if (select_all) {
+      base = chunk0;
+    } else {
+      __syncthreads();
+      int c = 0;
+      for (int i = (int)threadIdx.x * 4; i < chunk0; i += kChunk) {     // whole chunks: no tail, 16-byte aligned
+        const float4 v = *reinterpret_cast<const float4*>(scores + i);
+        c += (!(v.x <= tau) ? 1 : 0) + (!(v.y <= tau) ? 1 : 0) + (!(v.z <= tau) ? 1 : 0) + (!(v.w <= tau) ? 1 : 0);
+      }
+      c = __reduce_add_sync(0xffffffffu, c);
+      if (lane == 0 && c != 0) atomicAdd(&before_chunk, c);
+      __syncthreads();
+      base = before_chunk;
+    }
+  }
+  for (int start = chunk0; start < chunk0 + kChunk && start < T; start += kChunk) {
     const int t0 = start + threadIdx.x * kSelPerThread;
     // all loads of the chunk first (scores and staleness counters): one memory round trip
     float sc[kSelPerThread];
@@ -327,7 +350,7 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
     base += total;
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
     *count = base;
     batch_off[g.batch] = base;
   }
@@ -390,7 +413,8 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
   if (g.tokens() <= 2048)
     launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta);
   else
-    launch_pdl(select_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta);
+    launch_pdl(select_kernel, dim3((g.tokens() + 1024 * kSelPerThread - 1) / (1024 * kSelPerThread)), dim3(1024), 0, st, 1,
+               scores, tau, all, g, idx, count, batch_off, delta);
 }
 
 // ------------------------------------------------------------------------------------------------ reused rows
