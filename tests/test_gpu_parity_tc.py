@@ -297,3 +297,26 @@ def test_step_replays_from_a_cuda_graph(dare, mode):
     for l in (eager, graphed):
         assert l.status() == 0
         l.close()
+
+
+def test_selection_across_chunks_and_threshold_extremes(dare):
+    """5700 tokens (three sequences of 1900): the selection launch has two CTAs, the second one starting its part of
+    the list at the first one's count.  Ordinary threshold, a negative one (everything refreshed) and +inf (nothing)."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=256, n_heads=2, batch=3, seq=1900, prompt=900)
+    w = wl.make_weights(shape, 41)
+    hs = wl.HiddenStream(shape, 41)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    for n, tau in ((300, 0.1), (40, -1.0), (500, float("inf")), (1900, 0.1), (0, 0.1)):
+        ch = wl.uniform_positions(hs.rng, shape, n)
+        parity.compare_step(g, o, hs.advance(ch), 3, tau, shape)
+        sel = g.last_selection(3, 1900)
+        if tau == 0.1:
+            np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
+        elif tau < 0:
+            assert sel["count"] == 5700
+        else:
+            assert sel["count"] == 0
+    assert g.status() == 0
+    g.close()
