@@ -271,7 +271,8 @@ def run_ours(args):
 
     # ---- the same steps replayed from a CUDA graph (two steps of every layer instance captured once): what a caller
     # gains by taking the launches off the host.  Diagnostics only; `value` stays the stream-launched number.
-    graph_ms_per_step = None
+    # (no collective inside the try: a rank whose capture failed must still meet the others at the same barriers)
+    graph_local = -1.0
     try:
         prime(mode)
         one_pass(max(args.warmup, 3), mode)
@@ -284,20 +285,25 @@ def run_ours(args):
         for _ in range(3):
             graph.replay()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
+        torch.cuda.synchronize()
         ev0.record(stream)
         for _ in range(reps):
             graph.replay()
         ev1.record(stream)
         torch.cuda.synchronize()
-        graph_ms_per_step = distrib.max_over_ranks(ev0.elapsed_time(ev1), dist, device) / (reps * n_cap)
         sel = layers[0].last_selection(shape.batch, shape.seq)
         assert sel["count"] == expect and all(l.status() == 0 for l in layers)
+        graph_local = ev0.elapsed_time(ev1) / (reps * n_cap)
         del graph
     except Exception as e:                # diagnostics only
         print(f"graph replay not measured: {e!r}", file=sys.stderr)
-        graph_ms_per_step = None
+        graph_local = -1.0
     barrier()
+    # slowest rank's figure; dropped if any rank has none
+    graph_failed = distrib.max_over_ranks(1.0 if graph_local < 0 else 0.0, dist, device) > 0
+    graph_ms_per_step = distrib.max_over_ranks(graph_local, dist, device)
+    if graph_failed:
+        graph_ms_per_step = None
 
     # ---- end to end through the host-buffer entry point (pinned host x and y, copies inside the timed region)
     prime(mode)
