@@ -118,7 +118,13 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
  * The first step after create/reset must have pos_begin = 0; it fixes batch and the cached extent
  * kv_len = seq_act.  Later steps may cover any window inside [0, kv_len) and must keep the same batch
  * (DARE_ERR_STATE otherwise).  Rows outside the window keep their cached K/V/O; attention always spans
- * keys [0, kv_len). */
+ * keys [0, kv_len).
+ * The call only enqueues: it neither synchronises nor allocates, and every data-dependent decision (the refresh set
+ * and its size) is taken on the device.  It may therefore be captured into a CUDA graph, once a call of the same shape
+ * and mode has run outside a capture (the first use of a kernel sets its attributes).  A captured step replays the
+ * kernels chosen for the host-side state at capture time (first step or not, batch, kv_len), so replay it in that
+ * state only; several steps per graph are worth more than one (a graph's first kernel cannot overlap the kernel
+ * before it). */
 dare_status_t dare_layer_step(dare_layer_t* layer, const void* x, int batch, int seq_act, int pos_begin,
                               int mode, float threshold, void* y, void* cuda_stream);
 
