@@ -153,12 +153,12 @@ __global__ void __launch_bounds__(kThreads) tile_scatter_kernel(const unsigned s
                                                                 int* __restrict__ idx) {
   __shared__ unsigned long long warp_sums[32];
   __shared__ unsigned long long total;
-  const unsigned bits = flags[(size_t)blockIdx.x * kThreads + threadIdx.x];      // written two kernels back
+  ptx::pdl_wait();                         // before any read: decisions (two kernels back) and offsets (one back)
+  const unsigned bits = flags[(size_t)blockIdx.x * kThreads + threadIdx.x];
   unsigned long long packed = 0;
 #pragma unroll
   for (int k = 0; k < kVecs; ++k) packed |= (unsigned long long)__popc((bits >> (4 * k)) & 0xfu) << (16 * k);
   const unsigned long long ex = block_exclusive_scan<unsigned long long>(packed, warp_sums, &total);
-  ptx::pdl_wait();                                                               // the tile offsets: one kernel back
   const long long base = (long long)blockIdx.x * kTile;
   int out = tile_offsets[blockIdx.x];
   const unsigned long long tot = total;
