@@ -146,7 +146,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // set before spending anything on set-up.
   if (p.idx != nullptr && tile > 0) {
     pdl_wait();
-    if (p.batch_off[b] + tile * BQ >= p.batch_off[b + 1]) return;
+    if (__ldcg(p.batch_off + b) + tile * BQ >= __ldcg(p.batch_off + b + 1)) return;
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -169,12 +169,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // The previous kernel in the stream (the K/V projection) writes the K and V caches only.  The queries and the
   // refresh set come from kernels further back, which are complete by the time any CTA of this grid runs (every
   // kernel lets its successor start only after its own wait): they are read without waiting, so that the gather
-  // of the Q tile overlaps the projection's tail.  Warp 0 waits right away and starts the first K and V blocks.
+  // of the Q tile overlaps the projection's tail.  Those reads go to the L2 (ld.global.cg): ahead of the wait this
+  // SM's L1 may still hold the lines an earlier step's CTA read from the same addresses.  Warp 0 waits right away and starts the first K and V blocks.
   // ---- rows of this tile (uniform over the CTA)
   int row0 = 0, rows_valid = 0;
   bool active = true;
   if (p.idx != nullptr) {
-    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
+    const int lo = __ldcg(p.batch_off + b), hi = __ldcg(p.batch_off + b + 1);
     row0 = lo + tile * BQ;
     active = row0 < hi;
     rows_valid = min(BQ, hi - row0);
@@ -218,13 +219,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     for (int k = 0; k < QU; ++k) {
       const int u = u0 + k * kGather, r = u >> 4;              // 16 units of 8 bf16 per row
       tok[k] = -1;
-      if (u < BQ * 16 && r < rows_valid) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
+      if (u < BQ * 16 && r < rows_valid) tok[k] = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
       const int unit = (u0 + k * kGather) & 15;
       qv[k] = make_uint4(0u, 0u, 0u, 0u);
-      if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
+      if (tok[k] >= 0) qv[k] = __ldcg(reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8));
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
@@ -438,7 +439,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // normalise, store
       const float inv = 1.f / l_row;
       if (r < rows_valid) {
-        const int t = p.idx ? p.idx[row0 + r] : row0 + r;
+        const int t = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
         __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + st * 64;
 #pragma unroll
         for (int i = 0; i < 64; ++i) acc[i] *= inv;
@@ -511,7 +512,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         lsum = fmaf(w, lz[s2 + 1], lsum);
       }
       const float inv = 1.f / lsum;
-      const int t = p.idx ? p.idx[row0 + r] : row0 + r;
+      const int t = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + 4 * lane;
       __nv_bfloat162 lo2 = __floats2bfloat162_rn(o.x * inv, o.y * inv), hi2 = __floats2bfloat162_rn(o.z * inv, o.w * inv);
       uint2 packed;
@@ -600,7 +601,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   }
   if (p.idx != nullptr && tile > 0) {
     pdl_wait();
-    if (p.batch_off[b] + tile * kPairRows >= p.batch_off[b + 1]) return;
+    if (__ldcg(p.batch_off + b) + tile * kPairRows >= __ldcg(p.batch_off + b + 1)) return;
   }
   // diagnostics: [0] first CTA's start, [1] its set-up done, [3] its key loop done, [4] its end; over the CTAs with
   // work: [5] latest start, [6] latest end, [7] their number
@@ -631,7 +632,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   int row0 = 0, rows_all = 0;
   bool active = true;
   if (p.idx != nullptr) {
-    const int lo = p.batch_off[b], hi = p.batch_off[b + 1];
+    const int lo = __ldcg(p.batch_off + b), hi = __ldcg(p.batch_off + b + 1);
     row0 = lo + tile * kPairRows;
     active = row0 < hi;
     rows_all = min(kPairRows, hi - row0);
@@ -673,13 +674,13 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int k = 0; k < QU; ++k) {
       const int u = u0 + k * kGather, r = u >> 4;
       tok[k] = -1;
-      if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? p.idx[row0 + r] : row0 + r;
+      if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
       const int unit = (u0 + k * kGather) & 15;
       qv[k] = make_uint4(0u, 0u, 0u, 0u);
-      if (tok[k] >= 0) qv[k] = *reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8);
+      if (tok[k] >= 0) qv[k] = __ldcg(reinterpret_cast<const uint4*>(p.q + (size_t)tok[k] * g.d + h * HD + unit * 8));
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
@@ -855,7 +856,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const bool ok = r < rows_valid;
       const float inv = 1.f / l;
       const int rr = st * BQ + (ok ? r : 0);
-      const int t = p.idx ? p.idx[row0 + rr] : row0 + rr;
+      const int t = p.idx ? __ldcg(p.idx + row0 + rr) : row0 + rr;
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
