@@ -79,3 +79,28 @@ def test_drift_scores_match_oracle(dare, rows, hd):
     np.testing.assert_allclose(out.cpu().numpy(), want, rtol=0, atol=2e-6)
     assert out[0].item() == 1.0
     assert dare.dare_drift_scores(ad.data_ptr(), bd.data_ptr(), rows, 6, out.data_ptr()) == dare.ERR_SHAPE
+
+
+@pytest.mark.parametrize("n", [300_000, (1 << 24) + 20_000])
+def test_select_compact_alternating_thresholds_on_one_scratch(dare, n):
+    """Calls in a row on the same scratch whose decisions differ completely (nothing refreshed, then the ordinary set,
+    then everything): a pass that read what an earlier call left at the same addresses would show here."""
+    import torch
+    s = _scores(n, 5)
+    sd = torch.from_numpy(s).cuda()
+    idx = torch.empty(n, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(1, dtype=torch.int32, device="cuda")
+    nb = dare.dare_select_compact_scratch_bytes(n)
+    scratch = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    want = {tau: np.nonzero(orc.refresh_mask(s, tau))[0] for tau in (float("inf"), 0.1, -1.0)}
+    for rep in range(4):
+        for tau in (float("inf"), 0.1, -1.0):
+            idx.fill_(-1)
+            assert dare.dare_select_compact(sd.data_ptr(), n, tau, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(),
+                                            nb, stream) == 0
+            torch.cuda.synchronize()
+            k = int(cnt.item())
+            assert k == len(want[tau]), (rep, tau)
+            assert np.array_equal(idx[:k].cpu().numpy(), want[tau]), (rep, tau)
+            assert bool((idx[k:] == -1).all())
