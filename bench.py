@@ -534,14 +534,24 @@ def run_micro(args):
     def compact():
         s = bufs[turn[0] & 3]
         turn[0] += 1
-        dare.dare_select_compact(s.data_ptr(), n, 0.1, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(), nb, st)
+        dare.dare_select_compact(s.data_ptr(), n, 0.1, idx.data_ptr(), cnt.data_ptr(), scratch.data_ptr(), nb,
+                                 torch.cuda.current_stream(dev).cuda_stream)
 
-    t = time_it(compact)
+    t_stream = time_it(compact)
+    # the call is three short launches: issued one by one the host sets the pace, so the figure reported is that of
+    # the same calls replayed from a CUDA graph (four calls, one per score array); the stream-launched one is kept
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(dev)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(4):
+            compact()
+    t = time_it(graph.replay) / 4
     k = int(cnt.item())
     algo = 4.0 * n + 4.0 * k            # scores in, index list out
     out["kernels"].append({"kernel": "select_compact", "tokens": n, "refreshed": k, "us": round(t * 1e6, 1),
                            "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3),
                            "l2": "four score arrays in rotation (256 MB)",
+                           "timing": "four calls per CUDA graph, replayed", "us_stream_launched": round(t_stream * 1e6, 1),
                            "bytes_moved": 4.0 * n + 2.0 * (n / 8.0) + 4.0 * k})   # + decision bits out and back in
     print(json.dumps(out))
 

@@ -586,7 +586,7 @@ dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float t
   const size_t half = align_up((size_t)select_large_tiles(n_tokens) * sizeof(int));
   int* counts = (int*)scratch;
   int* offsets = (int*)((char*)scratch + half);
-  unsigned short* flags = (unsigned short*)((char*)scratch + 2 * half);
+  unsigned* flags = (unsigned*)((char*)scratch + 2 * half);
   CUDA_TRY(launch_select_large(scores, n_tokens, threshold, idx, count, counts, offsets, flags,
                                (cudaStream_t)cuda_stream));
   return DARE_OK;

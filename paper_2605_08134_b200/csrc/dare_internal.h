@@ -101,7 +101,7 @@ void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* 
 int select_large_tiles(long long n);
 cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, int hd, float* scores, cudaStream_t st);
 cudaError_t launch_select_large(const float* scores, long long n, float tau, int* idx, int* count, int* tile_counts,
-                                int* tile_offsets, unsigned short* flags, cudaStream_t st);
+                                int* tile_offsets, unsigned* flags, cudaStream_t st);
 size_t select_large_flag_bytes(long long n);   // bytes of the decision words for n scores
 
 // ---- SIMT path (simt.cu) ----------------------------------------------------------------------------------

@@ -2,7 +2,7 @@
 // the same arithmetic as inside the layer step, organised for HBM bandwidth.
 //   drift score (Sec. 3.1): one warp per row, 16-byte loads of both query rows, shuffle reduction
 //   compaction (Eq. 2, complement): three passes over tiles of 16384 scores; the scores are read once
-//     (1) per-tile count of refreshed tokens and the decisions themselves, one bit per score -> scratch
+//     (1) per-tile count of refreshed tokens and the decisions themselves, a plain bit array -> scratch
 //     (2) exclusive scan of the tile counts (one CTA) -> scratch, total -> *count
 //     (3) per-tile compaction from the decision bits, written at the tile's offset: ascending index list
 // No CTA waits for another; the order of the list does not depend on scheduling.  Passes 2 and 3 are launched
@@ -18,6 +18,7 @@ namespace dare {
 namespace {
 constexpr int kThreads = 1024, kVecs = 4;
 constexpr int kTile = kThreads * kVecs * 4;     // 16384 scores per CTA: four 16-byte vectors per thread
+constexpr int kTileWords = kTile / 32;          // 512 words of decision bits per tile
 
 __global__ void __launch_bounds__(256) drift_score_kernel(const float* __restrict__ a, const float* __restrict__ b,
                                                           long long rows, int hd, float* __restrict__ scores) {
@@ -49,8 +50,8 @@ __global__ void __launch_bounds__(256) drift_score_kernel(const float* __restric
 
 // refreshed <=> !(s <= tau): a NaN score refreshes.
 // Thread t of a tile owns the four 16-byte vectors k = 0..3 at scores[base + (k * 1024 + t) * 4 ...]: every load
-// instruction of a warp covers 512 contiguous bytes, and all four are in flight before the first is used.  Its 16
-// decisions are one 16-bit word, bit 4k + j <-> element j of vector k.
+// instruction of a warp covers 512 contiguous bytes, and all four are in flight before the first is used.  Returns
+// its 16 decisions, bit 4k + j <-> element j of vector k.
 __device__ __forceinline__ unsigned tile_flags(const float* __restrict__ scores, long long n, long long base, float tau) {
   float4 v[kVecs];
   bool full[kVecs];
@@ -82,8 +83,7 @@ __device__ __forceinline__ unsigned tile_flags(const float* __restrict__ scores,
   return bits;
 }
 
-// exclusive prefix of `v` over the 1024 threads of the CTA; *total = sum.  T: int, or four 16-bit counts packed into
-// 64 bits (no field of a sum over one tile can carry: it is at most 4096).
+// exclusive prefix of `v` over the threads of the CTA (whole warps, at most 32 of them); *total = sum
 template <typename T>
 __device__ __forceinline__ T block_exclusive_scan(T v, T* warp_sums, T* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -96,7 +96,7 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* warp_sums, T* total) {
   if (lane == 31) warp_sums[warp] = inc;
   __syncthreads();
   if (warp == 0) {
-    const T w = warp_sums[lane];
+    const T w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : T(0);
     T winc = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -110,18 +110,30 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* warp_sums, T* total) {
   return warp_sums[warp] + inc - v;
 }
 
-// pass 1: the only pass that reads the scores.  Leaves every thread's 16 decisions and the tile's count.
+// pass 1: the only pass that reads the scores.  Leaves the decisions as a plain bit array (bit i of the array <->
+// score i) and the tile's count.  For one vector index k the 32 lanes of a warp hold the decisions on 128 consecutive
+// scores, four bits each: eight lanes' nibbles make one 32-bit word of the array, put together with three shuffles.
 __global__ void __launch_bounds__(kThreads) tile_flag_kernel(const float* __restrict__ scores, long long n, float tau,
                                                              int* __restrict__ tile_counts,
-                                                             unsigned short* __restrict__ flags) {
+                                                             unsigned* __restrict__ flags) {
   __shared__ int total;
   ptx::pdl_launch_dependents();            // the scan's CTA may take its place now; it waits for this grid to complete
   if (threadIdx.x == 0) total = 0;
   __syncthreads();
   const unsigned bits = tile_flags(scores, n, (long long)blockIdx.x * kTile, tau);
-  flags[(size_t)blockIdx.x * kThreads + threadIdx.x] = (unsigned short)bits;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned* tile_words = flags + (size_t)blockIdx.x * kTileWords;
+#pragma unroll
+  for (int k = 0; k < kVecs; ++k) {
+    unsigned v = ((bits >> (4 * k)) & 0xfu) << (4 * (lane & 7));
+    v |= __shfl_xor_sync(0xffffffffu, v, 1);
+    v |= __shfl_xor_sync(0xffffffffu, v, 2);
+    v |= __shfl_xor_sync(0xffffffffu, v, 4);
+    // scores [(k * 1024 + 32 * warp + 8 * w) * 4, + 32) of the tile, w = lane / 8
+    if ((lane & 7) == 0) tile_words[k * (kThreads / 8) + warp * 4 + (lane >> 3)] = v;
+  }
   const int c = __reduce_add_sync(0xffffffffu, __popc(bits));
-  if ((threadIdx.x & 31) == 0) atomicAdd(&total, c);
+  if (lane == 0) atomicAdd(&total, c);
   __syncthreads();
   if (threadIdx.x == 0) tile_counts[blockIdx.x] = total;
 }
@@ -145,39 +157,29 @@ __global__ void __launch_bounds__(kThreads) tile_scan_kernel(const int* __restri
   if (threadIdx.x == 0) *count = base;
 }
 
-// pass 3: from the decisions alone (2 bytes per thread instead of 64 bytes of scores).  The list is ascending, so a
-// tile's order is vector k first, then thread, then element: one scan of the four per-vector counts packed into one
-// 64-bit word gives every thread its place among the threads for each k; the totals of the lower k come before.
-__global__ void __launch_bounds__(kThreads) tile_scatter_kernel(const unsigned short* __restrict__ flags,
-                                                                const int* __restrict__ tile_offsets,
-                                                                int* __restrict__ idx) {
-  __shared__ unsigned long long warp_sums[32];
-  __shared__ unsigned long long total;
+// pass 3: from the decision bits alone (4 bytes per thread instead of 128 bytes of scores).  One thread per word of
+// 32 consecutive scores, 512 threads per tile: one scan of the words' popcounts places every thread, which then
+// writes the indices of its set bits, ascending, at consecutive places.
+__global__ void __launch_bounds__(kTileWords) tile_scatter_kernel(const unsigned* __restrict__ flags,
+                                                                  const int* __restrict__ tile_offsets,
+                                                                  int* __restrict__ idx) {
+  __shared__ int warp_sums[32];
+  __shared__ int total;
   ptx::pdl_wait();                         // before any read: decisions (two kernels back) and offsets (one back)
-  const unsigned bits = flags[(size_t)blockIdx.x * kThreads + threadIdx.x];
-  unsigned long long packed = 0;
-#pragma unroll
-  for (int k = 0; k < kVecs; ++k) packed |= (unsigned long long)__popc((bits >> (4 * k)) & 0xfu) << (16 * k);
-  const unsigned long long ex = block_exclusive_scan<unsigned long long>(packed, warp_sums, &total);
-  const long long base = (long long)blockIdx.x * kTile;
+  unsigned word = flags[(size_t)blockIdx.x * kTileWords + threadIdx.x];
   int out = tile_offsets[blockIdx.x];
-  const unsigned long long tot = total;
-#pragma unroll
-  for (int k = 0; k < kVecs; ++k) {
-    int o = out + (int)((ex >> (16 * k)) & 0xffffu);
-    const unsigned b = (bits >> (4 * k)) & 0xfu;
-    const int i0 = (int)(base + ((long long)k * kThreads + threadIdx.x) * 4);
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (b & (1u << j)) idx[o++] = i0 + j;
-    out += (int)((tot >> (16 * k)) & 0xffffu);
+  out += block_exclusive_scan<int>(__popc(word), warp_sums, &total);
+  const int i0 = (int)((long long)blockIdx.x * kTile) + (int)threadIdx.x * 32;
+  while (word != 0u) {
+    idx[out++] = i0 + __ffs((int)word) - 1;
+    word &= word - 1u;
   }
 }
 
 }  // namespace
 
 int select_large_tiles(long long n) { return (int)((n + kTile - 1) / kTile); }
-size_t select_large_flag_bytes(long long n) { return (size_t)select_large_tiles(n) * kThreads * sizeof(unsigned short); }
+size_t select_large_flag_bytes(long long n) { return (size_t)select_large_tiles(n) * kTileWords * sizeof(unsigned); }
 
 cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, int hd, float* scores,
                                 cudaStream_t st) {
@@ -188,16 +190,16 @@ cudaError_t launch_drift_scores(const float* a, const float* b, long long rows, 
   return cudaGetLastError();
 }
 
-// tile_counts and tile_offsets: device arrays of select_large_tiles(n) ints each; flags: 1024 16-bit words per tile
+// tile_counts and tile_offsets: device arrays of select_large_tiles(n) ints each; flags: 512 32-bit words per tile
 cudaError_t launch_select_large(const float* scores, long long n, float tau, int* idx, int* count, int* tile_counts,
-                                int* tile_offsets, unsigned short* flags, cudaStream_t st) {
+                                int* tile_offsets, unsigned* flags, cudaStream_t st) {
   const int tiles = select_large_tiles(n);
   if (tiles == 0) return cudaMemsetAsync(count, 0, sizeof(int), st);
   tile_flag_kernel<<<tiles, kThreads, 0, st>>>(scores, n, tau, tile_counts, flags);
   cudaError_t e = launch_pdl(tile_scan_kernel, dim3(1), dim3(kThreads), 0, st, 1, (const int*)tile_counts, tiles,
                              tile_offsets, count);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(tile_scatter_kernel, dim3(tiles), dim3(kThreads), 0, st, 1, (const unsigned short*)flags,
+  e = launch_pdl(tile_scatter_kernel, dim3(tiles), dim3(kTileWords), 0, st, 1, (const unsigned*)flags,
                  (const int*)tile_offsets, idx);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
@@ -211,8 +213,8 @@ cudaError_t launch_select_large(const float* scores, long long n, float tau, int
 // Some hosts of this library hand all of the device's memory to one arena at start-up and forbid every later
 // cudaMalloc (an inference server with a fixed memory plan), or sit in a latency-critical loop where the device-wide
 // synchronisation an allocation implies is not acceptable.  For them the per-tile counts and offsets and the decision
-// bits of the three-pass compaction live in arrays that are part of the library image: 2 x 1024 ints + 1024 x 1024
-// 16-bit words = 2 MB + 8 KB of device memory on every GPU that loads the library, held until the process exits.
+// bits of the three-pass compaction live in arrays that are part of the library image: 2 x 1024 ints + 1024 x 512
+// 32-bit words = 2 MB + 8 KB of device memory on every GPU that loads the library, held until the process exits.
 // That bounds the call at 1024 tiles = 16,777,216 scores.
 //
 // In host code the name `g_select_scratch` is only a stand-in for the symbol; the address a kernel may use comes from
@@ -224,7 +226,7 @@ namespace dare {
 namespace {
 constexpr int kStaticTiles = 1024;
 // [0, 2 * tiles) ints: counts, offsets; behind them the decision words
-static __device__ __align__(256) int g_select_scratch[2 * kStaticTiles + kStaticTiles * kThreads / 2];
+static __device__ __align__(256) int g_select_scratch[2 * kStaticTiles + kStaticTiles * kTileWords];
 constexpr int kMaxDevices = 64;
 int* g_select_scratch_addr[kMaxDevices] = {};
 std::mutex g_select_scratch_mutex;
@@ -259,7 +261,7 @@ extern "C" dare_status_t dare_select_compact_static(const float* scores, int64_t
   if (dare::static_scratch_for_current_device(&scratch) != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
   cudaError_t e = dare::launch_select_large(scores, n_tokens, threshold, idx, count, scratch,
                                             scratch + dare::kStaticTiles,
-                                            reinterpret_cast<unsigned short*>(scratch + 2 * dare::kStaticTiles),
+                                            reinterpret_cast<unsigned*>(scratch + 2 * dare::kStaticTiles),
                                             (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; }
   return DARE_OK;
