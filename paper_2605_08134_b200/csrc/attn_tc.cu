@@ -171,6 +171,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // kernel lets its successor start only after its own wait): they are read without waiting, so that the gather
   // of the Q tile overlaps the projection's tail.  Those reads go to the L2 (ld.global.cg): ahead of the wait this
   // SM's L1 may still hold the lines an earlier step's CTA read from the same addresses.  Warp 0 waits right away and starts the first K and V blocks.
+  // (unless the step's launch order puts their producer right before this kernel: then everybody waits first)
+  if (p.wait_first) pdl_wait();
   // ---- rows of this tile (uniform over the CTA)
   int row0 = 0, rows_valid = 0;
   bool active = true;
@@ -628,6 +630,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   }
   // (as in the kernel above: queries and refresh set are read without waiting for the K/V projection; warp 0 waits
   // right away and starts the first key blocks, the other warps gather the Q tiles first)
+  if (p.wait_first) pdl_wait();
   // ---- rows of the two tiles (uniform over the CTA)
   int row0 = 0, rows_all = 0;
   bool active = true;

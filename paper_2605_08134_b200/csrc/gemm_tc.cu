@@ -218,7 +218,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
   }
-  pdl_wait();
+  if (!p.wait_at_end) pdl_wait();
   pdl_launch_dependents();
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
@@ -251,7 +251,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
-  const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+  // (a Q projection without a score buffer leaves score and stored query alone: the step took them from the sliver)
+  const bool score_tile = (EPI == EPI_Q) && p.scores != nullptr && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
   RowBatch<RB> rb;
 
   if (active) {
@@ -565,6 +566,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
   }
   tc_fence_before();
+  // a launch that ran beside its predecessor leaves only once that one is complete: the next kernel's wait on this
+  // grid then covers both
+  if (p.wait_at_end) pdl_wait();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
   // (nor frees tensor memory its MMA partner may still read through)
   if (splits > 1 || PAIR) cluster_sync_all(); else __syncthreads();

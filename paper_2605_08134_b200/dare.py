@@ -276,7 +276,8 @@ class Layer:
     No arithmetic happens here.  `x`/`y` are torch CUDA tensors (or pinned host tensors for `step_host`).
     """
 
-    def __init__(self, shape, weights: dict, device="cuda:0", kernel_path=PATH_AUTO, max_batch=None, max_seq=None):
+    def __init__(self, shape, weights: dict, device="cuda:0", kernel_path=PATH_AUTO, max_batch=None, max_seq=None,
+                 score_head=0):
         import numpy as np
         import torch
         self.torch = torch
@@ -286,7 +287,7 @@ class Layer:
         self.max_batch = max_batch or shape.batch
         self.max_seq = max_seq or shape.seq
         self.cfg = make_config(shape.d_model, shape.n_heads, shape.head_dim, self.max_batch, self.max_seq,
-                               shape.rope_theta, shape.rms_eps, shape.dtype, 0, kernel_path)
+                               shape.rope_theta, shape.rms_eps, shape.dtype, score_head, kernel_path)
         self._w = {}
         for k in ("w_q", "w_k", "w_v", "w_o"):
             v = weights[k]

@@ -6,7 +6,14 @@ from paper_2605_08134_b200 import workloads as wl
 
 TOL_F32 = 1e-4     # fp32 path: max-abs and RMS error, relative to max(1, RMS(oracle))
 TOL_BF16 = 2e-2    # bf16 path
-SCORE_ATOL = {wl.DTYPE_F32: 2e-6, wl.DTYPE_BF16: 5e-3}   # diagnostic only; bf16 x_norm rounding moves a cosine by ~2^-8/sqrt(head_dim)
+# Scores against the plain fp64 oracle.  fp32 path: fp32 noise of 1 - cos.  bf16 path: the score comes from fp32
+# accumulators over a bf16 x_norm, whose rounding alone (relative 2^-9..2^-8 per element, independent over the
+# head_dim components of the two queries) moves the cosine of two unrelated queries by up to 6.2e-4 over the 67 redrawn
+# tokens of the LLaDA-shaped layer (fp64 evaluation with only that rounding: tests/test_rounding_pins.py); reused tokens
+# (score ~1e-6) move by ~1e-6.  Largest deviation of a GPU score from the plain oracle's over every comparison of this
+# suite: 1.26e-3 (a layer of width 128; 1.09e-3 at head_dim 128).  The gate is below twice that maximum.
+# What decides the index set is the side of tau, which the margin tests check against both evaluations.
+SCORE_ATOL = {wl.DTYPE_F32: 2e-6, wl.DTYPE_BF16: 2e-3}
 MARGIN = 1e-3      # every oracle score must be at least this far from tau for the index set to be bit-exact
 
 
@@ -14,7 +21,9 @@ def tol_of(dtype):
     return TOL_BF16 if dtype == wl.DTYPE_BF16 else TOL_F32
 
 
-def assert_close(name, got, want, tol, max_factor=1.0):
+def assert_close(name, got, want, tol, max_factor=1.0, rel_rms=None):
+    """Both max|g - o| and RMS(g - o) within tol * max(1, RMS(o)) (max-abs gate times max_factor); with rel_rms also
+    RMS(g - o) <= rel_rms * RMS(o), which is the tighter gate wherever RMS(o) is far below 1."""
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape, (name, got.shape, want.shape)
@@ -26,13 +35,15 @@ def assert_close(name, got, want, tol, max_factor=1.0):
     rms = float(np.sqrt(np.mean(err ** 2))) if err.size else 0.0
     assert max_abs <= max_factor * bound, f"{name}: max-abs {max_abs:.3e} > {max_factor * bound:.3e} (rms(o)={rms_o:.3e})"
     assert rms <= bound, f"{name}: rms {rms:.3e} > {bound:.3e}"
+    if rel_rms is not None:
+        assert rms <= rel_rms * rms_o, f"{name}: rms {rms:.3e} > {rel_rms:.1e} * rms(o) = {rel_rms * rms_o:.3e}"
     return max_abs, rms, rms_o
 
 
-def oracle_layer(shape, w, max_batch=None, max_seq=None):
+def oracle_layer(shape, w, max_batch=None, max_seq=None, score_head=0):
     return orc.OracleLayer(shape.d_model, shape.n_heads, shape.head_dim, max_batch or shape.batch,
                            max_seq or shape.seq, shape.rope_theta, shape.rms_eps,
-                           w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"])
+                           w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"], score_head=score_head)
 
 
 def to_device(x, shape, device="cuda:0"):
@@ -71,15 +82,18 @@ def compare_step(glayer, olayer, x, mode, tau, shape, pos_begin=0, check_caches=
         assert np.isinf(sel["scores"]).all()
     else:
         np.testing.assert_allclose(sel["scores"], olayer.last_scores, rtol=0, atol=SCORE_ATOL[shape.dtype])
-    res = {"y": assert_close("y", yg.float().cpu().numpy(), yo, tol)}
+    # y also relative to its own size: RMS(o) is 0.009 at the tiny fp32 layer and 0.24 at the LLaDA-shaped one
+    res = {"y": assert_close("y", yg.float().cpu().numpy(), yo, tol, rel_rms=tol)}
     if check_caches:
         kv_len = olayer.kv_len
         c = glayer.read_caches(B, kv_len)
         # Caches in bf16 storage: the max-abs gate is doubled, the RMS gate is not.  K and V reach |v| ~ 6.5, where
         # half a bf16 ulp is already 1.6e-2, on top of the error carried in from the bf16 x_norm operand; in the
         # O cache the bf16 operands of the logits move single softmax weights by ~1 % and a few of the millions
-        # of elements by ~2.4e-2 (an fp64 run with only those operands rounded gives the same figure).  The layer
-        # output y keeps the plain gate.
+        # of elements by ~2.4e-2.  tests/test_rounding_pins.py evaluates the oracle's arithmetic in fp64 with only
+        # those stored tensors rounded and pins the figures (K 2.55e-2, V 2.50e-2, O 2.42e-2 at the LLaDA-shaped
+        # layer): the storage format alone passes the plain gate, so the gate is twice it.  The layer output y keeps
+        # the plain gate.
         mf = 2.0 if shape.dtype == wl.DTYPE_BF16 else 1.0
         res["k"] = assert_close("k_cache", c["k"], olayer.k_cache[:B, :kv_len], tol, max_factor=mf)
         res["v"] = assert_close("v_cache", c["v"], olayer.v_cache[:B, :kv_len], tol, max_factor=mf)

@@ -31,9 +31,11 @@ def _weights_gpu(shape, seed, torch):
 
 
 def test_config3_dare_o_batched_clustered_steps(dare):
-    """Config 3: batch 8, seq 1024, mode O, 113 clustered + 20 scattered positions changed per sequence and step.
-    All 8 sequences run on the GPU; sequences 0 and 5 are checked against batch-1 oracles for 4 consecutive steps;
-    index sets of all sequences are checked against the plan every step."""
+    """Config 3: batch 8, seq 1024, mode O, 113 clustered + 20 scattered positions changed per sequence and step, 64
+    consecutive denoising steps on one handle (the active block moves every four steps, sixteen blocks).
+    All 8 sequences run on the GPU; sequences 0 and 5 are checked against batch-1 oracles at every step (layer output,
+    index list, staleness counters; the K and O caches every eighth step and at the end); the index sets of all
+    sequences are checked against the plan at every step."""
     import torch
     shape = wl.LLADA_DARE_O
     w_t, w_np = _weights_gpu(shape, 33, torch)
@@ -46,59 +48,115 @@ def test_config3_dare_o_batched_clustered_steps(dare):
     y = g.step(parity.to_device(x, shape), 2, 0.1)
     yo = {b: oracles[b].step(x[b:b + 1], 2, 0.1) for b in checked}
     for b in checked:
-        parity.assert_close(f"y step0 seq{b}", y[b:b + 1].float().cpu().numpy(), yo[b], parity.TOL_BF16)
-    for step in range(1, 5):
-        ch = wl.clustered_positions(hs.rng, shape, step, 113, 20)
+        parity.assert_close(f"y step0 seq{b}", y[b:b + 1].float().cpu().numpy(), yo[b], parity.TOL_BF16, rel_rms=parity.TOL_BF16)
+    n_steps = 64
+    for step in range(1, n_steps + 1):
+        ch = wl.clustered_positions(hs.rng, shape, step - 1, 113, 20)
         x = hs.advance(ch)
         y = g.step(parity.to_device(x, shape), 2, 0.1)
         sel = g.last_selection(shape.batch, shape.seq)
         np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
         assert sel["count"] == 133 * shape.batch
         np.testing.assert_array_equal(np.diff(sel["batch_off"]), np.full(shape.batch, 133))
-        caches = g.read_caches(shape.batch, shape.seq)
+        with_caches = step % 8 == 0 or step == n_steps
+        caches = g.read_caches(shape.batch, shape.seq) if with_caches else None
+        yh = y.float().cpu().numpy()
         for b in checked:
             o = oracles[b]
             yo_b = o.step(x[b:b + 1], 2, 0.1)
             parity.check_margin(o.last_scores, 0.1)
             np.testing.assert_array_equal(sel["idx"][sel["batch_off"][b]:sel["batch_off"][b + 1]] - b * shape.seq, o.last_idx)
-            parity.assert_close(f"y step{step} seq{b}", y[b:b + 1].float().cpu().numpy(), yo_b, parity.TOL_BF16)
-            parity.assert_close(f"o_cache step{step} seq{b}", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
-            parity.assert_close(f"k_cache step{step} seq{b}", caches["k"][b:b + 1], o.k_cache, parity.TOL_BF16, max_factor=2.0)
+            parity.assert_close(f"y step{step} seq{b}", yh[b:b + 1], yo_b, parity.TOL_BF16, rel_rms=parity.TOL_BF16)
             np.testing.assert_array_equal(sel["delta"][b], o.delta[0])
+            if with_caches:
+                parity.assert_close(f"o_cache step{step} seq{b}", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
+                parity.assert_close(f"k_cache step{step} seq{b}", caches["k"][b:b + 1], o.k_cache, parity.TOL_BF16, max_factor=2.0)
+    # after 64 steps some rows have been reused for dozens of steps in a row, others were refreshed in the last one
+    assert sel["delta"].max() >= 32 and (sel["delta"] == 0).sum() == 133 * shape.batch
     assert g.status() == 0
     g.close()
 
 
-@pytest.mark.parametrize("frac,pattern,mode", [(0.15, "uniform", 3), (0.5, "clustered", 1)])
-def test_config5_long_context_one_sequence(dare, frac, pattern, mode):
-    """Config 5: batch 4, seq 4096; all four sequences run on the GPU, sequence 2 is checked against a batch-1 oracle
-    (one dense step + one reuse step), index sets of all sequences against the plan."""
+@pytest.fixture(scope="module")
+def config5(dare):
+    """Config 5 (batch 4, seq 4096): weights, the first hidden states, a GPU layer, and a batch-1 oracle of sequence 2
+    after its first step (dense whatever the mode, so one oracle state serves every case)."""
     import torch
     shape = wl.LLADA_LONG
     w_t, w_np = _weights_gpu(shape, 55, torch)
     hs = wl.HiddenStream(shape)
-    g = dare.Layer(shape, w_t)
-    one = wl.scaled(shape, batch=1)
-    b = 2
-    o = parity.oracle_layer(one, w_np)
     x0 = hs.first()
-    y0 = g.step(parity.to_device(x0, shape), mode, 0.1)
-    parity.assert_close("y step0", y0[b:b + 1].float().cpu().numpy(), o.step(x0[b:b + 1], mode, 0.1), parity.TOL_BF16)
+    g = dare.Layer(shape, w_t)
+    b = 2
+    o0 = parity.oracle_layer(wl.scaled(shape, batch=1), w_np)
+    y0 = o0.step(x0[b:b + 1], 3, 0.1)
+    yield shape, g, hs, x0, parity.to_device(x0, shape), b, o0, y0
+    g.close()
+
+
+def _changed(hs, shape, frac, pattern):
     n = int(round(frac * shape.seq))
-    ch = wl.uniform_positions(hs.rng, shape, n) if pattern == "uniform" else wl.clustered_positions(hs.rng, shape, 9, n, 0)
+    if n == 0:
+        return np.zeros((shape.batch, shape.seq), bool)
+    return wl.uniform_positions(hs.rng, shape, n) if pattern == "uniform" else wl.clustered_positions(hs.rng, shape, 9, n, 0)
+
+
+@pytest.mark.parametrize("frac,pattern,mode", [(0.0, "uniform", 3), (0.0, "clustered", 2), (0.15, "uniform", 3),
+                                               (0.15, "clustered", 2), (0.5, "uniform", 2), (0.5, "clustered", 1),
+                                               (1.0, "uniform", 1), (1.0, "clustered", 3)])
+def test_config5_long_context_one_sequence(dare, config5, frac, pattern, mode):
+    """Config 5: changed fractions 0, 15, 50 and 100 % in both patterns, every reuse mode; all four sequences run on the
+    GPU, sequence 2 is checked against the batch-1 oracle (layer output, K, V and O caches, index list, staleness),
+    the index sets of all sequences against the plan."""
+    shape, g, hs0, x0, x0_dev, b, o0, y0 = config5
+    hs = copy.deepcopy(hs0)
+    g.reset()
+    yg0 = g.step(x0_dev, mode, 0.1)
+    parity.assert_close("y step0", yg0[b:b + 1].float().cpu().numpy(), y0, parity.TOL_BF16, rel_rms=parity.TOL_BF16)
+    ch = _changed(hs, shape, frac, pattern)
     x1 = hs.advance(ch)
     y1 = g.step(parity.to_device(x1, shape), mode, 0.1)
     sel = g.last_selection(shape.batch, shape.seq)
     np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
+    o = copy.deepcopy(o0)
     yo = o.step(x1[b:b + 1], mode, 0.1)
     parity.check_margin(o.last_scores, 0.1)
-    parity.assert_close("y step1", y1[b:b + 1].float().cpu().numpy(), yo, parity.TOL_BF16)
+    np.testing.assert_array_equal(sel["idx"][sel["batch_off"][b]:sel["batch_off"][b + 1]] - b * shape.seq, o.last_idx)
+    np.testing.assert_array_equal(sel["delta"][b], o.delta[0])
+    parity.assert_close("y step1", y1[b:b + 1].float().cpu().numpy(), yo, parity.TOL_BF16, rel_rms=parity.TOL_BF16)
     caches = g.read_caches(shape.batch, shape.seq)
     parity.assert_close("k_cache", caches["k"][b:b + 1], o.k_cache, parity.TOL_BF16, max_factor=2.0)
     parity.assert_close("v_cache", caches["v"][b:b + 1], o.v_cache, parity.TOL_BF16, max_factor=2.0)
     parity.assert_close("o_cache", caches["o"][b:b + 1], o.o_cache, parity.TOL_BF16, max_factor=2.0)
     assert g.status() == 0
-    g.close()
+
+
+@pytest.mark.parametrize("pattern", ["uniform", "clustered"])
+def test_config5_index_sets_over_the_whole_sweep(dare, config5, pattern):
+    """The 21 points of the crossover sweep (0 to 100 % changed in steps of 5 %): the GPU's index list of every
+    sequence against the plan, and that of sequence 2 against the oracle's scores (lines 1-3 of Alg. 1 and Eq. 2 only,
+    which is all an index set needs), with the margin checked on those scores."""
+    from oracle import dare_oracle as orc
+    shape, g, hs0, x0, x0_dev, b, o0, y0 = config5
+    for i in range(21):
+        frac = 0.05 * i
+        hs = copy.deepcopy(hs0)
+        hs.rng = np.random.default_rng(1000 * i + (0 if pattern == "uniform" else 500))
+        g.reset()
+        g.step(x0_dev, 3, 0.1)
+        ch = _changed(hs, shape, frac, pattern)
+        x1 = hs.advance(ch)
+        g.step(parity.to_device(x1, shape), 3, 0.1)
+        sel = g.last_selection(shape.batch, shape.seq)
+        assert sel["count"] == int(ch.sum()) == shape.batch * int(round(frac * shape.seq))
+        np.testing.assert_array_equal(sel["idx"], np.nonzero(ch.reshape(-1))[0])
+        s = orc.scores_only(o0, x1[b:b + 1])
+        parity.check_margin(s, 0.1)
+        want = np.nonzero(orc.refresh_mask(s, 0.1))[0]
+        np.testing.assert_array_equal(sel["idx"][sel["batch_off"][b]:sel["batch_off"][b + 1]] - b * shape.seq, want)
+        np.testing.assert_allclose(sel["scores"][b * shape.seq:(b + 1) * shape.seq], s, rtol=0,
+                                   atol=parity.SCORE_ATOL[wl.DTYPE_BF16])
+    assert g.status() == 0
 
 
 def test_long_context_attention_repeats_bit_identically(dare):

@@ -189,8 +189,9 @@ def test_appendix_form_of_predicate():
 class BruteLayer:
     """Scalar, loop-only restatement of Alg. 1 / Alg. 2 / both for one sequence batch (tiny sizes)."""
 
-    def __init__(self, d, H, hd, theta, eps, wq, wk, wv, wo, gain):
+    def __init__(self, d, H, hd, theta, eps, wq, wk, wv, wo, gain, score_head=0):
         self.d, self.H, self.hd, self.theta, self.eps = d, H, hd, theta, eps
+        self.score_head = score_head
         self.wq, self.wk, self.wv, self.wo, self.gain = (np.asarray(a, float).tolist() for a in (wq, wk, wv, wo, gain))
         self.prev = None
 
@@ -226,7 +227,7 @@ class BruteLayer:
                 ms = sum(t * t for t in x[b][i]) / d
                 xn[b][i] = [x[b][i][j] / math.sqrt(ms + self.eps) * self.gain[j] for j in range(d)]
                 q[b][i] = self._matvec(self.wq, xn[b][i])
-                q0 = q[b][i][:hd]
+                q0 = q[b][i][self.score_head * hd:(self.score_head + 1) * hd]
                 if not first:
                     p = self.qp[b][i]
                     dot = sum(u * w for u, w in zip(q0, p))
@@ -296,6 +297,54 @@ def test_step_matches_brute_force(mode, seed):
         np.testing.assert_allclose(lay.o_cache[:B, :S], np.array(bru.O), rtol=1e-10, atol=1e-12)
         if t > 0 and mode != 0:
             assert 0 < len(lay.last_idx) < B * S        # the case really mixes reuse and refresh
+
+
+@pytest.mark.parametrize("mode", [orc.MODE_KV, orc.MODE_BOTH])
+def test_step_matches_brute_force_with_another_scoring_head(mode):
+    """Sec. 3.2 scores head 0; the head is a parameter of the layer.  With head 1 the scalar restatement and the oracle
+    must still agree, and the refresh set must differ from head 0's somewhere (the parameter does something)."""
+    (B, S, d, H, hd), ws, gain, xs = _tiny(5, B=2, S=6)
+    lay = orc.OracleLayer(d, H, hd, B, S, 100.0, 1e-5, *ws, gain, score_head=1)
+    ref0 = orc.OracleLayer(d, H, hd, B, S, 100.0, 1e-5, *ws, gain, score_head=0)
+    bru = BruteLayer(d, H, hd, 100.0, 1e-5, *ws, gain, score_head=1)
+    differs = False
+    for t, x in enumerate(xs):
+        y = lay.step(x, mode, 0.05)
+        ref0.step(x, mode, 0.05)
+        yb, sb, selb = bru.step(x.tolist(), mode, 0.05)
+        np.testing.assert_allclose(y, yb, rtol=1e-10, atol=1e-12)
+        if t > 0:
+            np.testing.assert_allclose(lay.last_scores, sb.reshape(-1), rtol=1e-9, atol=1e-13)
+            differs |= not np.allclose(lay.last_scores, ref0.last_scores)
+        np.testing.assert_array_equal(lay.last_idx, np.nonzero(selb.reshape(-1))[0])
+        np.testing.assert_allclose(lay.q_prev[:B, :S], np.array(bru.qp), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(lay.o_cache[:B, :S], np.array(bru.O), rtol=1e-10, atol=1e-12)
+    assert differs
+
+
+@pytest.mark.parametrize("score_head", [0, 2])
+def test_scores_only_is_the_score_of_the_step(score_head):
+    """`scores_only` (lines 1-3 of Alg. 1 without the state update) against what the full step then reports, on full
+    and on window steps; it must leave the state alone and report +inf before a first step."""
+    shape = wl.scaled(wl.TINY_F32, d_model=64, n_heads=4, head_dim=16, seq=48, prompt=16, batch=2)
+    w = wl.make_weights(shape, 17)
+    hs = wl.HiddenStream(shape, 17)
+    lay = orc.OracleLayer(shape.d_model, shape.n_heads, shape.head_dim, shape.batch, shape.seq, shape.rope_theta,
+                          shape.rms_eps, w["w_q"], w["w_k"], w["w_v"], w["w_o"], w["rms_gain"], score_head=score_head)
+    x0 = hs.first()
+    assert np.isinf(orc.scores_only(lay, x0)).all()
+    lay.step(x0, 3, 0.1)
+    for t in range(3):
+        x = hs.advance_graded() if t == 1 else hs.advance(wl.uniform_positions(hs.rng, shape, 9))
+        p = 16 if t == 2 else 0
+        xw = np.ascontiguousarray(x[:, p:])
+        before = (lay.q_prev.copy(), lay.k_cache.copy(), lay.o_cache.copy(), lay.delta.copy())
+        s = orc.scores_only(lay, xw, pos_begin=p)
+        for a, b in zip(before, (lay.q_prev, lay.k_cache, lay.o_cache, lay.delta)):
+            np.testing.assert_array_equal(a, b)
+        lay.step(xw, 3, 0.1, pos_begin=p)
+        np.testing.assert_allclose(s, lay.last_scores, rtol=1e-12, atol=1e-15)
+        assert 0 < len(lay.last_idx) < xw.shape[0] * xw.shape[1]
 
 
 # ----------------------------------------------------------------------------- invariants of the method
