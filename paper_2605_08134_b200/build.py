@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdare.so")
-SOURCES = ["api.cu", "common.cu", "simt.cu", "tc.cu", "gemm_tc.cu", "gemm_persist.cu", "attn_tc.cu", "score_tc.cu", "select_large.cu", "stack.cu"]
+SOURCES = ["api.cu", "common.cu", "simt.cu", "tc.cu", "gemm_tc.cu", "gemm_persist.cu", "attn_tc.cu", "select_large.cu", "stack.cu"]
 
 
 def _newest(paths):

@@ -72,16 +72,6 @@ size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) 
   B.y_stage = take(Tm * d * e);
   B.tmp = use_tc ? nullptr : (float*)take(Tm * 2 * d * sizeof(float));
   B.yc = use_tc ? take(Tm * d * e) : nullptr;
-  B.sliver = nullptr;
-  if (use_tc) {
-    int ksplit = 0, per = 0;
-    if (sliver_geometry(c->d_model, &ksplit, &per)) {
-      // (steps of at most eight 128-row tiles take this route: tc.cu)
-      const size_t tiles = (size_t)c->max_batch * ((c->max_seq + 127) / 128);
-      const size_t rows = (tiles < 8 ? tiles : 8) * 128;
-      B.sliver = (float*)take((size_t)ksplit * rows * 128 * sizeof(float));
-    }
-  }
   return off;
 }
 
@@ -567,8 +557,6 @@ const char* dare_kernel_slot_name(int slot) {
     case SLOT_KV_POST: return "kv_post";
     case SLOT_ATTN: return "attention";
     case SLOT_OUT_GEMM: return "out_gemm";
-    case SLOT_SLIVER: return "q_sliver";
-    case SLOT_SCORE: return "head_score";
   }
   return "?";
 }

@@ -270,11 +270,12 @@ template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, 
 constexpr int kSelPerThread = 4;
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
-                                                      int* __restrict__ batch_off, int* __restrict__ delta) {
+                                                      int* __restrict__ batch_off, int* __restrict__ delta,
+                                                      int wait_at_end) {
   __shared__ int warp_tot[32];
   __shared__ int before_chunk;
   if (threadIdx.x == 0) before_chunk = 0;
-  ptx::pdl_wait();
+  if (!wait_at_end) ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -354,16 +355,18 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
     *count = base;
     batch_off[g.batch] = base;
   }
+  if (wait_at_end) ptx::pdl_wait();
 }
 
 // The same for short steps: one token per thread and chunk of 1024, warp ballot + popcount (less index arithmetic
 // per token, which is what a step of a few hundred tokens pays for).
 __global__ void __launch_bounds__(1024) select_small_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
-                                                      int* __restrict__ batch_off, int* __restrict__ delta) {
+                                                      int* __restrict__ batch_off, int* __restrict__ delta,
+                                                      int wait_at_end) {
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
-  ptx::pdl_wait();
+  if (!wait_at_end) ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -405,16 +408,20 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float* __restr
     *count = base;
     batch_off[g.batch] = base;
   }
+  if (wait_at_end) ptx::pdl_wait();
 }
 
+// beside_predecessor: the selection refreshes every token (it reads no scores) and nothing the kernel before it in the
+// stream touches, so it runs beside that kernel and waits for it only before it leaves.
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, cudaStream_t st) {
+                   int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor) {
   const int all = (select_all || scores == nullptr) ? 1 : 0;
+  const int late = (beside_predecessor && all) ? 1 : 0;
   if (g.tokens() <= 2048)
-    launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta);
+    launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta, late);
   else
     launch_pdl(select_kernel, dim3((g.tokens() + 1024 * kSelPerThread - 1) / (1024 * kSelPerThread)), dim3(1024), 0, st, 1,
-               scores, tau, all, g, idx, count, batch_off, delta);
+               scores, tau, all, g, idx, count, batch_off, delta, late);
 }
 
 // ------------------------------------------------------------------------------------------------ reused rows

@@ -251,8 +251,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
-  // (a Q projection without a score buffer leaves score and stored query alone: the step took them from the sliver)
-  const bool score_tile = (EPI == EPI_Q) && p.scores != nullptr && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+  const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
   RowBatch<RB> rb;
 
   if (active) {

@@ -25,14 +25,13 @@ struct Buffers {
   void* y_stage;
   void* yc;         // tensor-core path: cache of projected outputs y = W_O O by cache row (gathered output projection)
   float* tmp;       // SIMT path: fp32 projection results [T, 2d]
-  float* sliver;    // tensor-core path: partial sums of the scoring head's query sliver [slices][<= 1024 rows][128]
 };
 
 struct TcState;
 
 // Kernel slots for the optional per-kernel timing.
 enum { SLOT_NORM = 0, SLOT_Q_GEMM, SLOT_Q_POST, SLOT_SELECT, SLOT_GATHER, SLOT_KV_GEMM, SLOT_KV_POST, SLOT_ATTN,
-       SLOT_OUT_GEMM, SLOT_SLIVER, SLOT_SCORE, SLOT_COUNT };
+       SLOT_OUT_GEMM, SLOT_COUNT };
 constexpr int kMaxMarks = 16;
 
 }  // namespace dare

@@ -140,51 +140,24 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   prof_mark(L, SLOT_NORM, st);
   launch_rmsnorm<bf16>((const bf16*)x, L->w.rms_gain, (bf16*)B.xn, T_, d, L->cfg.rms_eps, st, dbg ? dbg + 40 : nullptr);
   ++launches;
-  // Short DARE-KV steps take the scoring head first (Alg. 1 lines 2-5 need only its 128 columns of Q): sliver of the Q
-  // projection with the reduction spread over many CTAs -> drift score -> selection, and then the gathered K/V
-  // projection (a stream of W_K, W_V) and the full Q projection (tensor work) run side by side instead of one after the
-  // other.  Every other step scores in the epilogue of the Q projection.
-  const int sliver_rows = (L->cfg.max_batch * ((L->cfg.max_seq + 127) / 128) < 8 ? L->cfg.max_batch * ((L->cfg.max_seq + 127) / 128) : 8) * 128;
-  const bool head_first = kv_sparse && m_tiles_dense <= 8 && B.sliver != nullptr && m_tiles_dense * 128 <= sliver_rows;
-  // line 2 (+ line 3, the stored-query update when the step scores here) + rotary embedding, one kernel
-  auto q_projection = [&](bool beside_kv) -> cudaError_t {
+  // line 2 + line 3 + stored-query update + rotary embedding, one kernel
+  {
     GemmParams p = base;
     p.out0 = (bf16*)B.q;
     p.debug = dbg;
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_Q_GEMM, st);
-    if (beside_kv) {
-      // score and stored query are done; the launch shares the GPU with the K/V projection issued just before it, so
-      // it takes about half of the SMs: the reduction is split only while that leaves it below 84 CTAs
-      p.scores = nullptr; p.wait_at_end = 1;
-      const int mt2 = (m_tiles_dense + 1) / 2 * 2;
-      const int sp = (n_tiles * mt2 * 2 <= 84 && kblocks >= 2) ? 2 : 1;
-      if (m_tiles_dense >= 2) return launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
-      return launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, sp, st);
-    }
     const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
     if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
-      return launch_gemm_tc(EPI_Q, 128, S.a_xn, S.w_q64, S.w_q64, p, d / 128, m_tiles_dense, 2, st, 1);
-    if (use_persist(n_tiles, m_tiles_dense, sp))
-      return DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_Q, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, st, 1)
-                               : launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st);
-    if (use_pairs(n_tiles, m_tiles_dense, sp))
-      return launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
-    return launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, sp, st);
-  };
-  if (head_first) {
-    SliverParams sp;
-    sp.K = d; sp.seq_act = g.seq_act; sp.tiles_per_seq = tiles_per_seq; sp.w_row0 = g.score_head * 128;
-    sliver_geometry(d, &sp.ksplit, &sp.kb_per_cta);
-    sp.rows_pad = m_tiles_dense * 128; sp.partial = B.sliver; sp.status = B.status;
-    prof_mark(L, SLOT_SLIVER, st);
-    e = launch_q_sliver(S.a_xn, S.w_q128, sp, m_tiles_dense, st); ++launches;
-    if (e != cudaSuccess) return DARE_ERR_CUDA;
-    prof_mark(L, SLOT_SCORE, st);
-    e = launch_head_score(sp, g, B.q_prev, B.scores, st); ++launches;
-    if (e != cudaSuccess) return DARE_ERR_CUDA;
-  } else {
-    e = q_projection(false); ++launches;
+      e = launch_gemm_tc(EPI_Q, 128, S.a_xn, S.w_q64, S.w_q64, p, d / 128, m_tiles_dense, 2, st, 1);
+    else if (use_persist(n_tiles, m_tiles_dense, sp))
+      e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_Q, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, st, 1)
+                               : launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st));
+    else if (use_pairs(n_tiles, m_tiles_dense, sp))
+      e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
+    else
+      e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, sp, st);
+    ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // A dense K/V projection (Alg. 2 line 7, or the full forward of Appendix E.2) needs nothing from the Q projection
@@ -194,9 +167,11 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   // K/V tiles do not.  The selection then follows both.
   const bool kv_beside_q = !kv_sparse && m_tiles_dense <= 8;
   // lines 4-5 + Sec. 4
+  const bool select_all = !has_prev || mode == DARE_MODE_DENSE;
   auto select_now = [&]() {
     prof_mark(L, SLOT_SELECT, st);
-    launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st);
+    // (a selection that refreshes everything reads no scores: behind the two projections it runs beside them)
+    launch_select(B.scores, tau, select_all, g, B.idx, B.count, B.batch_off, B.delta, st, kv_beside_q && select_all);
     ++launches;
   };
   if (!kv_beside_q) select_now();
@@ -217,10 +192,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
         // Narrower tiles put twice as many CTAs on it; the reduction split is sized for one row tile.
         p.n_split = d / 128;
         const int n_tiles128 = 2 * d / 128;
-        // (beside the Q projection it keeps to one CTA per column tile: the two launches share the SMs)
         e = launch_gemm_tc(EPI_KV, 128, S.a_xn, S.w_k128, S.w_v128, p, n_tiles128, m_tiles,
-                           head_first ? 1 : pick_splits(n_tiles128, kblocks), st); ++launches;
-        if (head_first && e == cudaSuccess) { e = q_projection(true); ++launches; }
+                           pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
         if (DARE_PERSIST_LIST && use_persist(n_tiles, m_tiles, 1) && compact_ok) {
@@ -258,8 +231,9 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     p.q = (const bf16*)B.q; p.oc = (bf16*)B.oc; p.idx = o_sparse ? B.idx : nullptr;
     p.batch_off = o_sparse ? B.batch_off : nullptr; p.g = g; p.status = B.status;
     p.debug = dbg ? dbg + 16 : nullptr;
-    // the refresh set, or the queries, then come from the kernel right before
-    p.wait_first = ((kv_beside_q && o_sparse) || head_first) ? 1 : 0;
+    // the refresh set then comes from the kernel right before; or the two kernels before ran beside the Q projection
+    // without waiting for it, so the queries are not known to be complete before this kernel's own wait
+    p.wait_first = kv_beside_q ? 1 : 0;
     e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }

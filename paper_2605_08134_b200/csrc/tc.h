@@ -62,26 +62,6 @@ struct AttnParams {
                             // so nothing of the step is read ahead of the dependency wait
 };
 
-// Scoring-head sliver of the Q projection with the reduction spread over many CTAs, and the drift score from its
-// partial sums (score_tc.cu).
-constexpr int kSliverMaxKb = 4;        // 64-element k-blocks per CTA (all of them in shared memory at once)
-constexpr int kSliverMaxSplit = 32;    // slices of the reduction
-constexpr int kSliverMaxRows = 1024;   // rows of a step that takes this route (eight row tiles)
-struct SliverParams {
-  int K;                 // reduction length
-  int seq_act;           // rows per sequence of the compact A matrix ...
-  int tiles_per_seq;     // ... and 128-row tiles per sequence
-  int w_row0;            // first row of W_Q of the scoring head
-  int ksplit, kb_per_cta;
-  int rows_pad;          // rows of one slice's plane of the partial buffer (row tiles x 128)
-  float* partial;        // [ksplit][rows_pad][128] fp32
-  int* status;
-};
-// slices and k-blocks per CTA for a reduction of length K; false if the route does not cover it
-bool sliver_geometry(int K, int* ksplit, int* kb_per_cta);
-cudaError_t launch_q_sliver(const CUtensorMap& a, const CUtensorMap& w, const SliverParams& p, int m_tiles, cudaStream_t st);
-cudaError_t launch_head_score(const SliverParams& p, const StepGeom& g, float* q_prev, float* scores, cudaStream_t st);
-
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st);
 
