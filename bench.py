@@ -11,12 +11,18 @@ step (87 % reuse), mode "both".  Steps rotate over `--layers` layer instances (8
 the 126 MB L2) and alternate between two hidden-state buffers so that every timed step refreshes the same
 planned token set.
 
-Prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle on the same workload instead.
+Timing: after W warm-up steps the region of exactly K steps (barrier + synchronise on both sides, CUDA events, max over
+ranks) is repeated until at least a second of it has been timed; `ms_per_step` is the median over the repeats, p10 / p90
+and the number of repeats go with it.  The dense path and the end-to-end figure follow the same protocol.
+
+Prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle on the same workload instead.  `--gpus N` with
+N > 1 and no torchrun environment starts N ranks itself (one replica per GPU).
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -73,7 +79,7 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             if len(r) < 7:
@@ -82,11 +88,44 @@ class ClockSampler:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(r[2]))
+            except ValueError:
+                pass
             for name, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "power_w_max": max(pw) if pw else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_config(shape, args, n_refreshed, world):
+    """The `config` object of the JSON line: the workload and how the timed steps see HBM; both arms print the same."""
+    d = shape.d_model
+    return {"workload": shape.name, "d_model": d, "n_heads": shape.n_heads, "head_dim": shape.head_dim,
+            "batch": shape.batch, "seq_len": shape.seq, "mode": args.mode, "changed_fraction": args.changed,
+            "refreshed_tokens": int(n_refreshed), "threshold": TAU, "layers_rotated": args.layers,
+            "l2": "inputs larger than L2: weights of %d layer instances (%.0f MB) rotate"
+                  % (args.layers, args.layers * 4 * d * d * 2 / 1e6),
+            "parallelism": "replicas" if world > 1 else "single"}
+
+
+def percentiles(values):
+    """(median, p10, p90) of a list of per-step times."""
+    v = sorted(values)
+    pick = lambda q: v[min(len(v) - 1, max(0, int(round(q * (len(v) - 1)))))]
+    return statistics.median(v), pick(0.10), pick(0.90)
+
+
+def load_traffic(workload):
+    """DRAM bytes per launch and kernel from the ncu capture summarised under profiles/ (None when there is none)."""
+    path = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}_both13.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except OSError:
+        return None
 
 
 def make_inputs_np(shape, changed_frac, seed):
@@ -186,7 +225,7 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def timed(steps, m, host=None, pipelined=False):
+    def timed_once(steps, m, host=None, pipelined=False):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         t0 = time.perf_counter()
@@ -201,16 +240,27 @@ def run_ours(args):
         barrier()
         return ms, launches
 
-    # ---- reuse path: warm-up, then exactly K timed steps with the clocks sampled
+    def timed(steps, m, host=None, pipelined=False, min_total_ms=1000.0, max_repeats=4000):
+        """The K-step region repeated until `min_total_ms` of it have been timed (every rank sees the same max-over-ranks
+        times, so all stop together).  -> per-step times of the repeats (ms), launches of one region."""
+        per_step, total, launches = [], 0.0, 0
+        while True:
+            ms, launches = timed_once(steps, m, host=host, pipelined=pipelined)
+            per_step.append(ms / steps)
+            total += ms
+            if total >= min_total_ms or len(per_step) >= max_repeats:
+                return per_step, launches
+
+    # ---- reuse path: warm-up, then regions of exactly K timed steps with the clocks sampled
     prime(mode)
     one_pass(max(args.warmup, 3), mode)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.15)
-    total_ms, launches = timed(args.steps, mode)
+    reuse_times, launches = timed(args.steps, mode, min_total_ms=args.min_ms)
     clocks = sampler.stop() if rank == 0 else None
-    ms_per_step = total_ms / args.steps
+    ms_per_step, ms_p10, ms_p90 = percentiles(reuse_times)
     # selection really is the planned one
     sel = layers[0].last_selection(shape.batch, shape.seq)
     expect = T if mode == 0 else n_planned
@@ -222,8 +272,13 @@ def run_ours(args):
     # ---- dense path of the same library, same protocol
     prime(0)
     one_pass(max(args.warmup, 3), 0)
-    dense_ms, _ = timed(args.steps, 0)
-    dense_ms_per_step = dense_ms / args.steps
+    dense_sampler = ClockSampler(local_rank)
+    if rank == 0:
+        dense_sampler.start()
+        time.sleep(0.15)
+    dense_times, _ = timed(args.steps, 0, min_total_ms=args.min_ms)
+    dense_clocks = dense_sampler.stop() if rank == 0 else None
+    dense_ms_per_step, dense_p10, dense_p90 = percentiles(dense_times)
 
     # ---- per-kernel times: a second pass of K steps with an event before every kernel
     prime(mode)
@@ -247,7 +302,7 @@ def run_ours(args):
     # themselves, from the return of a kernel's wait on its predecessor to the exit of its last CTA.  The events of
     # the pass above break the programmatic launch overlap and add a few microseconds to every kernel; these do not.
     in_chain = {}
-    if True:
+    if not args.no_in_chain:
         try:
             one_pass(2 * len(layers), mode)
             for lay in layers:
@@ -310,14 +365,21 @@ def run_ours(args):
     xh = [torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).pin_memory() for a in (xa_np, xb_np)]
     yh = [torch.empty_like(xh[0]).pin_memory() for _ in layers]          # one result buffer per layer instance
     one_pass(max(args.warmup, 3), mode, host=(xh[0], xh[1], yh))
-    e2e_sync_ms, _ = timed(args.steps, mode, host=(xh[0], xh[1], yh))
-    e2e_sync_ms_per_step = e2e_sync_ms / args.steps
+    sync_times, _ = timed(args.steps, mode, host=(xh[0], xh[1], yh), min_total_ms=args.min_ms / 4)
+    e2e_sync_ms_per_step = percentiles(sync_times)[0]
     # ... and through the enqueue-only entry point: a layer's copy in, step and copy out run on three streams, so the
-    # copies of one layer instance overlap the kernels of another (every step still copies its 4 MB in and out)
+    # copies of one layer instance overlap the kernels of another (every step still copies its 4 MB in and out).
+    # A region of K steps that starts and ends drained does not fill that pipeline when K is small, so two figures are
+    # taken: the K-step region as it is (median over the repeats), and regions long enough to run full (a tenth of the
+    # time budget each, ten of them): the second is what a caller who keeps stepping sees and is the one reported as
+    # `e2e.value`.
     prime(mode)
     one_pass(max(args.warmup, 3), mode, host=(xh[0], xh[1], yh), pipelined=True)
-    e2e_ms, _ = timed(args.steps, mode, host=(xh[0], xh[1], yh), pipelined=True)
-    e2e_ms_per_step = e2e_ms / args.steps
+    drained_times, _ = timed(args.steps, mode, host=(xh[0], xh[1], yh), pipelined=True, min_total_ms=args.min_ms / 4)
+    e2e_drained_ms = percentiles(drained_times)[0]
+    long_steps = max(args.steps, int(math.ceil(args.min_ms / 10.0 / e2e_drained_ms / len(layers))) * len(layers))
+    long_times = [timed_once(long_steps, mode, host=(xh[0], xh[1], yh), pipelined=True)[0] / long_steps for _ in range(10)]
+    e2e_ms_per_step, e2e_p10, e2e_p90 = percentiles(long_times)
 
     if rank != 0:
         if dist is not None:
@@ -363,11 +425,12 @@ def run_ours(args):
         else:
             rows.append({"kernel": name, "us": round(us, 2)})
     dom = max((r for r in rows if "bound" in r), key=lambda r: r["us"])
-    # DRAM bytes per launch of that kernel from one ncu capture of this workload (profiles/ holds the summaries)
-    ncu_traffic = {"q_gemm": 38.3e6, "kv_gemm": 68.7e6, "out_gemm": 37.8e6}
+    # DRAM bytes per launch of that kernel from the ncu capture of this workload summarised under profiles/
+    traffic = load_traffic(shape.name) or {}
     roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
                 "unit": dom["unit"], "frac": dom["frac"],
-                "traffic": ncu_traffic.get(dom["kernel"]) if shape.name == wl.LLADA_LAYER.name else None,
+                "traffic": traffic.get("dram_bytes_per_launch", {}).get(dom["kernel"]),
+                "traffic_source": traffic.get("source"),
                 "peak_source": f"of {peaks['source']} (sustained figure: the kernel is timed inside the step)",
                 "timing": "CUDA events recorded by the library around each kernel, second pass of K steps",
                 "in_chain": dom.get("in_chain"),
@@ -382,19 +445,23 @@ def run_ours(args):
         "metric": "tokens_per_s_through_one_dare_layer", "value": round(tokens_per_s, 1), "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
         "us_per_layer": round(ms_per_step * 1e3, 2),
+        "timing": {"what": "median over repeats of the K-step region (CUDA events, max over ranks)", "repeats": len(reuse_times),
+                   "p10_ms_per_step": round(ms_p10, 5), "p90_ms_per_step": round(ms_p90, 5),
+                   "first_region_ms_per_step": round(reuse_times[0], 5), "timed_ms_total": round(sum(reuse_times) * args.steps, 1)},
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": shape.name, "d_model": d, "n_heads": shape.n_heads, "head_dim": shape.head_dim,
-                   "batch": shape.batch, "seq_len": shape.seq, "mode": args.mode, "changed_fraction": args.changed,
-                   "refreshed_tokens": n, "threshold": TAU, "layers_rotated": args.layers,
-                   "l2": "inputs larger than L2: weights of %d layer instances (%.0f MB) rotate"
-                         % (args.layers, args.layers * 4 * d * d * 2 / 1e6),
-                   "parallelism": "replicas" if world > 1 else "single"},
+        "config": workload_config(shape, args, n, world),
         "dense": {"ms_per_step": round(dense_ms_per_step, 5), "value": round(world * T / (dense_ms_per_step * 1e-3), 1),
+                  "p10_ms_per_step": round(dense_p10, 5), "p90_ms_per_step": round(dense_p90, 5), "repeats": len(dense_times),
+                  "clocks": dense_clocks, "first_region_ms_per_step": round(dense_times[0], 5),
                   "speedup_of_reuse_path": round(dense_ms_per_step / ms_per_step, 3)},
         "e2e": {"value": round(world * T / (e2e_ms_per_step * 1e-3), 1), "unit": "tokens/s",
-                "ms_per_step": round(e2e_ms_per_step, 5),
+                "ms_per_step": round(e2e_ms_per_step, 5), "p10_ms_per_step": round(e2e_p10, 5),
+                "p90_ms_per_step": round(e2e_p90, 5), "repeats": len(long_times), "steps_per_region": long_steps,
                 "h2d_bytes_per_step": T * d * 2, "d2h_bytes_per_step": T * d * 2,
-                "api": "dare_layer_step_host_async + dare_layer_wait_host (copies overlapped across layer instances)",
+                "api": "dare_layer_step_host_async + dare_layer_wait_host (copies overlapped across layer instances); "
+                       "wall clock over regions long enough to keep the copy pipeline full",
+                "k_step_region_drained": {"ms_per_step": round(e2e_drained_ms, 5), "repeats": len(drained_times),
+                                          "what": "the same call over regions of exactly K steps that start and end drained"},
                 "synchronous_call": {"api": "dare_layer_step_host", "ms_per_step": round(e2e_sync_ms_per_step, 5),
                                      "value": round(world * T / (e2e_sync_ms_per_step * 1e-3), 1)}},
         "graph_replay": None if graph_ms_per_step is None else
@@ -436,6 +503,7 @@ def cpu_baseline(shape, xa_np, xb_np, layer0, mode, budget_s):
     except Exception:
         cores = os.cpu_count()
     return {"value": round(steps * shape.tokens / dt, 1), "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+            "cores_what": "threads of numpy's BLAS pool (threadpoolctl)",
             "sample": f"{steps} reuse steps of the full workload after one dense step, {dt:.1f} s, numpy fp64"}
 
 
@@ -478,8 +546,10 @@ def run_reference(args):
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": warm,
         "ms_per_step": round(dt / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": shape.name, "mode": args.mode, "changed_fraction": args.changed, "threshold": TAU},
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": int(cores), "kind": "oracle", "sample": sample},
+        "config": workload_config(shape, args, int(changed.sum()) if mode != 0 else shape.tokens,
+                                  int(os.environ.get("WORLD_SIZE", "1"))),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+                         "cores_what": "threads of numpy's BLAS pool (threadpoolctl)", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -731,6 +801,8 @@ def main():
     ap.add_argument("--changed", type=float, default=0.13)
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-ms", type=float, default=1000.0, help="repeat the K-step region until this much has been timed")
+    ap.add_argument("--no-in-chain", action="store_true", help="skip the device-timestamp pass")
     ap.add_argument("--d-model", type=int, default=0, help="exploration: other layer width (multiple of 128)")
     ap.add_argument("--seq", type=int, default=0, help="exploration: other sequence length")
     ap.add_argument("--batch", type=int, default=0, help="exploration: other batch size")
@@ -739,6 +811,19 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="long-context crossover sweep (config 5) instead")
     ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
     args = ap.parse_args()
+    # one process per GPU: under torchrun the world size must be the one asked for; started plainly with --gpus N > 1
+    # this process becomes the launcher of N ranks (replicas, NCCL for the barrier and the max over ranks only)
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is not None and int(world_env) != args.gpus and args.impl == "ours" and not (args.stack or args.sweep or args.micro):
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world_env}: start one rank per GPU")
+    if world_env is None and args.gpus > 1 and not (args.stack or args.sweep or args.micro):
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     if args.stack:
         run_stack(args)
     elif args.sweep:
