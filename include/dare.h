@@ -34,9 +34,13 @@
  *   `import_state`, `step_host`) synchronise the stream themselves.
  *
  * Errors
- *   Status codes only; nothing is thrown, nothing aborts.  Problems seen by a kernel (a bounded wait that
- *   ran out, an index that failed its range check) are recorded in a device status word that
- *   `dare_layer_status` returns.
+ *   Status codes only; nothing is thrown, nothing aborts.  Problems seen by a kernel are recorded in a device
+ *   status word that `dare_layer_status` returns: a bounded wait that ran out (every wait of a kernel on a barrier
+ *   gives up after two seconds, and the kernel runs on to its normal exit), or a value of the device-side selection
+ *   that failed its range check before it was used as an address (a token of the refresh list outside the step, a
+ *   list length or a sequence's slice outside the list: the access is skipped and the launch goes on).  A recorded
+ *   error stays until `dare_layer_clear_status`; while a time-out stands, every wait gives up at once, so results
+ *   are undefined until it is cleared.
  *
  * Threading: one host thread per handle at a time.
  */
@@ -152,6 +156,21 @@ dare_status_t dare_layer_destroy(dare_layer_t* layer);
  * DARE_ERR_DEVICE_CHECK) or DARE_ERR_CUDA if the stream reports an error. */
 dare_status_t dare_layer_status(dare_layer_t* layer, void* cuda_stream);
 
+/* Clears the device status word (asynchronous on the stream); the handle is usable again afterwards.  Call
+ * dare_layer_reset as well if the failed step may have left the caches half written. */
+dare_status_t dare_layer_clear_status(dare_layer_t* layer, void* cuda_stream);
+
+/* Diagnostics of the error paths (nothing here faults, traps or hangs the device).
+ * dare_layer_debug_wait_probe: runs the kernels' bounded wait in a one-CTA launch on a barrier that nothing ever
+ *   arrives on, with `limit_ns` (at most 1e9) as its limit; the wait gives up, the launch ends normally, the status
+ *   word then reads DARE_ERR_TIMEOUT.  *waited_ns_host receives how long the wait took (the call synchronises).
+ * dare_layer_debug_inject: the next step overwrites, right after its selection, what = 1: the first entry of the
+ *   refresh list with batch * seq_act (one past the step's tokens), what = 2: the list's length with
+ *   batch * seq_act + 3; the kernels that consume the selection must flag DARE_ERR_DEVICE_CHECK and skip the access.
+ *   One step only; what = 0 withdraws it. */
+dare_status_t dare_layer_debug_wait_probe(dare_layer_t* layer, uint64_t limit_ns, uint64_t* waited_ns_host, void* cuda_stream);
+dare_status_t dare_layer_debug_inject(dare_layer_t* layer, int what);
+
 /* Selection of the last step, copied to host buffers (any of them may be NULL):
  *   idx_host        int32[count]  ascending flat indices b*seq_act + i of the refresh set (room for batch*seq_act)
  *   count_host      int32         |refresh set|
@@ -224,7 +243,9 @@ dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float t
  *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress with that device
  *     current): make that first call outside any stream capture.
  *   - All calls on a device share the array; it keeps the previous call's contents (nothing needs clearing: a call
- *     writes every entry before reading it).  Calls that overlap on the GPU, e.g. on two streams, race on it. */
+ *     writes every entry before reading it).  Calls that overlap on the GPU, e.g. on two streams, race on it: their
+ *     lists and counts are then undefined (entries may be missing, repeated or another call's), though no call ever
+ *     writes outside its own idx[0, n_tokens) and count.  Serialise them (one stream, or events). */
 int64_t dare_select_compact_static_max_tokens(void);
 dare_status_t dare_select_compact_static(const float* scores, int64_t n_tokens, float threshold, int32_t* idx,
                                          int32_t* count, void* cuda_stream);

@@ -89,6 +89,17 @@ dare_status_t check_handle(const dare_layer_t* L) {
     if (e_ != cudaSuccess) { cudaGetLastError(); return DARE_ERR_CUDA; } \
   } while (0)
 
+}  // namespace
+namespace dare {
+// Diagnostics (dare_layer_debug_inject): overwrites one value of the selection just made, once.
+void inject_selection_error(dare_layer* L, const StepGeom& g, cudaStream_t st) {
+  if (L->inject == 1) launch_poke_int(L->buf.idx, g.tokens(), st);            // first list entry: one past the step's tokens
+  else if (L->inject == 2) launch_poke_int(L->buf.count, g.tokens() + 3, st); // list longer than the step
+  L->inject = 0;
+}
+}  // namespace dare
+namespace {
+
 template <typename T>
 dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode, float tau, T* y, cudaStream_t st) {
   const Buffers& B = L->buf;
@@ -110,18 +121,19 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
   prof_mark(L, SLOT_SELECT, st);
   launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st); ++launches;
+  inject_selection_error(L, g, st);
   // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
   const int* kv_idx = kv_sparse ? B.idx : nullptr;
   const int* kv_cnt = kv_sparse ? B.count : nullptr;
   prof_mark(L, SLOT_KV_GEMM, st);
-  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_k, B.tmp, T_, d, d, 2 * d, st); ++launches;
-  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_v, B.tmp + d, T_, d, d, 2 * d, st); ++launches;
+  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_k, B.tmp, T_, d, d, 2 * d, st, T_, B.status); ++launches;
+  launch_gemm_simt<T>((const T*)B.xn, kv_idx, kv_cnt, (const T*)L->w.w_v, B.tmp + d, T_, d, d, 2 * d, st, T_, B.status); ++launches;
   prof_mark(L, SLOT_KV_POST, st);
-  launch_kv_post_simt<T>(B.tmp, 2 * d, kv_idx, kv_cnt, B.rope_cs, (T*)B.kc, (T*)B.vc, g, st); ++launches;
+  launch_kv_post_simt<T>(B.tmp, 2 * d, kv_idx, kv_cnt, B.rope_cs, (T*)B.kc, (T*)B.vc, g, st, B.status); ++launches;
   // attention: Alg. 1 line 10 (all rows) or Alg. 2 lines 6, 8-10 (refresh set rows, others keep the cache)
   prof_mark(L, SLOT_ATTN, st);
   launch_attention_simt<T>((const T*)B.q, (const T*)B.kc, (const T*)B.vc, o_sparse ? B.idx : nullptr,
-                           o_sparse ? B.count : nullptr, (T*)B.oc, g, st); ++launches;
+                           o_sparse ? B.count : nullptr, (T*)B.oc, g, st, B.status); ++launches;
   // last line: output projection of every row
   prof_mark(L, SLOT_OUT_GEMM, st);
   launch_out_proj_simt<T>((const T*)B.oc, (const T*)L->w.w_o, B.tmp, y, g, st); ++launches;
@@ -243,6 +255,7 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->prof_n = 0;
   L->prof_ev_ready = false;
   L->debug_on = false;
+  L->inject = 0;
   L->host_async_ready = false;
   memset(&L->last_geom, 0, sizeof(L->last_geom));
   carve(cfg, use_tc, (char*)workspace, &L->buf);
@@ -543,6 +556,36 @@ dare_status_t dare_layer_debug_timestamps(dare_layer_t* L, int enable, uint64_t*
     CUDA_TRY(cudaMemsetAsync(L->buf.debug, 0, (64 + 3 * 1024) * sizeof(uint64_t), st));
   }
   L->debug_on = enable != 0;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_clear_status(dare_layer_t* L, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  CUDA_TRY(cudaMemsetAsync(L->buf.status, 0, sizeof(int), (cudaStream_t)cuda_stream));
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_debug_wait_probe(dare_layer_t* L, uint64_t limit_ns, uint64_t* waited_ns_host, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return DARE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  unsigned long long* slot = L->buf.debug + 63;          // (a slot no kernel of a step writes)
+  launch_wait_probe(L->buf.status, limit_ns, slot, st);
+  CUDA_TRY(cudaGetLastError());
+  unsigned long long waited = 0;
+  CUDA_TRY(cudaMemcpyAsync(&waited, slot, sizeof(waited), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (waited_ns_host) *waited_ns_host = waited;
+  return DARE_OK;
+}
+
+dare_status_t dare_layer_debug_inject(dare_layer_t* L, int what) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (what < 0 || what > 2) return DARE_ERR_INVALID_ARG;
+  L->inject = what;
   return DARE_OK;
 }
 

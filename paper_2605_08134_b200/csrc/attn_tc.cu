@@ -79,16 +79,9 @@ constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 256;
 // S of stream 0 / 1: columns [0, 128) / [128, 256), P over the first 64 of them; O: [256, 384) / [384, 512)
 constexpr uint32_t kTmemCols = 512;
-#ifndef DARE_ATTN_PAIR_MIN_DENSE
-#define DARE_ATTN_PAIR_MIN_DENSE 128      // dense launches with longer windows take the two-tile kernel
-#endif
-#ifndef DARE_ATTN_PAIR_MIN_SPARSE
-#define DARE_ATTN_PAIR_MIN_SPARSE 1024    // row-sparse launches from this window length on
-#endif
-#ifndef DARE_RESCALE_STEP
-#define DARE_RESCALE_STEP 8.f
-#endif
-constexpr float kRescaleStep = DARE_RESCALE_STEP;     // log2 of the growth of the running maximum that triggers a rescale of O
+constexpr int kPairMinDense = 128;      // dense launches with longer windows take the two-tile kernel
+constexpr int kPairMinSparse = 1024;    // row-sparse launches from this window length on
+constexpr float kRescaleStep = 8.f;     // log2 of the growth of the running maximum that triggers a rescale of O
 
 }  // namespace
 
@@ -179,8 +172,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   if (p.idx != nullptr) {
     const int lo = __ldcg(p.batch_off + b), hi = __ldcg(p.batch_off + b + 1);
     row0 = lo + tile * BQ;
-    active = row0 < hi;
-    rows_valid = min(BQ, hi - row0);
+    active = slice_ok(lo, hi, g.tokens(), p.status) && row0 < hi;
+    rows_valid = active ? min(BQ, hi - row0) : 0;
   } else {
     row0 = b * g.seq_act + tile * BQ;
     rows_valid = min(BQ, g.seq_act - tile * BQ);
@@ -222,6 +215,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int u = u0 + k * kGather, r = u >> 4;              // 16 units of 8 bf16 per row
       tok[k] = -1;
       if (u < BQ * 16 && r < rows_valid) tok[k] = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
+      if (p.idx && tok[k] >= 0 && !token_ok(tok[k], g.tokens(), p.status)) tok[k] = -1;      // read as a row of zeros
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
@@ -440,8 +434,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (ksplit == 1) {
       // normalise, store
       const float inv = 1.f / l_row;
-      if (r < rows_valid) {
-        const int t = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
+      const int t = r < rows_valid ? (p.idx ? __ldcg(p.idx + row0 + r) : row0 + r) : -1;
+      if (t >= 0 && (p.idx == nullptr || token_ok(t, g.tokens(), p.status))) {      // (else: no cache row to write)
         __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + st * 64;
 #pragma unroll
         for (int i = 0; i < 64; ++i) acc[i] *= inv;
@@ -515,6 +509,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
       const float inv = 1.f / lsum;
       const int t = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
+      if (p.idx != nullptr && !token_ok(t, g.tokens(), p.status)) continue;        // no cache row to write
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + 4 * lane;
       __nv_bfloat162 lo2 = __floats2bfloat162_rn(o.x * inv, o.y * inv), hi2 = __floats2bfloat162_rn(o.z * inv, o.w * inv);
       uint2 packed;
@@ -637,8 +632,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   if (p.idx != nullptr) {
     const int lo = __ldcg(p.batch_off + b), hi = __ldcg(p.batch_off + b + 1);
     row0 = lo + tile * kPairRows;
-    active = row0 < hi;
-    rows_all = min(kPairRows, hi - row0);
+    active = slice_ok(lo, hi, g.tokens(), p.status) && row0 < hi;
+    rows_all = active ? min(kPairRows, hi - row0) : 0;
   } else {
     row0 = b * g.seq_act + tile * kPairRows;
     rows_all = min(kPairRows, g.seq_act - tile * kPairRows);
@@ -678,6 +673,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int u = u0 + k * kGather, r = u >> 4;
       tok[k] = -1;
       if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
+      if (p.idx && tok[k] >= 0 && !token_ok(tok[k], g.tokens(), p.status)) tok[k] = -1;      // read as a row of zeros
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
@@ -856,10 +852,11 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // ---- normalise and store this row (the tensor-memory loads are warp-wide; rows past the tile's end only skip
     // the store)
     {
-      const bool ok = r < rows_valid;
+      bool ok = r < rows_valid;
       const float inv = 1.f / l;
       const int rr = st * BQ + (ok ? r : 0);
-      const int t = p.idx ? __ldcg(p.idx + row0 + rr) : row0 + rr;
+      int t = p.idx ? __ldcg(p.idx + row0 + rr) : row0 + rr;
+      if (p.idx != nullptr && ok && !token_ok(t, g.tokens(), p.status)) { ok = false; t = 0; }   // no cache row to write
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
@@ -905,8 +902,8 @@ cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v
   // windows are where refresh sets of several tiles are.
   const int tps2 = (p.g.seq_act + kPairRows - 1) / kPairRows;
   const bool pair = ksplit == 1 &&
-                    (p.idx ? p.g.seq_act >= DARE_ATTN_PAIR_MIN_SPARSE && p.g.n_heads * p.g.batch >= 64
-                           : p.g.seq_act > DARE_ATTN_PAIR_MIN_DENSE && p.g.n_heads * p.g.batch * tps2 >= 148);
+                    (p.idx ? p.g.seq_act >= kPairMinSparse && p.g.n_heads * p.g.batch >= 64
+                           : p.g.seq_act > kPairMinDense && p.g.n_heads * p.g.batch * tps2 >= 148);
   if (pair) {
     dim3 grid(p.g.n_heads, p.g.batch * tps2, 1);
     if (grid.y == 0) return cudaSuccess;

@@ -424,6 +424,26 @@ void launch_select(const float* scores, float tau, bool select_all, const StepGe
                scores, tau, all, g, idx, count, batch_off, delta, late);
 }
 
+// ------------------------------------------------------------------------------------------------ diagnostics
+// A wait nobody ends, with a short limit: the bounded wait of the tensor-core kernels on a barrier no thread and no
+// copy ever arrives on.  It must give up after `limit_ns`, record the time-out in the status word and return normally.
+__global__ void wait_probe_kernel(int* status, unsigned long long limit_ns, unsigned long long* waited_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  const unsigned long long t0 = ptx::globaltimer_ns();
+  const bool ok = ptx::mbar_wait(&bar, 0, status, limit_ns);
+  if (threadIdx.x == 0 && waited_ns) *waited_ns = ok ? 0ull : ptx::globaltimer_ns() - t0;
+}
+void launch_wait_probe(int* status, unsigned long long limit_ns, unsigned long long* waited_ns, cudaStream_t st) {
+  wait_probe_kernel<<<1, 32, 0, st>>>(status, limit_ns, waited_ns);
+}
+__global__ void poke_int_kernel(int* dst, int value) { *dst = value; }
+void launch_poke_int(int* dst, int value, cudaStream_t st) { poke_int_kernel<<<1, 1, 0, st>>>(dst, value); }
+
 // ------------------------------------------------------------------------------------------------ reused rows
 // One warp per token row; rows refreshed in this step (staleness 0) are written by the projection itself.
 template <typename T>
@@ -477,14 +497,15 @@ void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, 
 template <typename T>
 __global__ void __launch_bounds__(256) gather_step_rows_kernel(const T* __restrict__ src, const int* __restrict__ idx,
                                                                const int* __restrict__ count, T* __restrict__ dst,
-                                                               StepGeom g, int by_cache_row) {
+                                                               StepGeom g, int by_cache_row, int* status) {
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
-  const int n = min(*count, g.tokens());
+  const int n = checked_count(*count, g.tokens(), status);
   constexpr int N = 16 / sizeof(T);
   const int nvec = g.d / N;
   for (int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += gridDim.x * (blockDim.x >> 5)) {
     const int tok = idx[r];
+    if (!token_ok(tok, g.tokens(), status)) continue;      // the row of the compact copy keeps what it held
     const size_t srow = by_cache_row ? (size_t)g.cache_row(tok) : (size_t)tok;
     const uint4* s = reinterpret_cast<const uint4*>(src + srow * g.d);
     uint4* o = reinterpret_cast<uint4*>(dst + (size_t)r * g.d);
@@ -493,14 +514,15 @@ __global__ void __launch_bounds__(256) gather_step_rows_kernel(const T* __restri
 }
 template <typename T>
 void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
-                             cudaStream_t st) {
+                             cudaStream_t st, int* status) {
   const int T_ = g.tokens();
   if (T_ <= 0) return;
   const int grid = (T_ + 7) / 8 < 148 * 8 ? (T_ + 7) / 8 : 148 * 8;
-  launch_pdl(gather_step_rows_kernel<T>, dim3(grid), dim3(256), 0, st, 1, src, idx, count, dst, g, by_cache_row ? 1 : 0);
+  launch_pdl(gather_step_rows_kernel<T>, dim3(grid), dim3(256), 0, st, 1, src, idx, count, dst, g, by_cache_row ? 1 : 0,
+             status);
 }
 template void launch_gather_step_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*,
-                                                     const StepGeom&, bool, cudaStream_t);
+                                                     const StepGeom&, bool, cudaStream_t, int*);
 template void launch_gather_rows<float>(const float*, const int*, const int*, float*, int, int, cudaStream_t);
 template void launch_gather_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*, int, int,
                                                 cudaStream_t);

@@ -15,6 +15,33 @@ constexpr int kDevOk = 0;
 constexpr int kDevTimeout = DARE_ERR_TIMEOUT;
 constexpr int kDevCheck = DARE_ERR_DEVICE_CHECK;
 
+#ifdef __CUDACC__
+// Range checks on what a kernel reads from the device-side selection before it uses it as an address: a token of the
+// refresh list must be a token of the step, the list's length and a sequence's slice of it must lie inside the step.
+// A value that fails is recorded in the layer's status word (DARE_ERR_DEVICE_CHECK; the first error of a handle stays)
+// and the access that would have used it is skipped.  They cost a compare per index and stand in for a memory checker.
+__device__ __forceinline__ void flag_device_check(int* status) {
+  if (status) atomicCAS(status, kDevOk, kDevCheck);
+}
+__device__ __forceinline__ bool token_ok(int tok, int n_tokens, int* status) {
+  if ((unsigned)tok < (unsigned)n_tokens) return true;
+  flag_device_check(status);
+  return false;
+}
+// the list's length, clamped into [0, cap]
+__device__ __forceinline__ int checked_count(int count, int cap, int* status) {
+  if ((unsigned)count <= (unsigned)cap) return count;
+  flag_device_check(status);
+  return count < 0 ? 0 : cap;
+}
+// a sequence's slice [lo, hi) of a list of at most cap entries; an impossible slice is flagged and read as empty
+__device__ __forceinline__ bool slice_ok(int lo, int hi, int cap, int* status) {
+  if (lo >= 0 && lo <= hi && hi <= cap) return true;
+  flag_device_check(status);
+  return false;
+}
+#endif
+
 // Geometry of one step, passed by value to kernels.
 struct StepGeom {
   int batch;      // B
@@ -95,7 +122,11 @@ void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, 
 // dst[r, :] = src[idx[r] (or its cache row), :] for the rows of a step's refresh set
 template <typename T>
 void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
-                             cudaStream_t st);
+                             cudaStream_t st, int* status = nullptr);
+
+// diagnostics: a bounded wait that nothing ends (one CTA, one barrier); a single int written in stream order
+void launch_wait_probe(int* status, unsigned long long limit_ns, unsigned long long* waited_ns, cudaStream_t st);
+void launch_poke_int(int* dst, int value, cudaStream_t st);
 
 // ---- stand-alone score / compaction for large token counts (select_large.cu)
 int select_large_tiles(long long n);
@@ -109,7 +140,7 @@ size_t select_large_flag_bytes(long long n);   // bytes of the decision words fo
 // rows m >= *count (when count != nullptr) are skipped.
 template <typename T>
 void launch_gemm_simt(const T* a, const int* a_idx, const int* count, const T* w, float* c, int m_max, int n, int k,
-                      int ldc, cudaStream_t st);
+                      int ldc, cudaStream_t st, int a_rows = 0, int* status = nullptr);   // a_rows: rows of a that a_idx may name
 // Q post-pass: score of the scoring head against q_prev (fp32, cache rows), q_prev update, rotary embedding,
 // store Q in the layer dtype.
 template <typename T>
@@ -118,12 +149,12 @@ void launch_q_post_simt(const float* qf, int ldq, const float* rope_cs, float* q
 // K/V post-pass: rows r < *count (or all when idx == nullptr): rotary embedding on K, store K and V to cache rows.
 template <typename T>
 void launch_kv_post_simt(const float* kvf, int ld, const int* idx, const int* count, const float* rope_cs, T* kc,
-                         T* vc, const StepGeom& g, cudaStream_t st);
+                         T* vc, const StepGeom& g, cudaStream_t st, int* status = nullptr);
 // Attention: query rows = idx[0..count) (or all rows when idx == nullptr), one warp per (row, head);
 // output rows go to the O cache.
 template <typename T>
 void launch_attention_simt(const T* q, const T* kc, const T* vc, const int* idx, const int* count, T* oc,
-                           const StepGeom& g, cudaStream_t st);
+                           const StepGeom& g, cudaStream_t st, int* status = nullptr);
 // y[t, :] = W_O oc[cache_row(t), :]
 template <typename T>
 void launch_out_proj_simt(const T* oc, const T* w_o, float* tmp, T* y, const StepGeom& g, cudaStream_t st);

@@ -133,7 +133,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   if (dbg && threadIdx.x == 0) p.debug[1] = globaltimer_ns();
 
   const int KB = p.K / BK;
-  const int n_rows = GATHER ? min(*p.count, p.m_total) : 0;
+  const int n_rows = GATHER ? checked_count(*p.count, p.m_total, p.status) : 0;
   // (PAIR: units = column tiles x pairs of row tiles; this CTA's row tile of unit u is 2 * (u / n_tiles) + pr, and
   // a row tile past the end of an odd count runs the main loop for its partner's sake and finishes no rows)
   const int m_tiles_live = GATHER ? (n_rows + BM - 1) / BM : p.m_tiles;
@@ -235,8 +235,12 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       // gathered rows: lane L holds the token of the warp's row L (-1 past the refresh set), lane-to-lane below
       int tok_own = -1, tok_first = 0;
       if (GATHER) {
-        if (q * 32 + lane < t.rows_valid) tok_own = p.idx[t.t0 + q * 32 + lane];
+        if (q * 32 + lane < t.rows_valid) {
+          tok_own = p.idx[t.t0 + q * 32 + lane];
+          if (!token_ok(tok_own, p.g.tokens(), p.status)) tok_own = -1;     // no row to write
+        }
         tok_first = t.rows_valid > 0 ? p.idx[t.t0] : 0;  // a row that exists, for the table reads of rows that do not
+        if ((unsigned)tok_first >= (unsigned)p.g.tokens()) tok_first = 0;
       }
       const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !t.is_b1);
       const int head0 = t.n0 / HD;
@@ -288,6 +292,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             size_t crowr = t.crow0 + rc;
             if (GATHER) {
               const int tk = __shfl_sync(0xffffffffu, tok_own, rr);
+              if (tk < 0) ok[k] = false;                 // (a token that failed its range check: the row is dropped)
               tokr = ok[k] ? tk : tok_first;
               pos = p.g.position(tokr);
               crowr = (size_t)p.g.cache_row(tokr);

@@ -55,15 +55,9 @@ struct Cfg {
 
 // Finishing pass, per warp: RB rows at a time (rows rl0, rl0 + #warps, ...); their table reads are issued together.
 // Warps of a CTA: producer, MMA issuer, the rest wait for the accumulator; all of them finish rows.
-#ifndef DARE_GEMM_WARPS_NARROW
-#define DARE_GEMM_WARPS_NARROW 6
-#endif
-#ifndef DARE_GEMM_WARPS_WIDE
-#define DARE_GEMM_WARPS_WIDE 8
-#endif
 template <int BN>
 struct Warps {
-  static constexpr int N = BN == 128 ? DARE_GEMM_WARPS_NARROW : DARE_GEMM_WARPS_WIDE;
+  static constexpr int N = BN == 128 ? 6 : 8;   // (eight warps on the 128-wide gathered projection: faster kernel, slower step)
   static constexpr int RB = N == 8 ? 4 : 6;          // rows a warp finishes at a time
 };
 template <int RB>
@@ -91,6 +85,7 @@ __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParam
     int pos;
     if (p.idx) {
       rb.tok[k] = p.idx[t0 + rc];
+      if (!token_ok(rb.tok[k], p.g.tokens(), p.status)) { rb.tok[k] = 0; rb.ok[k] = false; }   // no row to write
       pos = p.g.position(rb.tok[k]);
       rb.crow[k] = (size_t)p.g.cache_row(rb.tok[k]);
     } else {
@@ -163,7 +158,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const bool likely = p.count == nullptr || mt == 0;
   if (!likely) {
     pdl_wait();
-    if (mt * BM >= min(*p.count, p.m_total)) return;     // uniform over the cluster
+    if (mt * BM >= checked_count(*p.count, p.m_total, p.status)) return;     // uniform over the cluster
   }
   // Gathered A operand: the four epilogue warps fetch the rows of the refresh set themselves, 16 bytes at a time,
   // into the swizzled tile layout (the TMA producer then only brings the W tiles); each of them arrives on a stage
@@ -228,7 +223,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   size_t crow0 = 0;
   bool active = true;
   if (p.count != nullptr) {
-    const int n = min(*p.count, p.m_total);
+    const int n = checked_count(*p.count, p.m_total, p.status);
     t0 = mt * BM;
     active = t0 < n;
     rows_valid = min(BM, n - t0);
@@ -340,7 +335,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // (a gathering warp asks for its rows' tokens before the table reads below stall on theirs: one round trip, not two)
     const int r_own = quarter * 32 + lane;                     // the row whose token this lane looks up
     int tok_own = -1;
-    if (gather && warp < 6 && r_own < rows_valid) tok_own = p.idx[t0 + r_own];
+    if (gather && warp < 6 && r_own < rows_valid) {
+      tok_own = p.idx[t0 + r_own];
+      if (!token_ok(tok_own, p.g.tokens(), p.status)) tok_own = -1;      // read as a row of zeros
+    }
     load_row_batch<EPI, RB, kWarps, BN>(rb, p, warp, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
     if (gather && warp < 6) {
       // One stage of the A tile = 128 rows x 128 bytes (64 k-elements).  A warp takes 32 rows; one of its copy

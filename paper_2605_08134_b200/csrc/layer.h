@@ -58,6 +58,7 @@ struct dare_layer {
   cudaEvent_t prof_ev[dare::kMaxMarks + 1];
   bool prof_ev_ready;
   bool debug_on;
+  int inject;       // diagnostics: what the next step's selection is overwritten with (0 = nothing); see dare.h
   // asynchronous host-buffer steps: copy streams and the events that order staging-buffer reuse (created on first use)
   bool host_async_ready;
   cudaStream_t copy_in, copy_out;
@@ -76,6 +77,7 @@ inline void prof_begin(dare_layer* L) { L->prof_n = 0; }
 inline void prof_end(dare_layer* L, cudaStream_t st) {
   if (L->prof_on) cudaEventRecord(L->prof_ev[L->prof_n], st);
 }
+void inject_selection_error(dare_layer* L, const StepGeom& g, cudaStream_t st);
 dare_status_t tc_create(dare_layer* L);
 void tc_destroy(dare_layer* L);
 // add_input: y = x + W_O O instead of y = W_O O (the residual connection of a transformer block)

@@ -160,9 +160,11 @@ __global__ void __launch_bounds__(kThreads) tile_scan_kernel(const int* __restri
 // pass 3: from the decision bits alone (4 bytes per thread instead of 128 bytes of scores).  One thread per word of
 // 32 consecutive scores, 512 threads per tile: one scan of the words' popcounts places every thread, which then
 // writes the indices of its set bits, ascending, at consecutive places.
+// No store goes past entry n - 1 of the list, whatever the offsets say: if another call raced on a shared scratch
+// array, the list is wrong but the caller's buffer is the only memory written.
 __global__ void __launch_bounds__(kTileWords) tile_scatter_kernel(const unsigned* __restrict__ flags,
                                                                   const int* __restrict__ tile_offsets,
-                                                                  int* __restrict__ idx) {
+                                                                  int* __restrict__ idx, long long n) {
   __shared__ int warp_sums[32];
   __shared__ int total;
   ptx::pdl_wait();                         // before any read: decisions (two kernels back) and offsets (one back)
@@ -171,7 +173,8 @@ __global__ void __launch_bounds__(kTileWords) tile_scatter_kernel(const unsigned
   out += block_exclusive_scan<int>(__popc(word), warp_sums, &total);
   const int i0 = (int)((long long)blockIdx.x * kTile) + (int)threadIdx.x * 32;
   while (word != 0u) {
-    idx[out++] = i0 + __ffs((int)word) - 1;
+    if (out >= 0 && out < n) idx[out] = i0 + __ffs((int)word) - 1;
+    ++out;
     word &= word - 1u;
   }
 }
@@ -200,7 +203,7 @@ cudaError_t launch_select_large(const float* scores, long long n, float tau, int
                              tile_offsets, count);
   if (e != cudaSuccess) return e;
   e = launch_pdl(tile_scatter_kernel, dim3(tiles), dim3(kTileWords), 0, st, 1, (const unsigned*)flags,
-                 (const int*)tile_offsets, idx);
+                 (const int*)tile_offsets, idx, n);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }

@@ -24,6 +24,8 @@ struct ARowMap {
   const int* idx;   // gathered rows, or nullptr
   int use_cache_row;
   StepGeom g;
+  int a_rows;       // rows of A an index may name (range check)
+  int* status;
 };
 
 template <typename T, typename TC>
@@ -31,7 +33,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a,
                                                         const int* __restrict__ count, const T* __restrict__ w,
                                                         TC* __restrict__ c, int m_max, int n, int k, int ldc) {
   constexpr int BM = 64, BN = 64, BK = 16;
-  const int m_eff = count ? min(*count, m_max) : m_max;
+  const int m_eff = count ? checked_count(*count, m_max, map.status) : m_max;
   const int m0 = blockIdx.y * BM;
   if (m0 >= m_eff) return;
   const int n0 = blockIdx.x * BN;
@@ -40,9 +42,15 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a,
   const int tid = threadIdx.x;
   const int lrow = tid >> 2, lk = (tid & 3) * 4;
   const int gm = m0 + lrow;
-  const bool a_ok = gm < m_eff;
+  bool a_ok = gm < m_eff;
   size_t a_row = 0;
-  if (a_ok) a_row = map.idx ? (size_t)map.idx[gm] : (map.use_cache_row ? (size_t)map.g.cache_row(gm) : (size_t)gm);
+  if (a_ok && map.idx) {
+    const int t = map.idx[gm];
+    a_ok = token_ok(t, map.a_rows, map.status);          // a row that is not a row of A is read as zeros
+    a_row = a_ok ? (size_t)t : 0;
+  } else if (a_ok) {
+    a_row = map.use_cache_row ? (size_t)map.g.cache_row(gm) : (size_t)gm;
+  }
   const bool w_ok = (n0 + lrow) < n;
   const T* ap = a + a_row * k + lk;
   const T* wp = w + (size_t)(n0 + lrow) * k + lk;
@@ -81,23 +89,23 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a,
 
 template <typename T>
 void launch_gemm_simt(const T* a, const int* a_idx, const int* count, const T* w, float* c, int m_max, int n, int k,
-                      int ldc, cudaStream_t st) {
+                      int ldc, cudaStream_t st, int a_rows, int* status) {
   if (m_max <= 0) return;
-  ARowMap map{a_idx, 0, StepGeom{}};
+  ARowMap map{a_idx, 0, StepGeom{}, a_rows > 0 ? a_rows : m_max, status};
   dim3 grid((n + 63) / 64, (m_max + 63) / 64);
   gemm_simt_kernel<T, float><<<grid, 256, 0, st>>>(a, map, count, w, c, m_max, n, k, ldc);
 }
 template void launch_gemm_simt<float>(const float*, const int*, const int*, const float*, float*, int, int, int, int,
-                                      cudaStream_t);
+                                      cudaStream_t, int, int*);
 template void launch_gemm_simt<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, const __nv_bfloat16*,
-                                              float*, int, int, int, int, cudaStream_t);
+                                              float*, int, int, int, int, cudaStream_t, int, int*);
 
 template <typename T>
 void launch_out_proj_simt(const T* oc, const T* w_o, float* tmp, T* y, const StepGeom& g, cudaStream_t st) {
   (void)tmp;
   const int T_ = g.tokens();
   if (T_ <= 0) return;
-  ARowMap map{nullptr, 1, g};
+  ARowMap map{nullptr, 1, g, 0, nullptr};
   dim3 grid((g.d + 63) / 64, (T_ + 63) / 64);
   gemm_simt_kernel<T, T><<<grid, 256, 0, st>>>(oc, map, nullptr, w_o, y, T_, g.d, g.d, g.d);
 }
@@ -179,10 +187,11 @@ template <typename T>
 __global__ void __launch_bounds__(128) kv_post_kernel(const float* __restrict__ kvf, int ld,
                                                       const int* __restrict__ idx, const int* __restrict__ count,
                                                       const float2* __restrict__ rope_cs, T* __restrict__ kc,
-                                                      T* __restrict__ vc, StepGeom g) {
+                                                      T* __restrict__ vc, StepGeom g, int* status) {
   const int r = blockIdx.x;
-  if (count && r >= *count) return;
+  if (count && r >= checked_count(*count, g.tokens(), status)) return;
   const int t = idx ? idx[r] : r;
+  if (idx && !token_ok(t, g.tokens(), status)) return;   // no cache row to write
   const int hd = g.head_dim, half = hd >> 1, d = g.d;
   const size_t cr = (size_t)g.cache_row(t);
   const float* krow = kvf + (size_t)r * ld;
@@ -202,15 +211,15 @@ __global__ void __launch_bounds__(128) kv_post_kernel(const float* __restrict__ 
 
 template <typename T>
 void launch_kv_post_simt(const float* kvf, int ld, const int* idx, const int* count, const float* rope_cs, T* kc,
-                         T* vc, const StepGeom& g, cudaStream_t st) {
+                         T* vc, const StepGeom& g, cudaStream_t st, int* status) {
   if (g.tokens() <= 0) return;
   kv_post_kernel<T><<<g.tokens(), 128, 0, st>>>(kvf, ld, idx, count, reinterpret_cast<const float2*>(rope_cs), kc, vc,
-                                                g);
+                                                g, status);
 }
 template void launch_kv_post_simt<float>(const float*, int, const int*, const int*, const float*, float*, float*,
-                                         const StepGeom&, cudaStream_t);
+                                         const StepGeom&, cudaStream_t, int*);
 template void launch_kv_post_simt<__nv_bfloat16>(const float*, int, const int*, const int*, const float*,
-                                                 __nv_bfloat16*, __nv_bfloat16*, const StepGeom&, cudaStream_t);
+                                                 __nv_bfloat16*, __nv_bfloat16*, const StepGeom&, cudaStream_t, int*);
 
 // ------------------------------------------------------------------------------------------------ attention
 // Eq. 4 / Alg. 2 line 8 (row-sparse) and Alg. 1 line 10 (all rows): bidirectional softmax attention, no mask,
@@ -220,13 +229,14 @@ template <typename T, int EPL>
 __global__ void __launch_bounds__(128) attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ kc,
                                                              const T* __restrict__ vc, const int* __restrict__ idx,
                                                              const int* __restrict__ count, T* __restrict__ oc,
-                                                             StepGeom g, int rows_max) {
+                                                             StepGeom g, int rows_max, int* status) {
   const int task = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int r = task / g.n_heads, h = task - r * g.n_heads;
-  const int n_rows = count ? min(*count, rows_max) : rows_max;
+  const int n_rows = count ? checked_count(*count, rows_max, status) : rows_max;
   if (r >= n_rows) return;
   const int t = idx ? idx[r] : r;
+  if (idx && !token_ok(t, rows_max, status)) return;     // neither a query row to read nor a cache row to write
   const int b = t / g.seq_act;
   const int hd = g.head_dim, d = g.d;
   const float scale = rsqrtf((float)hd);
@@ -261,23 +271,23 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(const T* __restrict
 
 template <typename T>
 void launch_attention_simt(const T* q, const T* kc, const T* vc, const int* idx, const int* count, T* oc,
-                           const StepGeom& g, cudaStream_t st) {
+                           const StepGeom& g, cudaStream_t st, int* status) {
   const int rows_max = g.tokens();
   if (rows_max <= 0) return;
   const long tasks = (long)rows_max * g.n_heads;
   const int grid = (int)((tasks + 3) / 4);
   switch (g.head_dim / 32) {
-    case 1: attention_simt_kernel<T, 1><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max); break;
-    case 2: attention_simt_kernel<T, 2><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max); break;
-    case 4: attention_simt_kernel<T, 4><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max); break;
-    case 8: attention_simt_kernel<T, 8><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max); break;
+    case 1: attention_simt_kernel<T, 1><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max, status); break;
+    case 2: attention_simt_kernel<T, 2><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max, status); break;
+    case 4: attention_simt_kernel<T, 4><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max, status); break;
+    case 8: attention_simt_kernel<T, 8><<<grid, 128, 0, st>>>(q, kc, vc, idx, count, oc, g, rows_max, status); break;
     default: break;  // rejected at creation
   }
 }
 template void launch_attention_simt<float>(const float*, const float*, const float*, const int*, const int*, float*,
-                                           const StepGeom&, cudaStream_t);
+                                           const StepGeom&, cudaStream_t, int*);
 template void launch_attention_simt<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
                                                    const int*, const int*, __nv_bfloat16*, const StepGeom&,
-                                                   cudaStream_t);
+                                                   cudaStream_t, int*);
 
 }  // namespace dare

@@ -17,25 +17,10 @@ struct TcState {
 
 namespace {
 
-#ifndef DARE_PAIR_MMA
-#define DARE_PAIR_MMA 1
-#endif
-bool use_pairs(int n_tiles, int m_tiles, int splits) { return DARE_PAIR_MMA != 0 && pairs_pay(n_tiles, m_tiles, splits); }
-#ifndef DARE_NARROW_PAIRS
-#define DARE_NARROW_PAIRS 1
-#endif
-#ifndef DARE_PERSIST_PAIR
-#define DARE_PERSIST_PAIR 1
-#endif
+bool use_pairs(int n_tiles, int m_tiles, int splits) { return pairs_pay(n_tiles, m_tiles, splits); }
 // units (column tile x pair of row tiles) from which the two-CTA form of a listed launch runs: two rounds of the 74 clusters
 constexpr int kPairUnitGate = 148;
-#ifndef DARE_PERSIST_LIST
-#define DARE_PERSIST_LIST 1
-#endif
-#ifndef DARE_PERSIST
-#define DARE_PERSIST 1
-#endif
-bool use_persist(int n_tiles, int m_tiles, int splits) { return DARE_PERSIST != 0 && persist_pays(n_tiles, m_tiles, splits); }
+bool use_persist(int n_tiles, int m_tiles, int splits) { return persist_pays(n_tiles, m_tiles, splits); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -148,11 +133,10 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     const int n_tiles = d / 256;
     prof_mark(L, SLOT_Q_GEMM, st);
     const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-    if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
+    if (narrow_pairs_pay(d, m_tiles_dense, kblocks))
       e = launch_gemm_tc(EPI_Q, 128, S.a_xn, S.w_q64, S.w_q64, p, d / 128, m_tiles_dense, 2, st, 1);
     else if (use_persist(n_tiles, m_tiles_dense, sp))
-      e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_Q, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, st, 1)
-                               : launch_gemm_persist(EPI_Q, S.a_xn, S.w_q, S.w_q, p, n_tiles, m_tiles_dense, st));
+      e = launch_gemm_persist(EPI_Q, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, st, 1);
     else if (use_pairs(n_tiles, m_tiles_dense, sp))
       e = launch_gemm_tc(EPI_Q, 256, S.a_xn, S.w_q128, S.w_q128, p, n_tiles, m_tiles_dense, sp, st, 1);
     else
@@ -173,6 +157,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     // (a selection that refreshes everything reads no scores: behind the two projections it runs beside them)
     launch_select(B.scores, tau, select_all, g, B.idx, B.count, B.batch_off, B.delta, st, kv_beside_q && select_all);
     ++launches;
+    if (L->inject) inject_selection_error(L, g, st);
   };
   if (!kv_beside_q) select_now();
   // K/V projection with rotary embedding and cache scatter
@@ -196,10 +181,10 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
                            pick_splits(n_tiles128, kblocks), st); ++launches;
       } else {
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
-        if (DARE_PERSIST_LIST && use_persist(n_tiles, m_tiles, 1) && compact_ok) {
+        if (use_persist(n_tiles, m_tiles, 1) && compact_ok) {
           // a compact copy of the refresh set's rows first (a stream of n x d elements), then the projection with
           // every operand through TMA and two-CTA MMAs
-          launch_gather_step_rows((const bf16*)B.xn, B.idx, B.count, (bf16*)B.x_stage, g, false, st); ++launches;
+          launch_gather_step_rows((const bf16*)B.xn, B.idx, B.count, (bf16*)B.x_stage, g, false, st, B.status); ++launches;
           p.gather_src = nullptr;
           p.unit_gate = kPairUnitGate;
           e = launch_gemm_persist(EPI_KV, S.a_xg, S.w_k128, S.w_v128, p, n_tiles, m_tiles, st, 1); ++launches;
@@ -213,8 +198,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       p.wait_at_end = kv_beside_q ? 1 : 0;
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
       if (use_persist(n_tiles, m_tiles_dense, sp))
-        e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_KV, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, st, 1)
-                               : launch_gemm_persist(EPI_KV, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles_dense, st));
+        e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, st, 1);
       else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k128, S.w_v128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else
@@ -255,8 +239,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     prof_mark(L, SLOT_OUT_GEMM, st);
     if (y_sparse) {
       p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.oc; p.gather_cache_rows = 1;
-      if (DARE_PERSIST_LIST && use_persist(n_tiles, (T_ + 127) / 128, 1) && compact_ok) {
-        launch_gather_step_rows((const bf16*)B.oc, B.idx, B.count, (bf16*)B.x_stage, g, true, st); ++launches;
+      if (use_persist(n_tiles, (T_ + 127) / 128, 1) && compact_ok) {
+        launch_gather_step_rows((const bf16*)B.oc, B.idx, B.count, (bf16*)B.x_stage, g, true, st, B.status); ++launches;
         p.gather_src = nullptr;
         p.unit_gate = kPairUnitGate;
         e = launch_gemm_persist(EPI_OUT, S.a_xg, S.w_o128, S.w_o128, p, n_tiles, (T_ + 127) / 128, st, 1); ++launches;
@@ -268,11 +252,10 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
       launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
     } else {
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
-      if (DARE_PAIR_MMA && DARE_NARROW_PAIRS && narrow_pairs_pay(d, m_tiles_dense, kblocks))
+      if (narrow_pairs_pay(d, m_tiles_dense, kblocks))
         e = launch_gemm_tc(EPI_OUT, 128, S.a_oc, S.w_o64, S.w_o64, p, d / 128, m_tiles_dense, 2, st, 1);
       else if (use_persist(n_tiles, m_tiles_dense, sp))
-        e = (DARE_PERSIST_PAIR ? launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, st, 1)
-                               : launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o, S.w_o, p, n_tiles, m_tiles_dense, st));
+        e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, st, 1);
       else if (use_pairs(n_tiles, m_tiles_dense, sp))
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o128, S.w_o128, p, n_tiles, m_tiles_dense, sp, st, 1);
       else

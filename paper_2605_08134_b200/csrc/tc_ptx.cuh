@@ -42,15 +42,18 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 // Bounded wait for the phase with the given parity.  Returns false (after flagging the status word) on time-out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
-  // once a wait of this launch has given up, the others do not wait again: the kernel runs out quickly
-  if (status && *reinterpret_cast<volatile int*>(status) != 0) return false;
+  // once a wait has given up, the others do not wait again: the kernel runs out quickly (a failed range check is no
+  // reason to stop waiting: its access was skipped and the rest of the launch is in order)
+  if (status && *reinterpret_cast<volatile int*>(status) == 7 /* DARE_ERR_TIMEOUT */) return false;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 0x3ffu) == 0 && globaltimer_ns() - t0 > 2000000000ull) {
-      if (status) atomicExch(status, 7 /* DARE_ERR_TIMEOUT */);
+    if ((++spins & 0x3ffu) == 0 && globaltimer_ns() - t0 > limit_ns) {
+      if (status) atomicExch(status, 7 /* DARE_ERR_TIMEOUT */);      // (takes the place of a recorded range-check failure)
       return false;
     }
   }

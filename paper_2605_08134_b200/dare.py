@@ -69,6 +69,9 @@ def _load():
         "dare_layer_reset": (C.c_int, [vp]),
         "dare_layer_destroy": (C.c_int, [vp]),
         "dare_layer_status": (C.c_int, [vp, vp]),
+        "dare_layer_clear_status": (C.c_int, [vp, vp]),
+        "dare_layer_debug_wait_probe": (C.c_int, [vp, C.c_uint64, C.POINTER(C.c_uint64), vp]),
+        "dare_layer_debug_inject": (C.c_int, [vp, C.c_int]),
         "dare_layer_last_selection": (C.c_int, [vp, vp, vp, vp, vp, vp, vp]),
         "dare_layer_read_caches": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "dare_layer_state_bytes": (sz, [vp]),
@@ -157,6 +160,21 @@ def dare_layer_destroy(handle) -> int:
 
 def dare_layer_status(handle, stream=0) -> int:
     return _lib.dare_layer_status(handle, stream)
+
+
+def dare_layer_clear_status(handle, stream=0) -> int:
+    return _lib.dare_layer_clear_status(handle, stream)
+
+
+def dare_layer_debug_wait_probe(handle, limit_ns, stream=0):
+    """-> (status, nanoseconds the probe's wait took before it gave up)."""
+    waited = C.c_uint64(0)
+    st = _lib.dare_layer_debug_wait_probe(handle, limit_ns, C.byref(waited), stream)
+    return st, int(waited.value)
+
+
+def dare_layer_debug_inject(handle, what) -> int:
+    return _lib.dare_layer_debug_inject(handle, what)
 
 
 def dare_layer_last_selection(handle, idx_ptr, count_ptr, batch_off_ptr, scores_ptr, delta_ptr, stream=0) -> int:
@@ -347,6 +365,22 @@ class Layer:
 
     def status(self) -> int:
         return dare_layer_status(self.handle, self._stream())
+
+    def clear_status(self):
+        st = dare_layer_clear_status(self.handle, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_clear_status")
+
+    def wait_probe(self, limit_ns):
+        st, waited = dare_layer_debug_wait_probe(self.handle, limit_ns, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_debug_wait_probe")
+        return waited
+
+    def inject(self, what):
+        st = dare_layer_debug_inject(self.handle, what)
+        if st != OK:
+            raise DareError(st, "dare_layer_debug_inject")
 
     def last_selection(self, batch, seq_act):
         """-> dict(idx, count, batch_off, scores, delta) as numpy arrays."""

@@ -1,7 +1,8 @@
 """The compaction entry point for callers that cannot allocate device memory (a server whose arena owns all of HBM,
 or a loop that cannot afford cudaMalloc's device-wide synchronisation): its scratch is a fixed array inside the
-library.  Checked against the entry point that takes caller scratch, on two calls in a row, the second smaller than
-the first so that the array still holds the first call's tile counts beyond the second call's range.
+library.  Checked against the entry point that takes caller scratch, on calls in a row: the second smaller than the
+first, so that the array still holds the first call's tile counts beyond the second call's range, the third as large as
+the array allows.
 
 Collected last on purpose: a failure here must not hide any other test from a run that stops at the first failure.
 """
@@ -28,7 +29,8 @@ def test_static_scratch_variant_matches_caller_scratch_variant_twice_in_a_row():
     stream = torch.cuda.current_stream().cuda_stream
     limit = dare.dare_select_compact_static_max_tokens()
     assert limit == 4096 * 4096
-    for call, (n, tau, seed) in enumerate([(3_000_017, 0.1, 1), (70_001, 0.5, 2)]):
+    # (the third call is exactly as large as the built-in array allows: all of its 1024 tiles in use)
+    for call, (n, tau, seed) in enumerate([(3_000_017, 0.1, 1), (70_001, 0.5, 2), (limit, 0.1, 3)]):
         s = torch.from_numpy(_scores(n, seed)).cuda()
         idx_a = torch.full((n,), -1, dtype=torch.int32, device="cuda")
         idx_b = torch.full((n,), -2, dtype=torch.int32, device="cuda")
