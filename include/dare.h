@@ -132,6 +132,20 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
 dare_status_t dare_layer_step(dare_layer_t* layer, const void* x, int batch, int seq_act, int pos_begin,
                               int mode, float threshold, void* y, void* cuda_stream);
 
+/* The same step with a threshold the step takes from its own scores (Sec. 3.1: dynamic thresholding; the reuse-rate
+ * allocation of that section turns a reuse rate into the matching quantile of the drift scores, and this is that
+ * quantile taken per step): the `reuse_count` tokens of the call that drifted least are reused, i.e.
+ *   tau_t = the reuse_count-th smallest drift score of the step's batch * seq_act tokens,
+ * and Eq. 2 is applied with it, so tokens tied with that score are reused as well.  reuse_count = 0 refreshes every
+ * token, reuse_count >= batch * seq_act reuses every token; NaN scores sort last and are never reused; negative is
+ * rejected.  tau_t is found on the device (an exact four-pass radix selection, one more kernel ahead of the
+ * selection) and never travels to the host; dare_layer_last_threshold reads it back afterwards (the threshold of
+ * the last step, whichever call gave it; synchronises the stream if the value is on the device).  A first step and
+ * mode = DENSE refresh everything as always.  reuse_count = floor(phi * batch * seq_act) gives the reuse rate phi. */
+dare_status_t dare_layer_step_quantile(dare_layer_t* layer, const void* x, int batch, int seq_act, int pos_begin,
+                                       int mode, int reuse_count, void* y, void* cuda_stream);
+dare_status_t dare_layer_last_threshold(dare_layer_t* layer, float* tau_host, void* cuda_stream);
+
 /* Same step with HOST buffers: copies x_host to the device, runs the step, copies y back and synchronises.
  * x_host / y_host should be pinned for full copy bandwidth. */
 dare_status_t dare_layer_step_host(dare_layer_t* layer, const void* x_host, int batch, int seq_act, int pos_begin,
@@ -229,6 +243,10 @@ dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint6
  * offsets, and one decision bit per score: about n_tokens / 8 bytes); n_tokens <= 2^30; NaN threshold is rejected. */
 dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t rows, int head_dim, float* scores,
                                 void* cuda_stream);
+/* *tau_out (device) = the k-th smallest of n_tokens float32 scores (k clamped to [0, n_tokens]; k = 0: -inf,
+ * k = n_tokens or beyond the scores that are numbers: +inf), the threshold that reuses the k least-drifted tokens under
+ * Eq. 2 (Sec. 3.1).  One CTA, exact; 1 <= n_tokens <= 2^24. */
+dare_status_t dare_score_kth(const float* scores, int64_t n_tokens, int64_t k, float* tau_out, void* cuda_stream);
 size_t dare_select_compact_scratch_bytes(int64_t n_tokens);
 dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float threshold, int32_t* idx, int32_t* count,
                                   void* scratch, size_t scratch_bytes, void* cuda_stream);

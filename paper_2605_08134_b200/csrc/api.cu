@@ -72,6 +72,7 @@ size_t carve(const dare_layer_config_t* c, bool use_tc, char* base, Buffers* b) 
   B.y_stage = take(Tm * d * e);
   B.tmp = use_tc ? nullptr : (float*)take(Tm * 2 * d * sizeof(float));
   B.yc = use_tc ? take(Tm * d * e) : nullptr;
+  B.tau_dev = (float*)take(sizeof(float));
   return off;
 }
 
@@ -91,6 +92,17 @@ dare_status_t check_handle(const dare_layer_t* L) {
 
 }  // namespace
 namespace dare {
+// A step that was asked to reuse its k least-drifted tokens works its threshold out from the scores the Q projection
+// just left (one more kernel ahead of the selection); returns where the selection finds it, or nullptr when the
+// caller's threshold applies (also on a first step and in dense mode, which refresh everything anyway).
+const float* step_threshold_on_device(dare_layer* L, const StepGeom& g, int mode, cudaStream_t st, int* launches) {
+  L->last_tau_on_device = false;
+  if (L->reuse_count < 0 || !L->has_prev || mode == DARE_MODE_DENSE) return nullptr;
+  launch_kth_score(L->buf.scores, g.tokens(), L->reuse_count, L->buf.tau_dev, st);
+  ++*launches;
+  L->last_tau_on_device = true;
+  return L->buf.tau_dev;
+}
 // Diagnostics (dare_layer_debug_inject): overwrites one value of the selection just made, once.
 void inject_selection_error(dare_layer* L, const StepGeom& g, cudaStream_t st) {
   if (L->inject == 1) launch_poke_int(L->buf.idx, g.tokens(), st);            // first list entry: one past the step's tokens
@@ -120,7 +132,9 @@ dare_status_t step_simt(dare_layer_t* L, const T* x, const StepGeom& g, int mode
   launch_q_post_simt<T>(B.tmp, d, B.rope_cs, B.q_prev, B.scores, has_prev, (T*)B.q, g, st); ++launches;
   // lines 4-5: refresh set as a compacted index list; Sec. 4 staleness
   prof_mark(L, SLOT_SELECT, st);
-  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st); ++launches;
+  const float* tau_dev = step_threshold_on_device(L, g, mode, st, &launches);
+  launch_select(B.scores, tau, !has_prev || mode == DARE_MODE_DENSE, g, B.idx, B.count, B.batch_off, B.delta, st, false,
+                tau_dev); ++launches;
   inject_selection_error(L, g, st);
   // K/V: Alg. 1 lines 6-9 (refresh set only) or Alg. 2 line 7 (all rows)
   const int* kv_idx = kv_sparse ? B.idx : nullptr;
@@ -182,6 +196,7 @@ dare_status_t enqueue_step(dare_layer_t* L, const void* x, int batch, int seq_ac
   if (!L->has_prev) { L->kv_len = seq_act; L->batch = batch; }
   L->has_prev = true;
   L->last_geom = g;
+  L->last_tau = tau;
   return DARE_OK;
 }
 
@@ -256,6 +271,9 @@ dare_status_t dare_layer_create(const dare_layer_config_t* cfg, const dare_layer
   L->prof_ev_ready = false;
   L->debug_on = false;
   L->inject = 0;
+  L->reuse_count = -1;
+  L->last_tau = 0.f;
+  L->last_tau_on_device = false;
   L->host_async_ready = false;
   memset(&L->last_geom, 0, sizeof(L->last_geom));
   carve(cfg, use_tc, (char*)workspace, &L->buf);
@@ -291,6 +309,39 @@ dare_status_t dare_layer_step(dare_layer_t* L, const void* x, int batch, int seq
   if (s != DARE_OK) return s;
   if (!aligned16(x) || !aligned16(y)) return DARE_ERR_ALIGN;
   return enqueue_step(L, x, batch, seq_act, pos_begin, mode, threshold, y, (cudaStream_t)cuda_stream);
+}
+
+dare_status_t dare_layer_step_quantile(dare_layer_t* L, const void* x, int batch, int seq_act, int pos_begin, int mode,
+                                       int reuse_count, void* y, void* cuda_stream) {
+  dare_status_t s = validate_step(L, x, batch, seq_act, pos_begin, mode, 0.f, y);
+  if (s != DARE_OK) return s;
+  if (!aligned16(x) || !aligned16(y)) return DARE_ERR_ALIGN;
+  if (reuse_count < 0) return DARE_ERR_INVALID_ARG;
+  L->reuse_count = reuse_count;
+  s = enqueue_step(L, x, batch, seq_act, pos_begin, mode, 0.f, y, (cudaStream_t)cuda_stream);
+  L->reuse_count = -1;
+  return s;
+}
+
+dare_status_t dare_layer_last_threshold(dare_layer_t* L, float* tau_host, void* cuda_stream) {
+  dare_status_t s = check_handle(L);
+  if (s != DARE_OK) return s;
+  if (!tau_host) return DARE_ERR_INVALID_ARG;
+  if (!L->has_prev) return DARE_ERR_STATE;
+  if (!L->last_tau_on_device) { *tau_host = L->last_tau; return DARE_OK; }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(cudaMemcpyAsync(tau_host, L->buf.tau_dev, sizeof(float), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return DARE_OK;
+}
+
+dare_status_t dare_score_kth(const float* scores, int64_t n_tokens, int64_t k, float* tau_out, void* cuda_stream) {
+  if (!scores || !tau_out) return DARE_ERR_INVALID_ARG;
+  if (n_tokens <= 0 || n_tokens > (int64_t)1 << 24) return DARE_ERR_SHAPE;
+  const int kk = k < 0 ? 0 : (k > n_tokens ? (int)n_tokens : (int)k);
+  launch_kth_score(scores, (int)n_tokens, kk, tau_out, (cudaStream_t)cuda_stream);
+  CUDA_TRY(cudaGetLastError());
+  return DARE_OK;
 }
 
 dare_status_t dare_layer_step_host(dare_layer_t* L, const void* x_host, int batch, int seq_act, int pos_begin, int mode,

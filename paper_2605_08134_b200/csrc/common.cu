@@ -267,16 +267,74 @@ template void launch_rmsnorm<__nv_bfloat16>(const __nv_bfloat16*, const float*, 
 // With more than one chunk the launch has one CTA per chunk, and none waits for another: a CTA first counts the
 // refreshed tokens of the chunks before its own from their scores (a few 16-byte loads per thread, from the L2), which
 // is where its part of the list starts.
+// ---- the step's own threshold (Sec. 3.1 speaks of dynamic thresholding; the reuse-rate allocation turns a rate into
+// the matching quantile of the drift scores): tau_t = the k-th smallest score of this step, so that the k tokens that
+// drifted least are reused (and every token tied with the k-th).  Exact selection by four passes over the scores'
+// order-preserving 32-bit keys, eight bits at a time (histogram in shared memory, then the bin that holds rank k);
+// one CTA: a step has at most a few 10^4 tokens.  NaN scores sort last and are never reused.
+// k <= 0: tau = -inf (nothing reused); k >= n or more than the scores that are numbers: +inf.
+__device__ __forceinline__ unsigned score_key(float s) {
+  if (s != s) return 0xffffffffu;
+  const unsigned u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__global__ void __launch_bounds__(1024) kth_score_kernel(const float* __restrict__ scores, int n, int k,
+                                                         float* __restrict__ tau_out) {
+  __shared__ int hist[256];
+  __shared__ unsigned s_prefix;
+  __shared__ int s_rank;
+  ptx::pdl_wait();
+  ptx::pdl_launch_dependents();
+  if (k <= 0 || k >= n) {
+    if (threadIdx.x == 0) *tau_out = __int_as_float(k <= 0 ? 0xff800000 : 0x7f800000);
+    return;
+  }
+  unsigned prefix = 0u, mask = 0u;
+  int rank = k;                                       // rank (1-based) of the wanted key among the keys that match the prefix
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const unsigned key = score_key(scores[i]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int cum = 0, b = 0;
+      for (; b < 255; ++b) {
+        if (cum + hist[b] >= rank) break;
+        cum += hist[b];
+      }
+      s_prefix = prefix | ((unsigned)b << shift);
+      s_rank = rank - cum;
+    }
+    __syncthreads();
+    prefix = s_prefix;
+    rank = s_rank;
+    mask |= 255u << shift;
+  }
+  if (threadIdx.x == 0) {
+    const unsigned u = (prefix & 0x80000000u) ? (prefix & 0x7fffffffu) : ~prefix;
+    float tau = __uint_as_float(u);
+    if (tau != tau) tau = __int_as_float(0x7f800000);         // rank k falls among the NaN scores: every number is reused
+    *tau_out = tau;
+  }
+}
+void launch_kth_score(const float* scores, int n, int k, float* tau_out, cudaStream_t st) {
+  launch_pdl(kth_score_kernel, dim3(1), dim3(1024), 0, st, 1, scores, n, k, tau_out);
+}
+
 constexpr int kSelPerThread = 4;
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
                                                       int* __restrict__ batch_off, int* __restrict__ delta,
-                                                      int wait_at_end) {
+                                                      int wait_at_end, const float* __restrict__ tau_dev) {
   __shared__ int warp_tot[32];
   __shared__ int before_chunk;
   if (threadIdx.x == 0) before_chunk = 0;
   if (!wait_at_end) ptx::pdl_wait();
   ptx::pdl_launch_dependents();
+  if (tau_dev != nullptr) tau = *tau_dev;                // the threshold the step worked out itself
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kChunk = 1024 * kSelPerThread;
@@ -363,11 +421,12 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
 __global__ void __launch_bounds__(1024) select_small_kernel(const float* __restrict__ scores, float tau, int select_all,
                                                       StepGeom g, int* __restrict__ idx, int* __restrict__ count,
                                                       int* __restrict__ batch_off, int* __restrict__ delta,
-                                                      int wait_at_end) {
+                                                      int wait_at_end, const float* __restrict__ tau_dev) {
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
   if (!wait_at_end) ptx::pdl_wait();
   ptx::pdl_launch_dependents();
+  if (tau_dev != nullptr) tau = *tau_dev;
   const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int base = 0;
@@ -414,14 +473,15 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float* __restr
 // beside_predecessor: the selection refreshes every token (it reads no scores) and nothing the kernel before it in the
 // stream touches, so it runs beside that kernel and waits for it only before it leaves.
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor) {
+                   int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor, const float* tau_dev) {
   const int all = (select_all || scores == nullptr) ? 1 : 0;
   const int late = (beside_predecessor && all) ? 1 : 0;
   if (g.tokens() <= 2048)
-    launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta, late);
+    launch_pdl(select_small_kernel, dim3(1), dim3(1024), 0, st, 1, scores, tau, all, g, idx, count, batch_off, delta, late,
+               tau_dev);
   else
     launch_pdl(select_kernel, dim3((g.tokens() + 1024 * kSelPerThread - 1) / (1024 * kSelPerThread)), dim3(1024), 0, st, 1,
-               scores, tau, all, g, idx, count, batch_off, delta, late);
+               scores, tau, all, g, idx, count, batch_off, delta, late, tau_dev);
 }
 
 // ------------------------------------------------------------------------------------------------ diagnostics

@@ -116,7 +116,10 @@ void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float
 template <typename T>
 void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st);
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
-                   int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor = false);
+                   int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor = false,
+                   const float* tau_dev = nullptr);   // tau_dev: read the threshold from device memory instead
+// *tau_out = the k-th smallest of n scores (see common.cu); one CTA
+void launch_kth_score(const float* scores, int n, int k, float* tau_out, cudaStream_t st);
 template <typename T>
 void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, int max_rows, int d, cudaStream_t st);
 // dst[r, :] = src[idx[r] (or its cache row), :] for the rows of a step's refresh set

@@ -25,6 +25,7 @@ struct Buffers {
   void* y_stage;
   void* yc;         // tensor-core path: cache of projected outputs y = W_O O by cache row (gathered output projection)
   float* tmp;       // SIMT path: fp32 projection results [T, 2d]
+  float* tau_dev;   // [1] threshold of a step that takes it from its own scores (dare_layer_step_quantile)
 };
 
 struct TcState;
@@ -58,6 +59,9 @@ struct dare_layer {
   cudaEvent_t prof_ev[dare::kMaxMarks + 1];
   bool prof_ev_ready;
   bool debug_on;
+  int reuse_count;  // >= 0 while a step is being enqueued that derives its threshold from its scores; -1 otherwise
+  float last_tau;   // threshold of the last step when it was given by the caller
+  bool last_tau_on_device;
   int inject;       // diagnostics: what the next step's selection is overwritten with (0 = nothing); see dare.h
   // asynchronous host-buffer steps: copy streams and the events that order staging-buffer reuse (created on first use)
   bool host_async_ready;
@@ -78,6 +82,7 @@ inline void prof_end(dare_layer* L, cudaStream_t st) {
   if (L->prof_on) cudaEventRecord(L->prof_ev[L->prof_n], st);
 }
 void inject_selection_error(dare_layer* L, const StepGeom& g, cudaStream_t st);
+const float* step_threshold_on_device(dare_layer* L, const StepGeom& g, int mode, cudaStream_t st, int* launches);
 dare_status_t tc_create(dare_layer* L);
 void tc_destroy(dare_layer* L);
 // add_input: y = x + W_O O instead of y = W_O O (the residual connection of a transformer block)

@@ -155,7 +155,8 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   auto select_now = [&]() {
     prof_mark(L, SLOT_SELECT, st);
     // (a selection that refreshes everything reads no scores: behind the two projections it runs beside them)
-    launch_select(B.scores, tau, select_all, g, B.idx, B.count, B.batch_off, B.delta, st, kv_beside_q && select_all);
+    const float* tau_dev = step_threshold_on_device(L, g, mode, st, &launches);
+    launch_select(B.scores, tau, select_all, g, B.idx, B.count, B.batch_off, B.delta, st, kv_beside_q && select_all, tau_dev);
     ++launches;
     if (L->inject) inject_selection_error(L, g, st);
   };

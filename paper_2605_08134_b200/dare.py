@@ -66,6 +66,9 @@ def _load():
         "dare_layer_step_host": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
         "dare_layer_step_host_async": (C.c_int, [vp, vp, i32, i32, i32, i32, f32, vp, vp]),
         "dare_layer_wait_host": (C.c_int, [vp]),
+        "dare_layer_step_quantile": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, vp, vp]),
+        "dare_layer_last_threshold": (C.c_int, [vp, C.POINTER(C.c_float), vp]),
+        "dare_score_kth": (C.c_int, [vp, C.c_int64, C.c_int64, vp, vp]),
         "dare_layer_reset": (C.c_int, [vp]),
         "dare_layer_destroy": (C.c_int, [vp]),
         "dare_layer_status": (C.c_int, [vp, vp]),
@@ -160,6 +163,21 @@ def dare_layer_destroy(handle) -> int:
 
 def dare_layer_status(handle, stream=0) -> int:
     return _lib.dare_layer_status(handle, stream)
+
+
+def dare_layer_step_quantile(handle, x_ptr, batch, seq_act, pos_begin, mode, reuse_count, y_ptr, stream=0) -> int:
+    return _lib.dare_layer_step_quantile(handle, x_ptr, batch, seq_act, pos_begin, mode, reuse_count, y_ptr, stream)
+
+
+def dare_layer_last_threshold(handle, stream=0):
+    """-> (status, tau of the last step)."""
+    tau = C.c_float(0.0)
+    st = _lib.dare_layer_last_threshold(handle, C.byref(tau), stream)
+    return st, float(tau.value)
+
+
+def dare_score_kth(scores_ptr, n_tokens, k, tau_out_ptr, stream=0) -> int:
+    return _lib.dare_score_kth(scores_ptr, n_tokens, k, tau_out_ptr, stream)
 
 
 def dare_layer_clear_status(handle, stream=0) -> int:
@@ -338,6 +356,24 @@ class Layer:
         if st != OK:
             raise DareError(st, "dare_layer_step")
         return y
+
+    def step_quantile(self, x, mode, reuse_count, y=None, pos_begin=0):
+        """The step with the threshold taken from its own scores: the `reuse_count` least-drifted tokens are reused."""
+        torch = self.torch
+        assert x.is_cuda and x.dtype == self.tdtype and x.is_contiguous()
+        if y is None:
+            y = torch.empty_like(x)
+        st = dare_layer_step_quantile(self.handle, x.data_ptr(), x.shape[0], x.shape[1], pos_begin, mode, reuse_count,
+                                      y.data_ptr(), self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_step_quantile")
+        return y
+
+    def last_threshold(self) -> float:
+        st, tau = dare_layer_last_threshold(self.handle, self._stream())
+        if st != OK:
+            raise DareError(st, "dare_layer_last_threshold")
+        return tau
 
     def step_host(self, x_host, mode, threshold, y_host, pos_begin=0):
         st = dare_layer_step_host(self.handle, x_host.data_ptr(), x_host.shape[0], x_host.shape[1], pos_begin, mode,

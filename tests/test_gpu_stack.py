@@ -57,14 +57,18 @@ def oracle_stack(shape, w, batch):
                            lay.seq, lay.rope_theta, lay.rms_eps, w)
 
 
-@pytest.mark.parametrize("mode", [3, 1])
-def test_small_stack_decoding_trajectory(dare, mode):
+@pytest.mark.parametrize("mode,policy", [(3, "fixed"), (1, "fixed"), (3, "first-layers-dense-refresh-every-2nd-step")])
+def test_small_stack_decoding_trajectory(dare, mode, policy):
+    """policy "fixed": one threshold for every layer and step.  The other one is the schedule of the paper's Fast-dLLM-v2
+    experiment (Sec. 5) scaled to four layers: the first layers never reuse, and every second step refreshes
+    everything (refresh interval 2); both are per-layer thresholds below zero handed to the step by the caller."""
     import torch
     shape = small_stack()
     lay = shape.layer
     B, P, S = 2, lay.prompt, lay.seq
     w = wl.make_stack_weights(shape)
-    taus = [0.1] * shape.n_layers
+    base_taus = [0.1] * shape.n_layers
+    n_dense_layers = 2
     g = dare.Stack(shape, w, B)
     o = oracle_stack(shape, w, B)
     prompt = wl.random_prompt(shape, B)
@@ -73,10 +77,17 @@ def test_small_stack_decoding_trajectory(dare, mode):
     agree = 0
     steps = 0
     near = seen = 0
+    reused_rows = 0
     for blk in range(shape.gen_len // lay.block):
         lo, hi = P + blk * lay.block, P + (blk + 1) * lay.block
         for _ in range(lay.block):
             first = steps == 0
+            if policy == "fixed":
+                taus = base_taus
+            elif steps % 2 == 0:
+                taus = [-1.0] * shape.n_layers                                   # refresh step: nothing is reused
+            else:
+                taus = [-1.0] * n_dense_layers + base_taus[n_dense_layers:]      # the first layers never reuse
             pos_begin = 0 if first else P
             S_act = S - pos_begin
             before = toks_np.copy()
@@ -93,6 +104,10 @@ def test_small_stack_decoding_trajectory(dare, mode):
             for l in range(shape.n_layers):
                 ol = o.layers[l]
                 np.testing.assert_array_equal(gsel[l]["idx"], ol.last_idx, err_msg=f"step {steps} layer {l}")
+                if taus[l] < 0:
+                    assert gsel[l]["count"] == B * S_act                          # a layer told not to reuse refreshes all
+                else:
+                    reused_rows += B * S_act - gsel[l]["count"]
                 if not first:
                     np.testing.assert_allclose(gsel[l]["scores"], ol.last_scores, rtol=0, atol=SCORE_GATE_STACK)
                     near += int((np.abs(ol.last_scores - taus[l]) < MARGIN_STACK).sum())
@@ -125,6 +140,7 @@ def test_small_stack_decoding_trajectory(dare, mode):
     print(f"mode {mode}: {agree} of {steps * B} choices are the oracle's own arg-max")
     assert agree > 0
     assert near < 0.01 * seen, (near, seen)           # the margin decides for a small minority of the tokens only
+    assert reused_rows > 0                            # ... and the layers allowed to reuse did
     for l in range(shape.n_layers):
         assert g.layer(l).status() == 0
     g.close()

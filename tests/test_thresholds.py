@@ -48,3 +48,40 @@ def test_thresholds_give_the_planned_reuse_rate():
     tau, phi, _ = th.thresholds(smp, 0.4, 0.3)
     for x, t, p in zip(smp, tau, phi):
         assert abs(np.mean(x <= t) - p) < 2e-3
+
+
+# ----------------------------------------------------------------------------- per-step threshold (order statistic)
+def test_step_threshold_closed_forms():
+    inf = float("inf")
+    s = [0.5, 0.1, 0.3, 0.2, 0.4]
+    assert tor.step_threshold(s, 0) == -inf and tor.step_threshold(s, -3) == -inf
+    assert tor.step_threshold(s, 5) == inf and tor.step_threshold(s, 9) == inf
+    assert [tor.step_threshold(s, k) for k in (1, 2, 3, 4)] == [0.1, 0.2, 0.3, 0.4]
+    # ties: the threshold is the tied value, and Eq. 2 then reuses every token that has it
+    t = [0.3, 0.1, 0.3, 0.3, 0.7]
+    assert tor.step_threshold(t, 2) == 0.3 and sum(v <= 0.3 for v in t) == 4
+    # negative zero-ish scores (1 - cos rounds below zero) order below positive ones
+    assert tor.step_threshold([1e-7, -1e-7, 0.0, 0.5], 1) == -1e-7
+    # NaN scores are refreshed whatever the threshold: they are not counted among the reusable ones
+    u = [0.2, float("nan"), 0.1, float("nan"), 0.9]
+    assert tor.step_threshold(u, 2) == 0.2 and tor.step_threshold(u, 3) == 0.9 and tor.step_threshold(u, 4) == inf
+    assert tor.step_threshold([0.2, inf, 0.1], 2) == 0.2
+
+
+def test_step_threshold_reuses_exactly_the_least_drifted_tokens():
+    """Against numpy's partition, and the two counting properties that define an order statistic: fewer than k scores
+    lie strictly below tau, at least k lie at or below it; with distinct scores Eq. 2 then reuses exactly k tokens."""
+    rng = np.random.default_rng(4)
+    for n in (1, 2, 17, 1000):
+        s = rng.random(n) ** 4
+        for k in sorted({1, n // 3, n // 2, n - 1} - {0, n}):
+            tau = tor.step_threshold(s.tolist(), k)
+            assert tau == np.partition(s, k - 1)[k - 1]
+            assert (s < tau).sum() < k <= (s <= tau).sum()
+            assert (s <= tau).sum() == k
+    # reuse rate phi -> count floor(phi * n): the quantile form of Sec. 3.1 on one step's scores
+    s = np.linspace(0.0, 1.0, 101)
+    for phi in (0.0, 0.3, 0.5, 0.87, 1.0):
+        k = int(np.floor(phi * len(s) + 1e-9))
+        tau = tor.step_threshold(s.tolist(), k)
+        assert (s <= tau).sum() == min(k, len(s))
