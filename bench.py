@@ -732,6 +732,7 @@ def run_sweep(args):
     xa = torch.randn((B, S, d), generator=gen, device=dev).to(torch.bfloat16)
     y = torch.empty_like(xa)
     rng = np.random.default_rng(shape.seed)
+    all_curves = {}
 
     def changed_mask(frac, pattern):
         n = int(round(frac * S))
@@ -741,7 +742,7 @@ def run_sweep(args):
             m = wl.clustered_positions(rng, shape, step=4 * 9, clustered_per_seq=n, scattered_per_seq=0)
         return m
 
-    def time_mode(xb, m, steps=6):
+    def time_mode(xb, m, steps=args.sweep_steps):
         for lay in layers:
             lay.reset()
             lay.step(xa, m, TAU, y)
@@ -759,9 +760,10 @@ def run_sweep(args):
 
     fracs = [round(0.05 * i, 2) for i in range(21)]
     out = {"metric": "us_per_layer_step_vs_changed_fraction", "config": {"workload": shape.name, "batch": B, "seq_len": S,
-           "threshold": TAU, "layers_rotated": 2}, "points": [], "break_even": {}}
-    dense_us = time_mode(xa, 0)
-    out["dense_us"] = round(dense_us, 1)
+           "threshold": TAU, "layers_rotated": 2, "timed_steps_per_point": args.sweep_steps}, "points": [], "break_even": {}}
+    # the dense path before, between and after the two patterns (the clocks of these long steps move with the state of
+    # the power cap): its median is what the curves are compared with
+    dense_runs = [time_mode(xa, 0)]
     for pattern in ("uniform", "clustered"):
         curves = {"kv": [], "o": [], "both": []}
         for f in fracs:
@@ -778,7 +780,15 @@ def run_sweep(args):
                 row[name + "_us"] = round(us, 1)
                 curves[name].append(us)
             out["points"].append(row)
+        dense_runs.append(time_mode(xa, 0))
+        all_curves[pattern] = curves
+    dense_us = statistics.median(dense_runs)
+    out["dense_us"] = round(dense_us, 1)
+    out["dense_runs_us"] = [round(v, 1) for v in dense_runs]
+    worst = 0.0
+    for pattern, curves in all_curves.items():
         for name, ys in curves.items():
+            worst = max(worst, max(ys) / dense_us)
             be = None
             for i in range(len(fracs) - 1):
                 a, b_ = ys[i] - dense_us, ys[i + 1] - dense_us
@@ -788,6 +798,7 @@ def run_sweep(args):
             if be is None and ys[0] > dense_us:
                 be = 0.0
             out["break_even"][f"{pattern}/{name}"] = be
+    out["worst_ratio_to_dense"] = round(worst, 3)
     print(json.dumps(out))
 
 
@@ -810,6 +821,7 @@ def main():
     ap.add_argument("--gen", type=int, default=0, help="with --stack: stop after this many generated tokens (profiling)")
     ap.add_argument("--sweep", action="store_true", help="long-context crossover sweep (config 5) instead")
     ap.add_argument("--micro", action="store_true", help="time the stand-alone memory-bound kernels instead")
+    ap.add_argument("--sweep-steps", type=int, default=20, help="with --sweep: timed steps per point")
     args = ap.parse_args()
     # one process per GPU: under torchrun the world size must be the one asked for; started plainly with --gpus N > 1
     # this process becomes the launcher of N ranks (replicas, NCCL for the barrier and the max over ranks only)

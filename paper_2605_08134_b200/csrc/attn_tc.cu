@@ -137,6 +137,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   // Row tiles past the first one of a sequence are usually empty in the row-sparse case: they look at the refresh
   // set before spending anything on set-up.
+  // A launch issued in two forms (row-sparse over the refresh set, dense with its stores masked) runs in the one
+  // the size of the refresh set favours; the other leaves here, before it has set anything up.
+  if (p.gate_count != nullptr) {
+    pdl_wait();
+    const int c = __ldcg(p.gate_count);
+    if (c < p.gate_lo || c >= p.gate_hi) return;          // uniform over the launch
+  }
   if (p.idx != nullptr && tile > 0) {
     pdl_wait();
     if (__ldcg(p.batch_off + b) + tile * BQ >= __ldcg(p.batch_off + b + 1)) return;
@@ -177,6 +184,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   } else {
     row0 = b * g.seq_act + tile * BQ;
     rows_valid = min(BQ, g.seq_act - tile * BQ);
+    if (p.store_mask != nullptr) {
+      // dense form of a row-sparse step: a tile none of whose rows was refreshed has nothing to store
+      // (the gate above has waited for the selection)
+      const int r = (int)threadIdx.x;
+      const int mine = r < rows_valid && __ldcg(p.store_mask + g.cache_row(row0 + r)) == 0;
+      active = __syncthreads_or(mine) != 0;
+    }
   }
   const int n_blocks_all = (g.kv_len + BKV - 1) / BKV;
   const int n_blocks = n_blocks_all > z ? (n_blocks_all - z + ksplit - 1) / ksplit : 0;   // blocks z, z + ksplit, ...
@@ -435,7 +449,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // normalise, store
       const float inv = 1.f / l_row;
       const int t = r < rows_valid ? (p.idx ? __ldcg(p.idx + row0 + r) : row0 + r) : -1;
-      if (t >= 0 && (p.idx == nullptr || token_ok(t, g.tokens(), p.status))) {      // (else: no cache row to write)
+      if (t >= 0 && (p.idx == nullptr ? (p.store_mask == nullptr || __ldcg(p.store_mask + g.cache_row(t)) == 0)
+                                      : token_ok(t, g.tokens(), p.status))) {      // (else: no cache row to write)
         __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + st * 64;
 #pragma unroll
         for (int i = 0; i < 64; ++i) acc[i] *= inv;
@@ -510,6 +525,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const float inv = 1.f / lsum;
       const int t = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
       if (p.idx != nullptr && !token_ok(t, g.tokens(), p.status)) continue;        // no cache row to write
+      if (p.idx == nullptr && p.store_mask != nullptr && __ldcg(p.store_mask + g.cache_row(t)) != 0) continue;   // a reused row
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + 4 * lane;
       __nv_bfloat162 lo2 = __floats2bfloat162_rn(o.x * inv, o.y * inv), hi2 = __floats2bfloat162_rn(o.z * inv, o.w * inv);
       uint2 packed;
@@ -596,6 +612,11 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       b = rest / g.n_heads;
     }
   }
+  if (p.gate_count != nullptr) {
+    pdl_wait();
+    const int c = __ldcg(p.gate_count);
+    if (c < p.gate_lo || c >= p.gate_hi) return;          // uniform over the launch
+  }
   if (p.idx != nullptr && tile > 0) {
     pdl_wait();
     if (__ldcg(p.batch_off + b) + tile * kPairRows >= __ldcg(p.batch_off + b + 1)) return;
@@ -637,6 +658,11 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   } else {
     row0 = b * g.seq_act + tile * kPairRows;
     rows_all = min(kPairRows, g.seq_act - tile * kPairRows);
+    if (p.store_mask != nullptr) {
+      const int r = (int)threadIdx.x;
+      const int mine = r < rows_all && __ldcg(p.store_mask + g.cache_row(row0 + r)) == 0;
+      active = __syncthreads_or(mine) != 0;
+    }
   }
   const int n_blocks = (g.kv_len + BKV - 1) / BKV;
   const int n_half = (g.kv_len + kHalf - 1) / kHalf;   // half blocks: the unit of the score / softmax / P V pipeline
@@ -857,6 +883,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int rr = st * BQ + (ok ? r : 0);
       int t = p.idx ? __ldcg(p.idx + row0 + rr) : row0 + rr;
       if (p.idx != nullptr && ok && !token_ok(t, g.tokens(), p.status)) { ok = false; t = 0; }   // no cache row to write
+      if (p.idx == nullptr && p.store_mask != nullptr && ok && __ldcg(p.store_mask + g.cache_row(t)) != 0) ok = false;   // a reused row
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {

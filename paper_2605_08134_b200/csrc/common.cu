@@ -508,9 +508,11 @@ void launch_poke_int(int* dst, int value, cudaStream_t st) { poke_int_kernel<<<1
 // One warp per token row; rows refreshed in this step (staleness 0) are written by the projection itself.
 template <typename T>
 __global__ void __launch_bounds__(256) copy_reused_rows_kernel(const T* __restrict__ yc, T* __restrict__ y,
-                                                               const int* __restrict__ delta, StepGeom g) {
+                                                               const int* __restrict__ delta, StepGeom g,
+                                                               const int* __restrict__ gate_count, int gate_hi) {
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
+  if (gate_count != nullptr && *gate_count >= gate_hi) return;     // the dense form of the projection writes every row
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= g.tokens()) return;
   const int cr = g.cache_row(t);
@@ -522,13 +524,14 @@ __global__ void __launch_bounds__(256) copy_reused_rows_kernel(const T* __restri
 }
 
 template <typename T>
-void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st) {
+void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st,
+                             const int* gate_count, int gate_hi) {
   const int T_ = g.tokens();
   if (T_ <= 0) return;
-  launch_pdl(copy_reused_rows_kernel<T>, dim3((T_ + 7) / 8), dim3(256), 0, st, 1, yc, y, delta, g);
+  launch_pdl(copy_reused_rows_kernel<T>, dim3((T_ + 7) / 8), dim3(256), 0, st, 1, yc, y, delta, g, gate_count, gate_hi);
 }
 template void launch_copy_reused_rows<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, const int*, const StepGeom&,
-                                                     cudaStream_t);
+                                                     cudaStream_t, const int*, int);
 
 // ------------------------------------------------------------------------------------------------ row gather
 // dst[r, :] = src[idx[r], :] for r < *count (Alg. 1 line 6: x_norm restricted to the refresh set).
@@ -557,10 +560,11 @@ void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, 
 template <typename T>
 __global__ void __launch_bounds__(256) gather_step_rows_kernel(const T* __restrict__ src, const int* __restrict__ idx,
                                                                const int* __restrict__ count, T* __restrict__ dst,
-                                                               StepGeom g, int by_cache_row, int* status) {
+                                                               StepGeom g, int by_cache_row, int* status, int gate_hi) {
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   const int n = checked_count(*count, g.tokens(), status);
+  if (n >= gate_hi) return;                              // the launch that would read the copy leaves as well
   constexpr int N = 16 / sizeof(T);
   const int nvec = g.d / N;
   for (int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += gridDim.x * (blockDim.x >> 5)) {
@@ -574,15 +578,15 @@ __global__ void __launch_bounds__(256) gather_step_rows_kernel(const T* __restri
 }
 template <typename T>
 void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
-                             cudaStream_t st, int* status) {
+                             cudaStream_t st, int* status, int gate_hi) {
   const int T_ = g.tokens();
   if (T_ <= 0) return;
   const int grid = (T_ + 7) / 8 < 148 * 8 ? (T_ + 7) / 8 : 148 * 8;
   launch_pdl(gather_step_rows_kernel<T>, dim3(grid), dim3(256), 0, st, 1, src, idx, count, dst, g, by_cache_row ? 1 : 0,
-             status);
+             status, gate_hi);
 }
 template void launch_gather_step_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*,
-                                                     const StepGeom&, bool, cudaStream_t, int*);
+                                                     const StepGeom&, bool, cudaStream_t, int*, int);
 template void launch_gather_rows<float>(const float*, const int*, const int*, float*, int, int, cudaStream_t);
 template void launch_gather_rows<__nv_bfloat16>(const __nv_bfloat16*, const int*, const int*, __nv_bfloat16*, int, int,
                                                 cudaStream_t);

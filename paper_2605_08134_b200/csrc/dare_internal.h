@@ -114,7 +114,8 @@ void launch_rmsnorm(const T* x, const float* gain, T* xn, int rows, int d, float
 // y[t] = yc[cache_row(t)] for the tokens of the step that were not refreshed (staleness counter != 0 after the
 // selection of the step): the rows a gathered output projection leaves out.
 template <typename T>
-void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st);
+void launch_copy_reused_rows(const T* yc, T* y, const int* delta, const StepGeom& g, cudaStream_t st,
+                             const int* gate_count = nullptr, int gate_hi = 0);   // leaves at once when *gate_count >= gate_hi
 void launch_select(const float* scores, float tau, bool select_all, const StepGeom& g, int* idx, int* count,
                    int* batch_off, int* delta, cudaStream_t st, bool beside_predecessor = false,
                    const float* tau_dev = nullptr);   // tau_dev: read the threshold from device memory instead
@@ -125,7 +126,7 @@ void launch_gather_rows(const T* src, const int* idx, const int* count, T* dst, 
 // dst[r, :] = src[idx[r] (or its cache row), :] for the rows of a step's refresh set
 template <typename T>
 void launch_gather_step_rows(const T* src, const int* idx, const int* count, T* dst, const StepGeom& g, bool by_cache_row,
-                             cudaStream_t st, int* status = nullptr);
+                             cudaStream_t st, int* status = nullptr, int gate_hi = 1 << 30);  // leaves at once when *count >= gate_hi
 
 // diagnostics: a bounded wait that nothing ends (one CTA, one barrier); a single int written in stream order
 void launch_wait_probe(int* status, unsigned long long limit_ns, unsigned long long* waited_ns, cudaStream_t st);

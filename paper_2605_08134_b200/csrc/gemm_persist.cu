@@ -141,6 +141,11 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   // A listed launch whose size only the device knows is issued in both forms; each looks at the count and one of them
   // leaves at once: pairs pay when there are enough units to keep every cluster busy for two rounds or more.
   if (GATHER && p.unit_gate > 0 && (n_tiles * ((m_tiles_live + 1) / 2) >= p.unit_gate) != PAIR) total_tiles = 0;
+  // ... and in its listed and its dense form: the size of the refresh set decides which of the two runs
+  if (p.gate_count != nullptr) {
+    const int c = *p.gate_count;
+    if (c < p.gate_lo || c >= p.gate_hi) total_tiles = 0;
+  }
   auto tile_of = [&](int u) {
     if (!PAIR) return tile_geom(p, u, n_tiles, GATHER, n_rows);
     const int nt = u % n_tiles, mt = 2 * (u / n_tiles) + pr;
@@ -298,6 +303,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
               crowr = (size_t)p.g.cache_row(tokr);
             }
             tok_k[k] = tokr; crow_k[k] = crowr;
+            if (!GATHER && EPI == EPI_KV && p.store_mask != nullptr && ok[k] && p.store_mask[crowr] != 0) ok[k] = false;
             const uint8_t* row = stg + rr * STG_ROW_BYTES;
             const uint32_t off = (uint32_t)((((l16 >> 1) ^ (rr & 7)) << 4) | ((l16 & 1) << 3));
             lo[k] = *reinterpret_cast<const float2*>(row + off);

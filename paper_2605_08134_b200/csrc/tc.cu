@@ -116,6 +116,13 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
   base.debug = nullptr; base.wait_at_end = 0;
+  base.gate_count = nullptr; base.gate_lo = 0; base.gate_hi = 1 << 30; base.store_mask = nullptr;
+  // Steps of many row tiles: from these refresh-set sizes on the dense forms of the K/V projection, of attention and of
+  // the output projection (results kept for the refreshed rows only) are faster than the listed forms.  Measured on
+  // the long-context sweep (batch 4 x 4096): the listed K/V projection with its compact copy passes the dense form's
+  // time at about 78 % of the tokens, row-sparse attention + gathered output projection with its copy of the reused
+  // rows at about 80 %, all of them together at about 85 %.
+  const int gate_kv = (int)(0.75 * T_), gate_o = (int)(0.80 * T_);
   unsigned long long* dbg = L->debug_on ? B.debug : nullptr;
   // (no clearing between steps: a copy or memset in the stream would break the kernels' launch overlap; the stamps
   // are plain stores or maxima of a clock that only grows)
@@ -184,12 +191,23 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
         // Many tokens: even a small refreshed fraction fills the GPU with 256-wide tiles, which re-read the least.
         if (use_persist(n_tiles, m_tiles, 1) && compact_ok) {
           // a compact copy of the refresh set's rows first (a stream of n x d elements), then the projection with
-          // every operand through TMA and two-CTA MMAs
-          launch_gather_step_rows((const bf16*)B.xn, B.idx, B.count, (bf16*)B.x_stage, g, false, st, B.status); ++launches;
+          // every operand through TMA and two-CTA MMAs; beyond gate_kv refreshed tokens the dense form instead: every
+          // row of the step projected, the rows of the refresh set stored (the others keep their cached K and V)
+          const bool dense_form = use_persist(n_tiles, m_tiles_dense, 1);
+          const int hi = dense_form ? gate_kv : 1 << 30;
+          launch_gather_step_rows((const bf16*)B.xn, B.idx, B.count, (bf16*)B.x_stage, g, false, st, B.status, hi); ++launches;
           p.gather_src = nullptr;
           p.unit_gate = kPairUnitGate;
+          p.gate_count = B.count; p.gate_hi = hi;
           e = launch_gemm_persist(EPI_KV, S.a_xg, S.w_k128, S.w_v128, p, n_tiles, m_tiles, st, 1); ++launches;
           if (e == cudaSuccess) e = launch_gemm_persist(EPI_KV, S.a_xg, S.w_k, S.w_v, p, n_tiles, m_tiles, st, 0);
+          if (dense_form && e == cudaSuccess) {
+            GemmParams pd = p;
+            pd.idx = nullptr; pd.count = nullptr; pd.unit_gate = 0;
+            pd.gate_lo = gate_kv; pd.gate_hi = 1 << 30; pd.store_mask = B.delta;
+            ++launches;
+            e = launch_gemm_persist(EPI_KV, S.a_xn, S.w_k128, S.w_v128, pd, n_tiles, m_tiles_dense, st, 1);
+          }
         } else
           e = launch_gemm_tc(EPI_KV, 256, S.a_xn, S.w_k, S.w_v, p, n_tiles, m_tiles, 1, st);
         ++launches;
@@ -219,7 +237,18 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     // the refresh set then comes from the kernel right before; or the two kernels before ran beside the Q projection
     // without waiting for it, so the queries are not known to be complete before this kernel's own wait
     p.wait_first = kv_beside_q ? 1 : 0;
+    p.gate_count = nullptr; p.gate_lo = 0; p.gate_hi = 1 << 30; p.store_mask = nullptr;
+    // a long row-sparse step is issued in both forms: over the refresh set's rows, and dense with only the refreshed
+    // rows stored (tiles without one skipped); the size of the set decides on the device which of them runs
+    const bool both_forms = o_sparse && m_tiles_dense > 8 && use_persist(d / 256, m_tiles_dense, 1);
+    if (both_forms) { p.gate_count = B.count; p.gate_hi = gate_o; }
     e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
+    if (both_forms && e == cudaSuccess) {
+      AttnParams pd = p;
+      pd.idx = nullptr; pd.batch_off = nullptr; pd.debug = nullptr;
+      pd.gate_lo = gate_o; pd.gate_hi = 1 << 30; pd.store_mask = B.delta;
+      e = launch_attention_tc(S.kc64, S.vc64, pd, st); ++launches;
+    }
     if (e != cudaSuccess) return DARE_ERR_CUDA;
   }
   // Output projection, read from the O cache.  Alg. 2 line 11 projects every row of the window.  A row whose
@@ -240,17 +269,29 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     prof_mark(L, SLOT_OUT_GEMM, st);
     if (y_sparse) {
       p.idx = B.idx; p.count = B.count; p.gather_src = (const bf16*)B.oc; p.gather_cache_rows = 1;
+      bool dense_form = false;
       if (use_persist(n_tiles, (T_ + 127) / 128, 1) && compact_ok) {
-        launch_gather_step_rows((const bf16*)B.oc, B.idx, B.count, (bf16*)B.x_stage, g, true, st, B.status); ++launches;
+        // (beyond gate_o refreshed tokens the dense projection of every row instead: Alg. 2 line 11 as written)
+        dense_form = use_persist(n_tiles, m_tiles_dense, 1);
+        const int hi = dense_form ? gate_o : 1 << 30;
+        launch_gather_step_rows((const bf16*)B.oc, B.idx, B.count, (bf16*)B.x_stage, g, true, st, B.status, hi); ++launches;
         p.gather_src = nullptr;
         p.unit_gate = kPairUnitGate;
+        p.gate_count = B.count; p.gate_hi = hi;
         e = launch_gemm_persist(EPI_OUT, S.a_xg, S.w_o128, S.w_o128, p, n_tiles, (T_ + 127) / 128, st, 1); ++launches;
         if (e == cudaSuccess) e = launch_gemm_persist(EPI_OUT, S.a_xg, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, st, 0);
+        if (dense_form && e == cudaSuccess) {
+          GemmParams pd = p;
+          pd.idx = nullptr; pd.count = nullptr; pd.unit_gate = 0; pd.gather_cache_rows = 0;
+          pd.gate_lo = gate_o; pd.gate_hi = 1 << 30;
+          ++launches;
+          e = launch_gemm_persist(EPI_OUT, S.a_oc, S.w_o128, S.w_o128, pd, n_tiles, m_tiles_dense, st, 1);
+        }
       } else
         e = launch_gemm_tc(EPI_OUT, 256, S.a_oc, S.w_o, S.w_o, p, n_tiles, (T_ + 127) / 128, 1, st);
       ++launches;
       if (e != cudaSuccess) return DARE_ERR_CUDA;
-      launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st); ++launches;
+      launch_copy_reused_rows((const bf16*)B.yc, (bf16*)y, B.delta, g, st, dense_form ? B.count : nullptr, gate_o); ++launches;
     } else {
       const int sp = pick_splits(n_tiles * m_tiles_dense, kblocks);
       if (narrow_pairs_pay(d, m_tiles_dense, kblocks))

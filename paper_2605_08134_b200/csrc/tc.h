@@ -44,6 +44,16 @@ struct GemmParams {
   int has_prev;
   int* status;
   unsigned long long* debug;   // 8 timestamp slots of this kernel or nullptr
+  // A step whose refresh set is large runs its projections and attention in their dense forms (every operand through
+  // TMA straight from the step's buffers, no compact copy, two-CTA MMAs) and only keeps the results of the rows that
+  // were refreshed; only the device knows the set's size, so both forms of a launch are issued and each looks at the
+  // count: a launch runs when gate_lo <= *gate_count < gate_hi and leaves at once otherwise (gate_count == nullptr:
+  // always runs).  store_mask (the staleness counters, by cache row): a dense-form K/V projection stores a row only
+  // where the counter is 0, i.e. where this step's selection refreshed the token (Eq. 3: every other row keeps its
+  // cached K and V).
+  const int* gate_count;
+  int gate_lo, gate_hi;
+  const int* store_mask;
   int wait_at_end;       // 1: the launch reads nothing its predecessor in the stream writes and writes nothing that one
                          // reads, so it runs beside it: its CTAs start as soon as the predecessor's have passed their own
                          // dependency wait (everything further back is then complete), and wait for the predecessor
@@ -58,6 +68,11 @@ struct AttnParams {
   StepGeom g;
   int* status;
   unsigned long long* debug;
+  const int* gate_count;    // as in GemmParams: the launch runs when gate_lo <= *gate_count < gate_hi
+  int gate_lo, gate_hi;
+  const int* store_mask;    // dense form of a row-sparse step: a row's output is stored only where the staleness counter
+                            // (by cache row) is 0 (Eq. 4: every other row keeps its cached output); tiles without such
+                            // a row are skipped
   int wait_first;           // 1: the queries or the refresh set come from the kernel just before this one in the stream,
                             // so nothing of the step is read ahead of the dependency wait
 };

@@ -159,6 +159,38 @@ def test_config5_index_sets_over_the_whole_sweep(dare, config5, pattern):
     assert g.status() == 0
 
 
+@pytest.mark.parametrize("pattern", ["uniform", "clustered"])
+def test_listed_and_dense_forms_on_both_sides_of_their_gates(dare, pattern):
+    """A step of many row tiles issues its K/V projection, its attention and its output projection in two forms, listed
+    (over the refresh set) and dense (over every row, results kept for the refreshed rows only), and the size of the
+    refresh set decides on the device which runs: from 75 % of the tokens on for the K/V projection, from 80 % for the
+    other two.  Width 2048, 2 x 2560 tokens (40 row tiles: every projection in the persistent kernel); consecutive steps
+    at 30, 78, 90, 100, 77 and 85 % changed in rotating modes, checked against the oracle in full: the forms must give
+    the same caches and outputs, and reused rows must stay untouched, whichever side of a gate a step falls on."""
+    shape = wl.scaled(wl.LLADA_LAYER, d_model=2048, n_heads=16, batch=2, seq=2560, prompt=1280)
+    w = wl.make_weights(shape, 71)
+    hs = wl.HiddenStream(shape, 71)
+    g = dare.Layer(shape, w, kernel_path=dare.PATH_TENSOR)
+    o = parity.oracle_layer(shape, w)
+    parity.compare_step(g, o, hs.first(), 3, 0.1, shape, first=True)
+    for i, frac in enumerate((0.30, 0.78, 0.90, 1.00, 0.77, 0.85)):
+        n = int(round(frac * shape.seq))
+        ch = (wl.uniform_positions(hs.rng, shape, n) if pattern == "uniform"
+              else wl.clustered_positions(hs.rng, shape, 4 * i, n, 0))
+        before = g.read_caches(shape.batch, shape.seq)
+        mode = (3, 3, 3, 3, 1, 2)[i]
+        parity.compare_step(g, o, hs.advance(ch), mode, 0.1, shape)
+        after = g.read_caches(shape.batch, shape.seq)
+        keep = ~ch
+        if mode & 1:
+            assert np.array_equal(after["k"][keep], before["k"][keep]) and np.array_equal(after["v"][keep], before["v"][keep])
+        if mode & 2:
+            assert np.array_equal(after["o"][keep], before["o"][keep])
+        assert g.last_selection(shape.batch, shape.seq)["count"] == n * shape.batch
+    assert g.status() == 0
+    g.close()
+
+
 def test_long_context_attention_repeats_bit_identically(dare):
     """Batch 4 x 4096, two steps (dense, then K/V reuse at 50 % clustered) on three fresh handles: the caches must be
     bit-identical from run to run.  The softmax warps of the two-tile attention kernel run up to two P V products
