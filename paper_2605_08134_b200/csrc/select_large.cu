@@ -159,7 +159,11 @@ __global__ void __launch_bounds__(kThreads) tile_scan_kernel(const int* __restri
 
 // pass 3: from the decision bits alone (4 bytes per thread instead of 128 bytes of scores).  One thread per word of
 // 32 consecutive scores, 512 threads per tile: one scan of the words' popcounts places every thread, which then
-// writes the indices of its set bits, ascending, at consecutive places.
+// writes the indices of its set bits, ascending, at consecutive places.  Every lane of such a store lands in another
+// sector (ncu: 10.7 sectors per request), yet the pass is bound by the chain load -> scan -> stores of its CTAs
+// rather than by the stores: two other forms measured slower on the same 2^24 scores (22.7 us per call for this one):
+// lane-consecutive stores, each list entry found by a binary search over the words' first places in shared memory
+// (27.5 us), and 256-thread CTAs with two words per thread so that every tile is resident at once (25.5 us).
 // No store goes past entry n - 1 of the list, whatever the offsets say: if another call raced on a shared scratch
 // array, the list is wrong but the caller's buffer is the only memory written.
 __global__ void __launch_bounds__(kTileWords) tile_scatter_kernel(const unsigned* __restrict__ flags,
@@ -169,7 +173,7 @@ __global__ void __launch_bounds__(kTileWords) tile_scatter_kernel(const unsigned
   __shared__ int total;
   ptx::pdl_wait();                         // before any read: decisions (two kernels back) and offsets (one back)
   unsigned word = flags[(size_t)blockIdx.x * kTileWords + threadIdx.x];
-  int out = tile_offsets[blockIdx.x];
+  long long out = tile_offsets[blockIdx.x];
   out += block_exclusive_scan<int>(__popc(word), warp_sums, &total);
   const int i0 = (int)((long long)blockIdx.x * kTile) + (int)threadIdx.x * 32;
   while (word != 0u) {
