@@ -589,6 +589,29 @@ def run_micro(args):
     out["kernels"].append({"kernel": "drift_scores", "rows": rows, "head_dim": hd, "us": round(t * 1e6, 1),
                            "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3)})
     del a, b
+    # RMSNorm over the rows of the long-context step (batch 4 x 4096 rows of 4096 bf16: 134 MB in, 134 MB out), four
+    # input/output pairs in rotation
+    rows_n, dm = 16384, 4096
+    xs = [torch.randn((rows_n, dm), device=dev).to(torch.bfloat16) for _ in range(4)]
+    ys = [torch.empty_like(xs[0]) for _ in range(4)]
+    gain = torch.ones(dm, device=dev)
+    turn_n = [0]
+
+    def norm():
+        i = turn_n[0] & 3
+        turn_n[0] += 1
+        dare.dare_rmsnorm(xs[i].data_ptr(), gain.data_ptr(), ys[i].data_ptr(), rows_n, dm, 1e-5, dare.BF16, st)
+
+    t = time_it(norm)
+    algo = 2.0 * rows_n * dm * 2
+    out["kernels"].append({"kernel": "rmsnorm", "rows": rows_n, "d_model": dm, "us": round(t * 1e6, 1),
+                           "achieved": round(algo / t / 1e9, 1), "frac": round(algo / t / 1e9 / peaks["hbm_gbs"], 3)})
+    ref = xs[0].float()
+    ref = (ref * torch.rsqrt((ref * ref).mean(dim=1, keepdim=True) + 1e-5)).to(torch.bfloat16)
+    dare.dare_rmsnorm(xs[0].data_ptr(), gain.data_ptr(), ys[0].data_ptr(), rows_n, dm, 1e-5, dare.BF16, st)
+    torch.cuda.synchronize()
+    assert float((ys[0].float() - ref.float()).abs().max()) <= 0.04, "rmsnorm micro-benchmark: wrong result"
+    del xs, ys, ref
     n = 1 << 24
     # four score arrays in rotation (256 MB, twice the L2): every call reads its scores from HBM
     bufs = []

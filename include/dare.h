@@ -243,6 +243,10 @@ dare_status_t dare_layer_debug_timestamps(dare_layer_t* layer, int enable, uint6
  * offsets, and one decision bit per score: about n_tokens / 8 bytes); n_tokens <= 2^30; NaN threshold is rejected. */
 dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t rows, int head_dim, float* scores,
                                 void* cuda_stream);
+/* Alg. 1/2 line 1 alone: y[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * gain, for `rows` rows of `d_model` elements
+ * (a multiple of 16) of the given dare_dtype_t; gain is float32 [d_model]; rows <= 2^24.  The kernel of the layer step. */
+dare_status_t dare_rmsnorm(const void* x, const float* gain, void* y, int64_t rows, int d_model, float eps, int dtype,
+                           void* cuda_stream);
 /* *tau_out (device) = the k-th smallest of n_tokens float32 scores (k clamped to [0, n_tokens]; k = 0: -inf,
  * k = n_tokens or beyond the scores that are numbers: +inf), the threshold that reuses the k least-drifted tokens under
  * Eq. 2 (Sec. 3.1).  One CTA, exact; 1 <= n_tokens <= 2^24. */

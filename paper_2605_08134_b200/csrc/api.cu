@@ -664,6 +664,21 @@ dare_status_t dare_drift_scores(const float* q_now, const float* q_prev, int64_t
   return DARE_OK;
 }
 
+dare_status_t dare_rmsnorm(const void* x, const float* gain, void* y, int64_t rows, int d_model, float eps, int dtype,
+                           void* cuda_stream) {
+  if (!x || !gain || !y) return DARE_ERR_INVALID_ARG;
+  if (dtype != DARE_F32 && dtype != DARE_BF16) return DARE_ERR_INVALID_ARG;
+  if (rows < 0 || rows > (int64_t)1 << 24 || d_model <= 0 || d_model % 16 != 0 || !(eps >= 0.f)) return DARE_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(gain)) return DARE_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (dtype == DARE_BF16)
+    launch_rmsnorm<__nv_bfloat16>((const __nv_bfloat16*)x, gain, (__nv_bfloat16*)y, (int)rows, d_model, eps, st);
+  else
+    launch_rmsnorm<float>((const float*)x, gain, (float*)y, (int)rows, d_model, eps, st);
+  CUDA_TRY(cudaGetLastError());
+  return DARE_OK;
+}
+
 size_t dare_select_compact_scratch_bytes(int64_t n_tokens) {
   if (n_tokens < 0 || n_tokens > (int64_t)1 << 30) return 0;
   return align_up((size_t)select_large_tiles(n_tokens) * sizeof(int)) * 2 + align_up(select_large_flag_bytes(n_tokens)) +

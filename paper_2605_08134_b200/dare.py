@@ -69,6 +69,7 @@ def _load():
         "dare_layer_step_quantile": (C.c_int, [vp, vp, i32, i32, i32, i32, i32, vp, vp]),
         "dare_layer_last_threshold": (C.c_int, [vp, C.POINTER(C.c_float), vp]),
         "dare_score_kth": (C.c_int, [vp, C.c_int64, C.c_int64, vp, vp]),
+        "dare_rmsnorm": (C.c_int, [vp, vp, vp, C.c_int64, i32, f32, i32, vp]),
         "dare_layer_reset": (C.c_int, [vp]),
         "dare_layer_destroy": (C.c_int, [vp]),
         "dare_layer_status": (C.c_int, [vp, vp]),
@@ -174,6 +175,10 @@ def dare_layer_last_threshold(handle, stream=0):
     tau = C.c_float(0.0)
     st = _lib.dare_layer_last_threshold(handle, C.byref(tau), stream)
     return st, float(tau.value)
+
+
+def dare_rmsnorm(x_ptr, gain_ptr, y_ptr, rows, d_model, eps, dtype, stream=0) -> int:
+    return _lib.dare_rmsnorm(x_ptr, gain_ptr, y_ptr, rows, d_model, eps, dtype, stream)
 
 
 def dare_score_kth(scores_ptr, n_tokens, k, tau_out_ptr, stream=0) -> int:
