@@ -95,7 +95,7 @@ __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParam
     }
     // no instruction consumes these loads before the finishing pass, so they stay in flight across the exchange
     if (rotate) rb.cs[k] = *reinterpret_cast<const float4*>(p.rope + (size_t)pos * (HD / 2) + 2 * lane);
-    if ((EPI == EPI_Q || EPI == EPI_QKV) && score_tile && p.has_prev) {
+    if (EPI == EPI_Q && score_tile && p.has_prev) {
       rb.qa[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + 2 * lane);
       rb.qb[k] = *reinterpret_cast<const float2*>(p.q_prev + rb.crow[k] * HD + HD / 2 + 2 * lane);
     }
@@ -113,7 +113,7 @@ __device__ __forceinline__ void load_row_batch(RowBatch<RB>& rb, const GemmParam
 template <int EPI, int BN, bool PAIR>
 __global__ void __launch_bounds__(Warps<BN>::N * 32, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
-               const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_b2, const GemmParams p) {
+               const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
   using C = Cfg<BN, PAIR>;
   constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
   constexpr int kWarps = Warps<BN>::N, RB = Warps<BN>::RB;
@@ -145,12 +145,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
   // ---- which columns?  Tiles [0, n_split) belong to W0/out0, the rest to W1/out1.
-  // (EPI_QKV: three matrices, n_split tiles each: Q, K, V)
-  const int mat = p.b_pair ? 0 : (EPI == EPI_QKV ? nt / p.n_split : (nt >= p.n_split ? 1 : 0));
-  const bool is_b1 = mat == 1;
-  const int n0 = p.b_pair ? nt * (BN / 2) : (nt - mat * (mat ? p.n_split : 0)) * BN;   // first output column / W row
-  const CUtensorMap* tm_b = mat == 0 ? &tm_b0 : (mat == 1 ? &tm_b1 : &tm_b2);
-  constexpr bool kScores = EPI == EPI_Q || EPI == EPI_QKV;
+  const bool is_b1 = !p.b_pair && nt >= p.n_split;
+  const int n0 = p.b_pair ? nt * (BN / 2) : (is_b1 ? nt - p.n_split : nt) * BN;   // first output column / W row
+  const CUtensorMap* tm_b = is_b1 ? &tm_b1 : &tm_b0;
   // ---- which slice of the reduction?
   const int KB = p.K / BK;
   const int kb_begin = (int)(((long long)KB * z) / splits), kb_end = (int)(((long long)KB * (z + 1)) / splits);
@@ -247,9 +244,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // epilogue geometry
   const int rows_per_cta = BM / splits;           // rows of the tile this CTA finishes
   const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
-  const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1) || (EPI == EPI_QKV && mat < 2);
+  const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
-  const bool score_tile = kScores && mat == 0 && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
+  const bool score_tile = (EPI == EPI_Q) && p.g.score_head >= head0 && p.g.score_head < head0 + BN / HD;
   RowBatch<RB> rb;
 
   if (active) {
@@ -433,10 +430,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // ---- finish the owned rows: one warp per row, lane <-> pairs (2*lane, 2*lane+1) of each head of the tile.
   // Rows are taken four at a time so that their table reads are in flight together.
   {
-    __nv_bfloat16* out = mat == 0 ? p.out0 : (mat == 1 ? p.out1 : p.out2);
-    // rows of the output: by cache row, by token, or by place in the list (a fused Q/K/V launch: Q by token, K and V
-    // by cache row)
-    const int out_rows = EPI == EPI_QKV ? (mat == 0 ? 0 : 1) : p.out_is_cache;
+    __nv_bfloat16* out = is_b1 ? p.out1 : p.out0;
 #pragma unroll 1
     for (int rl0 = warp; rl0 < rows_per_cta; rl0 += kWarps * RB) {
       if (rl0 != warp) load_row_batch<EPI, RB, kWarps, BN>(rb, p, rl0, z, rows_per_cta, rows_valid, t0, pos0, crow0, rotate, score_tile, lane, n0);
@@ -465,7 +459,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       // (2) Sec. 3.1 on the un-rotated query of the scoring head: 1 - cos(current, stored), all rows of the batch
       //     reduced across the lanes together; lane k finishes row k.  Then the current query is stored.
-      if (kScores && score_tile) {
+      if (EPI == EPI_Q && score_tile) {
         float dot[RB], n1[RB], n2[RB];
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
@@ -510,7 +504,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
       for (int k = 0; k < RB; ++k) {
         if (!rb.ok[k]) continue;
-        const size_t orow = out_rows == 1 ? rb.crow[k] : (out_rows == 2 ? (size_t)rb.row[k] : (size_t)rb.tok[k]);
+        const size_t orow = p.out_is_cache == 1 ? rb.crow[k] : (p.out_is_cache == 2 ? (size_t)rb.row[k] : (size_t)rb.tok[k]);
         if (EPI == EPI_SWIGLU) {
           // columns [0, 128) of a 256-wide tile are the gate, [128, 256) the up projection of the same 128 outputs
           const float2 g_lo = vlo[k][0], g_hi = vhi[k][0], u_lo = vlo[k][BN / HD - 1], u_hi = vhi[k][BN / HD - 1];
@@ -585,8 +579,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
 template <int EPI, int BN, bool PAIR>
 static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const GemmParams& p,
-                              int n_tiles, int m_tiles, int splits, cudaStream_t st, const CUtensorMap* b2p = nullptr) {
-  const CUtensorMap& b2 = b2p ? *b2p : b1;
+                              int n_tiles, int m_tiles, int splits, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
   auto kern = gemm_tc_kernel<EPI, BN, PAIR>;
   constexpr int SMEM_TOTAL = Cfg<BN, PAIR>::SMEM_TOTAL;
@@ -595,22 +588,16 @@ static cudaError_t launch_one(const CUtensorMap& a, const CUtensorMap& b0, const
   q.m_tiles = m_tiles;
   if (PAIR)
     return launch_pdl_xz(kern, dim3((m_tiles + 1) / 2 * 2, n_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, 2,
-                         splits, a, b0, b1, b2, q);
+                         splits, a, b0, b1, q);
   return launch_pdl_xz(kern, dim3(n_tiles, m_tiles, splits), dim3(Warps<BN>::N * 32), SMEM_TOTAL, st, 1, splits, a, b0, b1,
-                       b2, q);
+                       q);
 }
 
 // pair != 0: the launch uses two-CTA MMAs (256-wide tiles, A through the tensor map); b0 / b1 must then be maps with
 // 128-row boxes.
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair,
-                           const CUtensorMap* b2) {
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair) {
   if (m_tiles <= 0 || n_tiles <= 0) return cudaSuccess;
-  if (epi == EPI_QKV) {
-    if (bn != 256 || b2 == nullptr || p.gather_src != nullptr || p.count != nullptr || p.b_pair) return cudaErrorInvalidValue;
-    if (pair) return launch_one<EPI_QKV, 256, true>(a, b0, b1, p, n_tiles, m_tiles, splits, st, b2);
-    return launch_one<EPI_QKV, 256, false>(a, b0, b1, p, n_tiles, m_tiles, splits, st, b2);
-  }
   if (epi == EPI_OUT && p.resid != nullptr) epi = EPI_OUT_RES;
   if ((splits != 1 && splits != 2) || splits > p.K / BK) return cudaErrorInvalidValue;
   if (pair && bn == 128) {

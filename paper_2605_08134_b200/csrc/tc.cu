@@ -1,6 +1,5 @@
 // Host side of the tensor-core path: TMA tensor maps and the per-step kernel sequence.
 #include <new>
-#include <stdlib.h>
 
 #include "layer.h"
 #include "tc.h"
@@ -112,7 +111,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.K = d; base.m_total = T_; base.seq_act = g.seq_act; base.tiles_per_seq = tiles_per_seq;
   base.a_seq_stride = g.seq_act; base.a_row0 = 0; base.idx = nullptr; base.count = nullptr; base.g = g;
   base.gather_src = nullptr; base.gather_cache_rows = 0; base.unit_gate = 0;
-  base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.out2 = nullptr; base.ld_out = d;
+  base.n_split = 1 << 30; base.out0 = nullptr; base.out1 = nullptr; base.ld_out = d;
   base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
@@ -133,18 +132,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   prof_mark(L, SLOT_NORM, st);
   launch_rmsnorm<bf16>((const bf16*)x, L->w.rms_gain, (bf16*)B.xn, T_, d, L->cfg.rms_eps, st, dbg ? dbg + 40 : nullptr);
   ++launches;
-  static const int x_fused = getenv("DARE_FUSED") ? atoi(getenv("DARE_FUSED")) : 0;   // TEMP
-  const bool fused_qkv = x_fused != 0 && !kv_sparse && m_tiles_dense <= 8 && m_tiles_dense >= 2;   // TEMP
   // line 2 + line 3 + stored-query update + rotary embedding, one kernel
-  if (fused_qkv) {   // TEMP
-    GemmParams p = base;
-    p.out0 = (bf16*)B.q; p.out1 = (bf16*)B.kc; p.out2 = (bf16*)B.vc; p.n_split = d / 256;
-    p.debug = dbg;
-    prof_mark(L, SLOT_Q_GEMM, st);
-    e = launch_gemm_tc(EPI_QKV, 256, S.a_xn, S.w_q128, S.w_k128, p, 3 * (d / 256), m_tiles_dense, x_fused == 2 ? 2 : 1, st, 1, &S.w_v128);
-    ++launches;
-    if (e != cudaSuccess) return DARE_ERR_CUDA;
-  } else
   {
     GemmParams p = base;
     p.out0 = (bf16*)B.q;
@@ -181,7 +169,6 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   };
   if (!kv_beside_q) select_now();
   // K/V projection with rotary embedding and cache scatter
-  if (!fused_qkv)   // TEMP
   {
     GemmParams p = base;
     p.n_split = d / 256;

@@ -8,8 +8,7 @@
 namespace dare {
 
 enum { EPI_Q = 0, EPI_KV = 1, EPI_OUT = 2, EPI_SWIGLU = 3, EPI_F32 = 4,
-       EPI_OUT_RES = 5,     // EPI_OUT plus a residual row (chosen by the launcher when GemmParams::resid is set)
-       EPI_QKV = 6 };       // Q, K and V of every row in one grid: n_split column tiles per matrix, W maps b0, b1, b2
+       EPI_OUT_RES = 5 };   // EPI_OUT plus a residual row (chosen by the launcher when GemmParams::resid is set)
 
 struct GemmParams {
   int K;                 // reduction length (multiple of 64)
@@ -31,7 +30,6 @@ struct GemmParams {
   int n_split;           // n-tiles [0, n_split) use W0/out0, the rest W1/out1
   __nv_bfloat16* out0;
   __nv_bfloat16* out1;
-  __nv_bfloat16* out2;   // EPI_QKV: the V cache (out0 = Q by token, out1 = K cache)
   int ld_out;
   int out_is_cache;      // output rows addressed by cache row (1), by flat token index (0), or by the row's place
                          // in the gathered list (2)
@@ -105,8 +103,7 @@ inline bool narrow_pairs_pay(int d_out, int m_tiles, int kblocks) {
 }
 
 cudaError_t launch_gemm_tc(int epi, int bn, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
-                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair = 0,
-                           const CUtensorMap* b2 = nullptr);
+                           const GemmParams& p, int n_tiles, int m_tiles, int splits, cudaStream_t st, int pair = 0);
 
 
 // Persistent form for launches of many row tiles (dense rows, 256-wide tiles, no reduction split, epilogues Q, K/V,
