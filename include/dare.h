@@ -263,7 +263,8 @@ dare_status_t dare_select_compact(const float* scores, int64_t n_tokens, float t
  *   - n_tokens <= dare_select_compact_static_max_tokens() (= 16,777,216); more returns DARE_ERR_SHAPE.
  *   - The call allocates nothing and frees nothing, on the device or through any library.
  *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress with that device
- *     current): make that first call outside any stream capture.
+ *     current): make that first call outside any stream capture.  The address is kept for the life of the process; a
+ *     cudaDeviceReset of that device would leave it stale (do not reset a device this entry point has been used on).
  *   - All calls on a device share the array; it keeps the previous call's contents (nothing needs clearing: a call
  *     writes every entry before reading it).  Calls that overlap on the GPU, e.g. on two streams, race on it: their
  *     lists and counts are then undefined (entries may be missing, repeated or another call's), though no call ever
