@@ -104,3 +104,32 @@ def test_select_compact_alternating_thresholds_on_one_scratch(dare, n):
             assert k == len(want[tau]), (rep, tau)
             assert np.array_equal(idx[:k].cpu().numpy(), want[tau]), (rep, tau)
             assert bool((idx[k:] == -1).all())
+
+
+@pytest.mark.parametrize("rows,d,dtype", [(7, 256, "f32"), (300, 1024, "bf16"), (2049, 4096, "bf16"), (4100, 512, "bf16"),
+                                          (5000, 768, "f32")])
+def test_standalone_rmsnorm_matches_the_oracle(dare, rows, d, dtype):
+    """Alg. 1/2 line 1 through its own entry point, on both of its kernels (one row per CTA; two rows per CTA beyond 2048
+    bf16 rows), with a gain that is not all ones."""
+    import torch
+    from oracle import dare_oracle as orc
+    from paper_2605_08134_b200 import workloads as wl
+    rng = np.random.default_rng(rows + d)
+    bf = dtype == "bf16"
+    x = wl.round_to(rng.standard_normal((rows, d), dtype=np.float32) * 1.7, wl.DTYPE_BF16 if bf else wl.DTYPE_F32)
+    gain = (1.0 + 0.2 * rng.standard_normal(d)).astype(np.float32)
+    tdt = torch.bfloat16 if bf else torch.float32
+    xd = torch.from_numpy(x).cuda().to(tdt)
+    gd = torch.from_numpy(gain).cuda()
+    yd = torch.empty_like(xd)
+    st = dare.dare_rmsnorm(xd.data_ptr(), gd.data_ptr(), yd.data_ptr(), rows, d, 1e-5, dare.BF16 if bf else dare.F32,
+                           torch.cuda.current_stream().cuda_stream)
+    assert st == 0
+    torch.cuda.synchronize()
+    want = orc.rmsnorm(x, gain, 1e-5)
+    got = yd.float().cpu().numpy().astype(np.float64)
+    # bf16: one rounding of the result (relative 2^-9); fp32: fp32 arithmetic on O(1) values
+    tol = 2.0 ** -8 if bf else 2e-6
+    assert np.max(np.abs(got - want) / (np.abs(want) + 1.0)) <= tol
+    assert dare.dare_rmsnorm(0, gd.data_ptr(), yd.data_ptr(), rows, d, 1e-5, dare.F32, 0) == dare.ERR_INVALID_ARG
+    assert dare.dare_rmsnorm(xd.data_ptr(), gd.data_ptr(), yd.data_ptr(), rows, d + 1, 1e-5, dare.F32, 0) == dare.ERR_SHAPE
