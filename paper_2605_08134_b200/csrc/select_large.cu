@@ -7,6 +7,14 @@
 //     (3) per-tile compaction from the decision bits, written at the tile's offset: ascending index list
 // No CTA waits for another; the order of the list does not depend on scheduling.  Passes 2 and 3 are launched
 // programmatically dependent: their launch latency hides behind the pass before.
+// A single pass (tiles handed out by ticket, every CTA publishing its tile's count and adding up the counts published
+// before it back to the nearest known running total, entries staged in shared memory and written as whole lines) was
+// built as well, list and count identical, and measured on the same 2^24 scores against 22.6 us for the three passes:
+// 27.7-32.3 us with one tile per CTA (16384 down to 4096 scores per tile, walk by one warp), 33-40 us with the walk by
+// the whole CTA, 40-65 us with resident CTAs that have the next two tiles copied into shared memory (bulk copies on
+// an mbarrier) while they work.  All CTAs of a wave reach the walk at the same time, so the nearest known total is a
+// whole wave back, and a CTA's loads do not overlap its walk: the chain per tile (scores -> scan -> publish -> walk
+// -> write) is several microseconds long, and what a CTA has in flight during it does not cover it.
 #include <math.h>
 #include <mutex>
 
