@@ -595,12 +595,26 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const StepGeom& g = p.g;
+  // Which form runs?  A launch that carries both (dense_from > 0) decides here, from the size of the refresh set:
+  // below dense_from the rows of the refresh set, from there on every row with only the refreshed ones stored.
+  const int* idx = p.idx;
+  const int* batch_off = p.batch_off;
+  const int* store_mask = p.store_mask;
+  if (p.gate_count != nullptr) {
+    pdl_wait();
+    const int c = __ldcg(p.gate_count);
+    if (p.dense_from > 0) {
+      if (c >= p.dense_from) { idx = nullptr; batch_off = nullptr; store_mask = p.dense_mask; }
+    } else if (c < p.gate_lo || c >= p.gate_hi) {
+      return;                                             // uniform over the launch
+    }
+  }
   // CTA -> (head, sequence, 256-row tile): same launch orders as the kernel above
   const int tps = (g.seq_act + kPairRows - 1) / kPairRows;
   int h, b, tile;
   {
     const int lin = blockIdx.y * gridDim.x + blockIdx.x;
-    if (p.idx != nullptr) {
+    if (idx != nullptr) {
       h = lin % g.n_heads;
       const int rest = lin / g.n_heads;
       tile = rest / g.batch;
@@ -612,14 +626,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       b = rest / g.n_heads;
     }
   }
-  if (p.gate_count != nullptr) {
+  if (idx != nullptr && tile > 0) {
     pdl_wait();
-    const int c = __ldcg(p.gate_count);
-    if (c < p.gate_lo || c >= p.gate_hi) return;          // uniform over the launch
-  }
-  if (p.idx != nullptr && tile > 0) {
-    pdl_wait();
-    if (__ldcg(p.batch_off + b) + tile * kPairRows >= __ldcg(p.batch_off + b + 1)) return;
+    if (__ldcg(batch_off + b) + tile * kPairRows >= __ldcg(batch_off + b + 1)) return;
   }
   // diagnostics: [0] first CTA's start, [1] its set-up done, [3] its key loop done, [4] its end; over the CTAs with
   // work: [5] latest start, [6] latest end, [7] their number
@@ -650,17 +659,17 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   // ---- rows of the two tiles (uniform over the CTA)
   int row0 = 0, rows_all = 0;
   bool active = true;
-  if (p.idx != nullptr) {
-    const int lo = __ldcg(p.batch_off + b), hi = __ldcg(p.batch_off + b + 1);
+  if (idx != nullptr) {
+    const int lo = __ldcg(batch_off + b), hi = __ldcg(batch_off + b + 1);
     row0 = lo + tile * kPairRows;
     active = slice_ok(lo, hi, g.tokens(), p.status) && row0 < hi;
     rows_all = active ? min(kPairRows, hi - row0) : 0;
   } else {
     row0 = b * g.seq_act + tile * kPairRows;
     rows_all = min(kPairRows, g.seq_act - tile * kPairRows);
-    if (p.store_mask != nullptr) {
+    if (store_mask != nullptr) {
       const int r = (int)threadIdx.x;
-      const int mine = r < rows_all && __ldcg(p.store_mask + g.cache_row(row0 + r)) == 0;
+      const int mine = r < rows_all && __ldcg(store_mask + g.cache_row(row0 + r)) == 0;
       active = __syncthreads_or(mine) != 0;
     }
   }
@@ -698,8 +707,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int k = 0; k < QU; ++k) {
       const int u = u0 + k * kGather, r = u >> 4;
       tok[k] = -1;
-      if (u < kPairRows * 16 && r < rows_all) tok[k] = p.idx ? __ldcg(p.idx + row0 + r) : row0 + r;
-      if (p.idx && tok[k] >= 0 && !token_ok(tok[k], g.tokens(), p.status)) tok[k] = -1;      // read as a row of zeros
+      if (u < kPairRows * 16 && r < rows_all) tok[k] = idx ? __ldcg(idx + row0 + r) : row0 + r;
+      if (idx && tok[k] >= 0 && !token_ok(tok[k], g.tokens(), p.status)) tok[k] = -1;      // read as a row of zeros
     }
 #pragma unroll
     for (int k = 0; k < QU; ++k) {
@@ -881,9 +890,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       bool ok = r < rows_valid;
       const float inv = 1.f / l;
       const int rr = st * BQ + (ok ? r : 0);
-      int t = p.idx ? __ldcg(p.idx + row0 + rr) : row0 + rr;
-      if (p.idx != nullptr && ok && !token_ok(t, g.tokens(), p.status)) { ok = false; t = 0; }   // no cache row to write
-      if (p.idx == nullptr && p.store_mask != nullptr && ok && __ldcg(p.store_mask + g.cache_row(t)) != 0) ok = false;   // a reused row
+      int t = idx ? __ldcg(idx + row0 + rr) : row0 + rr;
+      if (idx != nullptr && ok && !token_ok(t, g.tokens(), p.status)) { ok = false; t = 0; }   // no cache row to write
+      if (idx == nullptr && store_mask != nullptr && ok && __ldcg(store_mask + g.cache_row(t)) != 0) ok = false;   // a reused row
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
@@ -911,26 +920,41 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+namespace {
+// -> two query tiles per CTA?  else *ksplit = key split of the one-tile kernel
+bool pick_form(const StepGeom& g, bool row_sparse, int* ksplit_out) {
+  const int tps = (g.seq_act + BQ - 1) / BQ;
+  // CTAs expected to have work: every row tile (dense) or one row tile per sequence (row-sparse, small refresh set)
+  const int expected = g.n_heads * g.batch * (row_sparse ? 1 : tps);
+  const int n_blocks = (g.kv_len + BKV - 1) / BKV;
+  // The merge of a key split costs about as much as four key blocks (three cluster-wide barriers and the copies), so
+  // the keys are split only when every CTA still keeps at least four blocks.
+  int ksplit = 1;
+  while (ksplit < 4 && expected * ksplit * 2 <= 160 && ksplit * 2 * 4 <= n_blocks) ksplit *= 2;
+  *ksplit_out = ksplit;
+  // Many query rows per sequence (and enough work to fill the GPU without a key split): two tiles per CTA share
+  // the key blocks.  A row-sparse launch cannot know the size of the refresh set; the window length decides: long
+  // windows are where refresh sets of several tiles are.
+  const int tps2 = (g.seq_act + kPairRows - 1) / kPairRows;
+  return ksplit == 1 && (row_sparse ? g.seq_act >= kPairMinSparse && g.n_heads * g.batch >= 64
+                                    : g.seq_act > kPairMinDense && g.n_heads * g.batch * tps2 >= 148);
+}
+}  // namespace
+
+bool attention_tc_two_tiles(const StepGeom& g, bool row_sparse) {
+  int ksplit;
+  return pick_form(g, row_sparse, &ksplit);
+}
+
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st) {
   static std::atomic<unsigned long long> attr_one{0}, attr_pair{0};
   if (cudaError_t e = ensure_dyn_smem(attn_tc_kernel, AttnSmem::TOTAL, attr_one); e != cudaSuccess) return e;
   if (cudaError_t e = ensure_dyn_smem(attn_pair_kernel, PairSmem::TOTAL, attr_pair); e != cudaSuccess) return e;
   const int tps = (p.g.seq_act + BQ - 1) / BQ;
-  // CTAs expected to have work: every row tile (dense) or one row tile per sequence (row-sparse, small refresh set)
-  const int expected = p.g.n_heads * p.g.batch * (p.idx ? 1 : tps);
-  const int n_blocks = (p.g.kv_len + BKV - 1) / BKV;
-  // The merge of a key split costs about as much as four key blocks (three cluster-wide barriers and the copies), so
-  // the keys are split only when every CTA still keeps at least four blocks.
-  int ksplit = 1;
-  while (ksplit < 4 && expected * ksplit * 2 <= 160 && ksplit * 2 * 4 <= n_blocks) ksplit *= 2;
-  // Many query rows per sequence (and enough work to fill the GPU without a key split): two tiles per CTA share
-  // the key blocks.  A row-sparse launch cannot know the size of the refresh set; the window length decides: long
-  // windows are where refresh sets of several tiles are.
   const int tps2 = (p.g.seq_act + kPairRows - 1) / kPairRows;
-  const bool pair = ksplit == 1 &&
-                    (p.idx ? p.g.seq_act >= kPairMinSparse && p.g.n_heads * p.g.batch >= 64
-                           : p.g.seq_act > kPairMinDense && p.g.n_heads * p.g.batch * tps2 >= 148);
+  int ksplit = 1;
+  const bool pair = pick_form(p.g, p.idx != nullptr, &ksplit);
   if (pair) {
     dim3 grid(p.g.n_heads, p.g.batch * tps2, 1);
     if (grid.y == 0) return cudaSuccess;

@@ -241,9 +241,17 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
     // a long row-sparse step is issued in both forms: over the refresh set's rows, and dense with only the refreshed
     // rows stored (tiles without one skipped); the size of the set decides on the device which of them runs
     const bool both_forms = o_sparse && m_tiles_dense > 8 && use_persist(d / 256, m_tiles_dense, 1);
-    if (both_forms) { p.gate_count = B.count; p.gate_hi = gate_o; }
+    // (one launch carries both when both take the kernel with two query tiles per CTA: its CTAs pick the form; a
+    // launch that only looks at the count and leaves still costs a wave of CTAs per 148 of them)
+    const bool one_launch = both_forms && attention_tc_two_tiles(g, true) && attention_tc_two_tiles(g, false);
+    p.dense_from = 0; p.dense_mask = nullptr;
+    if (both_forms) {
+      p.gate_count = B.count;
+      if (one_launch) { p.dense_from = gate_o; p.dense_mask = B.delta; }
+      else p.gate_hi = gate_o;
+    }
     e = launch_attention_tc(S.kc64, S.vc64, p, st); ++launches;
-    if (both_forms && e == cudaSuccess) {
+    if (both_forms && !one_launch && e == cudaSuccess) {
       AttnParams pd = p;
       pd.idx = nullptr; pd.batch_off = nullptr; pd.debug = nullptr;
       pd.gate_lo = gate_o; pd.gate_hi = 1 << 30; pd.store_mask = B.delta;

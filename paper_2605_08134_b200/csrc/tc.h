@@ -75,7 +75,12 @@ struct AttnParams {
                             // a row are skipped
   int wait_first;           // 1: the queries or the refresh set come from the kernel just before this one in the stream,
                             // so nothing of the step is read ahead of the dependency wait
+  int dense_from;           // > 0 (two-tile kernel, row-sparse parameters above, gate_count set): one launch carries both
+  const int* dense_mask;    // forms; with *gate_count >= dense_from its CTAs run the dense form with this store mask
 };
+
+// does a launch of this geometry take the kernel with two query tiles per CTA?
+bool attention_tc_two_tiles(const StepGeom& g, bool row_sparse);
 
 cudaError_t launch_attention_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_v, const AttnParams& p,
                                 cudaStream_t st);
