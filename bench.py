@@ -741,7 +741,7 @@ def run_sweep(args):
     """Crossover sweep on the long-context layer (batch 4, seq 4096 unless overridden): changed-token fraction
     0..100 % in 5 % steps, uniform and block-clustered patterns, modes kv / o / both against the dense path of the
     same library.  Prints one JSON line with the per-point times and the break-even fraction per mode and pattern
-    (linear interpolation between grid points; null = no crossover below 100 %)."""
+    (running median of three points, then linear interpolation between grid points; null = no crossover below 100 %)."""
     import numpy as np
     import torch
     from paper_2605_08134_b200 import build
@@ -817,6 +817,9 @@ def run_sweep(args):
         for name, ys in curves.items():
             worst = max(worst, max(ys) / dense_us)
             be = None
+            # a running median of three points first: a single point that met another state of the power cap (they
+            # move by +- 3 %, now and then by more) does not decide where the curve crosses the dense path
+            ys = [statistics.median(ys[max(0, i - 1):i + 2]) for i in range(len(ys))]
             for i in range(len(fracs) - 1):
                 a, b_ = ys[i] - dense_us, ys[i + 1] - dense_us
                 if a <= 0 < b_:
