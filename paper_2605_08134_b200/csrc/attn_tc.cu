@@ -479,7 +479,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // ---- merge of the key split (all warps)
     __syncthreads();
     tc_fence_before();
-    cluster_sync_all();                                  // every CTA of the cluster is past its key loop
+    cluster_sync_relaxed();                              // every CTA of the cluster is past its key loop
     tc_fence_after();
     if (warp == 4 && lane < ksplit && lane != z) {
       // hand the rows owned by CTA `lane` to it: the rows, their maxima, their sums
@@ -537,7 +537,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }  // active
   tc_fence_before();
   // nobody leaves while a copy out of its shared memory may still be in flight (its receiver has seen it land)
-  if (ksplit > 1) cluster_sync_all(); else __syncthreads();
+  if (ksplit > 1) cluster_sync_relaxed(); else __syncthreads();
   if (dbg && threadIdx.x == 0) p.debug[4] = globaltimer_ns();
   if (p.debug != nullptr && threadIdx.x == 0) {      // latest end over the CTAs that had work, and their number
     atomicMax(&p.debug[6], globaltimer_ns());

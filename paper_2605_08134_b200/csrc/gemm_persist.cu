@@ -389,7 +389,7 @@ gemm_persist_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   }
   tc_fence_before();
   // (a pair: nobody frees tensor memory or leaves while its partner's MMAs or barrier arrivals may still refer to it)
-  if (PAIR) cluster_sync_all(); else __syncthreads();
+  if (PAIR) cluster_sync_relaxed(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
   if (warp == 1) {
     if (PAIR) tmem_dealloc2(*tmem_slot, 512);

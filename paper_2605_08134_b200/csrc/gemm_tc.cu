@@ -386,7 +386,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   // ---- every CTA of the cluster has finished its main loop: the rings are free to receive partial rows
   tc_fence_before();
-  if (splits > 1) cluster_sync_all(); else __syncthreads();
+  if (splits > 1) cluster_sync_relaxed(); else __syncthreads();
   tc_fence_after();
   if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[32] = globaltimer_ns();
   if (kWarps == 8 || warp >= 2) {
@@ -568,7 +568,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (p.wait_at_end) pdl_wait();
   // nobody leaves while a copy out of its shared memory may still be in flight (the partner has seen it land)
   // (nor frees tensor memory its MMA partner may still read through)
-  if (splits > 1 || PAIR) cluster_sync_all(); else __syncthreads();
+  if (splits > 1 || PAIR) cluster_sync_relaxed(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
   if (warp == 1) {

@@ -307,6 +307,12 @@ __device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster_addr, uint
                ::"r"(dst_cluster_addr), "r"(src_cta_addr), "r"(bytes), "r"(dst_bar_cluster_addr)
                : "memory");
 }
+// Barrier over every thread of the cluster without the release of earlier writes: for points where the threads only
+// tell each other that something they observed complete (an mbarrier phase) is complete.
+__device__ __forceinline__ void cluster_sync_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
 // Barrier over every thread of the cluster; the release/acquire pair orders the distributed shared-memory stores.
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
