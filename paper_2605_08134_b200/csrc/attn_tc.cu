@@ -329,6 +329,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)HD) * 1.4426950408889634f;   // softmax scale folded into the exp2 argument
     float m = -INFINITY, l = 0.f;               // maximum the exponentials are taken against; row sum against it
+    // the token whose cache row this thread writes at the end: asked for now, so that the read is not the first thing
+    // the epilogue waits for
+    const int t_row = r < rows_valid ? (p.idx ? __ldcg(p.idx + row0 + r) : row0 + r) : -1;
 
     for (int j = 0; j < n_st; ++j) {
       mbar_wait(&s_full[st], j & 1, p.status);
@@ -448,7 +451,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (ksplit == 1) {
       // normalise, store
       const float inv = 1.f / l_row;
-      const int t = r < rows_valid ? (p.idx ? __ldcg(p.idx + row0 + r) : row0 + r) : -1;
+      const int t = t_row;
       if (t >= 0 && (p.idx == nullptr ? (p.store_mask == nullptr || __ldcg(p.store_mask + g.cache_row(t)) == 0)
                                       : token_ok(t, g.tokens(), p.status))) {      // (else: no cache row to write)
         __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD + st * 64;
@@ -814,6 +817,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float c = rsqrtf((float)HD) * 1.4426950408889634f;
     float m = -INFINITY, l = 0.f;
+    // (the token whose cache row this thread writes at the end: asked for now, not in the epilogue)
+    const int t_row = idx ? __ldcg(idx + row0 + st * BQ + (r < rows_valid ? r : 0)) : row0 + st * BQ + (r < rows_valid ? r : 0);
     for (int hf = 0; hf < n_half; ++hf) {
       const uint32_t sbuf = tmem_s + (hf & 1) * kHalf + lane_addr;      // scores of half block hf, then its P
       mbar_wait(&s_full[2 * st + (hf & 1)], (hf >> 1) & 1, p.status);
@@ -889,8 +894,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     {
       bool ok = r < rows_valid;
       const float inv = 1.f / l;
-      const int rr = st * BQ + (ok ? r : 0);
-      int t = idx ? __ldcg(idx + row0 + rr) : row0 + rr;
+      int t = t_row;
       if (idx != nullptr && ok && !token_ok(t, g.tokens(), p.status)) { ok = false; t = 0; }   // no cache row to write
       if (idx == nullptr && store_mask != nullptr && ok && __ldcg(store_mask + g.cache_row(t)) != 0) ok = false;   // a reused row
       __nv_bfloat16* dst = p.oc + (size_t)g.cache_row(t) * g.d + h * HD;
