@@ -393,32 +393,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // The partial accumulator: tensor memory -> own shared memory, thread <-> row.  With eight warps the two warps
     // of a lane quarter (w and w + 4) take half of the columns each; with six, warps 2-5 take a quarter each.
     const int r = quarter * 32 + lane;
-    const uint32_t dst = smem_u32(smem + (size_t)r * PROW_BYTES);
+    // Layout of the partial tile in shared memory: [32-column chunk][row][128 bytes], the eight 16-byte units of a
+    // row's chunk XOR-swizzled by the row (thread <-> row stores of one unit would otherwise hit the same banks).
+    // The 32 rows a warp holds of one chunk are 4 KB in one piece: rows owned by the partner leave chunk by chunk,
+    // as soon as the warp has written them, so that the copies overlap the rest of the read-out.
+    const uint32_t dst = smem_u32(smem) + (uint32_t)r * 128u;
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     constexpr int ch_n = kWarps == 8 ? BN / 64 : BN / 32;
     const int ch0 = kWarps == 8 ? (warp >> 2) * ch_n : 0;
+    const int owner = r / rows_per_cta;                              // (uniform over the warp: 32 | rows_per_cta)
+    const bool send = splits > 1 && owner != z;
+    const int rl0 = quarter * 32 - owner * rows_per_cta;
+    const uint32_t rbar = send ? map_to_cta(smem_u32(recv_bar), rank_of_slice(owner)) : 0u;
+    const uint32_t rbase = send ? map_to_cta(smem_u32(smem + RECV_OFFSET), rank_of_slice(owner)) : 0u;
 #pragma unroll 1
     for (int ch = ch0; ch < ch0 + ch_n; ++ch) {
       float v[32];
       tmem_ld_32x32(t_lane + ch * 32, v);
+      const uint32_t cdst = dst + (uint32_t)ch * (uint32_t)(BM * 128);
 #pragma unroll
       for (int g4 = 0; g4 < 8; ++g4)
-        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(((ch * 8 + g4) ^ (r & 7)) << 4)),
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cdst + (uint32_t)((g4 ^ (r & 7)) << 4)),
                      "f"(v[4 * g4]), "f"(v[4 * g4 + 1]), "f"(v[4 * g4 + 2]), "f"(v[4 * g4 + 3]) : "memory");
-    }
-    if (splits > 1) {
-      const int owner = r / rows_per_cta;
-      if (owner != z) {                            // hand the 32 rows to their owner: one 32 KB bulk copy
+      if (send) {
         fence_proxy_async_smem();
-        if (kWarps == 8) asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory");   // both warps of the quarter
-        else __syncwarp();
-        if ((kWarps != 8 || warp < 4) && lane == 0) {
-          const int rl0 = quarter * 32 - owner * rows_per_cta;
-          const uint32_t src = smem_u32(smem + (size_t)(quarter * 32) * PROW_BYTES);
-          const uint32_t rdst = map_to_cta(smem_u32(smem + RECV_OFFSET + (size_t)rl0 * PROW_BYTES), rank_of_slice(owner));
-          const uint32_t rbar = map_to_cta(smem_u32(recv_bar), rank_of_slice(owner));
-          bulk_copy_to_cta(rdst, src, 32 * PROW_BYTES, rbar);
-        }
+        __syncwarp();
+        if (lane == 0)
+          bulk_copy_to_cta(rbase + (uint32_t)ch * (uint32_t)((BM / 2) * 128) + (uint32_t)rl0 * 128u,
+                           smem_u32(smem) + (uint32_t)ch * (uint32_t)(BM * 128) + (uint32_t)(quarter * 32) * 128u, 32 * 128, rbar);
       }
     }
   }
@@ -443,15 +445,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
         for (int hh = 0; hh < BN / HD; ++hh) {
           const int c_lo = hh * HD + 2 * lane, c_hi = c_lo + HD / 2;
-          const uint32_t off_lo = (uint32_t)((((c_lo >> 2) ^ (rl & 7)) << 4) | ((c_lo & 3) << 2));
-          const uint32_t off_hi = (uint32_t)((((c_hi >> 2) ^ (rl & 7)) << 4) | ((c_hi & 3) << 2));
-          const uint8_t* mine = smem + (size_t)(z * rows_per_cta + rl) * PROW_BYTES;      // this CTA's partial
-          float2 lo = *reinterpret_cast<const float2*>(mine + off_lo);
-          float2 hi = *reinterpret_cast<const float2*>(mine + off_hi);
+          // (unit of the column inside its 32-column chunk, swizzled by the row; rows_per_cta is a multiple of 8)
+          const uint32_t in_lo = (uint32_t)(((((c_lo >> 2) & 7) ^ (rl & 7)) << 4) | ((c_lo & 3) << 2));
+          const uint32_t in_hi = (uint32_t)(((((c_hi >> 2) & 7) ^ (rl & 7)) << 4) | ((c_hi & 3) << 2));
+          const uint8_t* mine = smem + (size_t)(z * rows_per_cta + rl) * 128;             // this CTA's partial
+          float2 lo = *reinterpret_cast<const float2*>(mine + (size_t)(c_lo >> 5) * (BM * 128) + in_lo);
+          float2 hi = *reinterpret_cast<const float2*>(mine + (size_t)(c_hi >> 5) * (BM * 128) + in_hi);
           if (splits > 1) {
-            const uint8_t* theirs = smem + RECV_OFFSET + (size_t)rl * PROW_BYTES;         // the partner's partial
-            const float2 a = *reinterpret_cast<const float2*>(theirs + off_lo);
-            const float2 b = *reinterpret_cast<const float2*>(theirs + off_hi);
+            const uint8_t* theirs = smem + RECV_OFFSET + (size_t)rl * 128;                // the partner's partial
+            const float2 a = *reinterpret_cast<const float2*>(theirs + (size_t)(c_lo >> 5) * ((BM / 2) * 128) + in_lo);
+            const float2 b = *reinterpret_cast<const float2*>(theirs + (size_t)(c_hi >> 5) * ((BM / 2) * 128) + in_hi);
             lo.x += a.x; lo.y += a.y; hi.x += b.x; hi.y += b.y;
           }
           vlo[k][hh] = lo; vhi[k][hh] = hi;
