@@ -57,7 +57,7 @@ struct Cfg {
 // Warps of a CTA: producer, MMA issuer, the rest wait for the accumulator; all of them finish rows.
 template <int BN>
 struct Warps {
-  static constexpr int N = BN == 128 ? 6 : 8;   // (eight warps on the 128-wide gathered projection: faster kernel, slower step)
+  static constexpr int N = 8;
   static constexpr int RB = N == 8 ? 4 : 6;          // rows a warp finishes at a time
 };
 template <int RB>
@@ -130,7 +130,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // it to be uniform over the warp
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   // (a pair launch has the row tiles along x: the two CTAs of an MMA pair are neighbours in x)
-  const int nt = PAIR ? blockIdx.y : blockIdx.x, mt = PAIR ? blockIdx.x : blockIdx.y;
+  const int nt = PAIR ? blockIdx.y : blockIdx.x, mt_first = PAIR ? blockIdx.x : blockIdx.y;
   const int splits = gridDim.z;                 // = cluster size along z
   // cluster = (PAIR ? 2 : 1, 1, splits): rank = place in the MMA pair + 2 * reduction slice
   const int crank = (int)cluster_ctarank();
@@ -140,7 +140,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   auto rank_of_slice = [&](int zz) { return (uint32_t)(PAIR ? 2 * zz + pr : zz); };
   const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  const int lin = (z * (int)(PAIR ? gridDim.x : gridDim.y) + mt) * (int)(PAIR ? gridDim.y : gridDim.x) + nt;
+  const int lin = (z * (int)(PAIR ? gridDim.x : gridDim.y) + mt_first) * (int)(PAIR ? gridDim.y : gridDim.x) + nt;
   const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
@@ -153,9 +153,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int kb_begin = (int)(((long long)KB * z) / splits), kb_end = (int)(((long long)KB * (z + 1)) / splits);
   const int nkb = kb_end - kb_begin;
 
+  // A gathered launch of few row tiles (p.loop_rows) has one row of the grid: its CTAs take the row tiles of the
+  // refresh set one after the other, setting their barriers up again for each (the refresh set is small, one tile
+  // as a rule; a grid with a row of CTAs per possible tile would send hundreds of CTAs through the SMs this launch
+  // leaves free only to look at the count and leave, and the next kernel cannot start before the last of them has).
+  for (int iter = 0;; ++iter) {
+  const int mt = mt_first + iter;
   // Row tiles past the first one of a gathered launch are usually empty (the refresh set is small): they look at
   // the count before spending anything on set-up.  The others set up first and wait for the previous kernel later.
-  const bool likely = p.count == nullptr || mt == 0;
+  const bool likely = p.count == nullptr || mt == 0 || iter > 0;
   if (!likely) {
     pdl_wait();
     if (mt * BM >= checked_count(*p.count, p.m_total, p.status)) return;     // uniform over the cluster
@@ -166,6 +172,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const bool gather = p.gather_src != nullptr;
   const uint32_t tx_bytes = gather ? (uint32_t)C::B_BYTES : (uint32_t)STAGE_BYTES;
   if (threadIdx.x == 0) {
+    if (iter > 0) {                              // (every CTA of the cluster is past the previous tile: nothing is in flight)
+      for (int s = 0; s < STAGES; ++s) { mbar_inval(&full_bar[s]); mbar_inval(&empty_bar[s]); }
+      mbar_inval(accum_bar);
+      mbar_inval(recv_bar);
+    }
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], gather ? 5 : 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(accum_bar, 1);
     mbar_init(recv_bar, 1);
@@ -174,7 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     prefetch_tmap(&tm_a);
     prefetch_tmap(tm_b);
   }
-  if (warp == 1) {
+  if (warp == 1 && iter == 0) {
     if (PAIR) { tmem_alloc2(tmem_slot, BN); tmem_relinquish2(); }
     else { tmem_alloc(tmem_slot, BN); tmem_relinquish(); }
   }
@@ -192,7 +203,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
   // The weights do not depend on the previous kernel in the stream: the producer starts their first tiles now, so
   // that they stream in while that kernel drains.  Everything it produced is needed only after pdl_wait().
-  const int n_early = likely ? (nkb < STAGES ? nkb : STAGES) : 0;
+  const int n_early = likely && iter == 0 ? (nkb < STAGES ? nkb : STAGES) : 0;
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
       uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
@@ -574,9 +585,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (splits > 1 || PAIR) cluster_sync_relaxed(); else __syncthreads();
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
+  if (!p.loop_rows || p.count == nullptr) break;
+  if ((mt + 1) * BM >= checked_count(*p.count, p.m_total, p.status)) break;      // uniform over the cluster
+  }  // row tiles
   if (warp == 1) {
     if (PAIR) tmem_dealloc2(*tmem_slot, BN);
-    else tmem_dealloc(tmem_base, BN);
+    else tmem_dealloc(*tmem_slot, BN);
   }
 }
 

@@ -54,6 +54,7 @@ struct GemmParams {
   const int* gate_count;
   int gate_lo, gate_hi;
   const int* store_mask;
+  int loop_rows;         // gathered launch with ONE row of CTAs in the grid: each takes the refresh set's row tiles in turn
   int wait_at_end;       // 1: the launch reads nothing its predecessor in the stream writes and writes nothing that one
                          // reads, so it runs beside it: its CTAs start as soon as the predecessor's have passed their own
                          // dependency wait (everything further back is then complete), and wait for the predecessor
