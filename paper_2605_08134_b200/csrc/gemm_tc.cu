@@ -402,7 +402,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[32] = globaltimer_ns();
   if (kWarps == 8 || warp >= 2) {
     // The partial accumulator: tensor memory -> own shared memory, thread <-> row.  With eight warps the two warps
-    // of a lane quarter (w and w + 4) take half of the columns each; with six, warps 2-5 take a quarter each.
+    // of a lane quarter (w and w + 4) take half of the columns each.
     const int r = quarter * 32 + lane;
     // Layout of the partial tile in shared memory: [32-column chunk][row][128 bytes], the eight 16-byte units of a
     // row's chunk XOR-swizzled by the row (thread <-> row stores of one unit would otherwise hit the same banks).
