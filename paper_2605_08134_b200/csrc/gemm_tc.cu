@@ -131,16 +131,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   // (a pair launch has the row tiles along x: the two CTAs of an MMA pair are neighbours in x)
   const int nt = PAIR ? blockIdx.y : blockIdx.x, mt_first = PAIR ? blockIdx.x : blockIdx.y;
-  const int splits = gridDim.z;                 // = cluster size along z
+  const int cl_splits = gridDim.z;              // = cluster size along z: slices of the reduction
   // cluster = (PAIR ? 2 : 1, 1, splits): rank = place in the MMA pair + 2 * reduction slice
   const int crank = (int)cluster_ctarank();
   const int pr = PAIR ? (crank & 1) : 0;        // place in the MMA pair; place 0 issues the MMAs
-  const int z = PAIR ? (crank >> 1) : crank;    // reduction slice
+  const int cl_z = PAIR ? (crank >> 1) : crank; // this CTA's slice
   const uint32_t lead = (uint32_t)(crank & ~1); // cluster rank of the pair's issuing CTA
   auto rank_of_slice = [&](int zz) { return (uint32_t)(PAIR ? 2 * zz + pr : zz); };
-  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && z == 0;
+  const bool dbg = p.debug != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && cl_z == 0;
   if (dbg && threadIdx.x == 0) p.debug[0] = globaltimer_ns();
-  const int lin = (z * (int)(PAIR ? gridDim.x : gridDim.y) + mt_first) * (int)(PAIR ? gridDim.y : gridDim.x) + nt;
+  const int lin = (cl_z * (int)(PAIR ? gridDim.x : gridDim.y) + mt_first) * (int)(PAIR ? gridDim.y : gridDim.x) + nt;
   const bool rec = EPI == EPI_Q && p.debug != nullptr && lin < 1024;
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin] = globaltimer_ns();
 
@@ -149,16 +149,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int n0 = p.b_pair ? nt * (BN / 2) : (is_b1 ? nt - p.n_split : nt) * BN;   // first output column / W row
   const CUtensorMap* tm_b = is_b1 ? &tm_b1 : &tm_b0;
   // ---- which slice of the reduction?
+  // (a CTA walks the k-blocks from the start of its slice on, modulo KB: its slice when the tile's reduction is
+  // split, all of them when it is not)
   const int KB = p.K / BK;
-  const int kb_begin = (int)(((long long)KB * z) / splits), kb_end = (int)(((long long)KB * (z + 1)) / splits);
-  const int nkb = kb_end - kb_begin;
+  const int kb0 = (int)(((long long)KB * cl_z) / cl_splits);
+  auto kb_of = [&](int i) { const int k = kb0 + i; return k >= KB ? k - KB : k; };
+  int tiles_done = 0;                           // (p.loop_rows) row tiles of the refresh set behind this cluster
 
   // A gathered launch of few row tiles (p.loop_rows) has one row of the grid: its CTAs take the row tiles of the
   // refresh set one after the other, setting their barriers up again for each (the refresh set is small, one tile
   // as a rule; a grid with a row of CTAs per possible tile would send hundreds of CTAs through the SMs this launch
   // leaves free only to look at the count and leave, and the next kernel cannot start before the last of them has).
   for (int iter = 0;; ++iter) {
-  const int mt = mt_first + iter;
+  int mt = mt_first + iter;
+  int splits = cl_splits, z = cl_z, tile_step = 1;   // (settled below, once the size of the refresh set is known)
   // Row tiles past the first one of a gathered launch are usually empty (the refresh set is small): they look at
   // the count before spending anything on set-up.  The others set up first and wait for the previous kernel later.
   const bool likely = p.count == nullptr || mt == 0 || iter > 0;
@@ -181,7 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     mbar_init(accum_bar, 1);
     mbar_init(recv_bar, 1);
     fence_mbar_init();
-    if (splits > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)(BM / 2) * PROW_BYTES);   // the partner's 64 rows
+    if (cl_splits > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)(BM / 2) * PROW_BYTES);   // the partner's 64 rows (if split)
     prefetch_tmap(&tm_a);
     prefetch_tmap(tm_b);
   }
@@ -203,7 +207,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
   // The weights do not depend on the previous kernel in the stream: the producer starts their first tiles now, so
   // that they stream in while that kernel drains.  Everything it produced is needed only after pdl_wait().
-  const int n_early = likely && iter == 0 ? (nkb < STAGES ? nkb : STAGES) : 0;
+  const int n_early = likely && iter == 0 ? (KB / cl_splits < STAGES ? KB / cl_splits : STAGES) : 0;
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
       uint8_t* b_dst = smem + i * STAGE_BYTES + A_BYTES;
@@ -211,16 +215,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // the bytes of both CTAs are counted on the issuing CTA's barrier; each CTA brings its half of the W rows
         // (a tile of two matrices: the even CTA brings the rows of the first, the odd one those of the second)
         if (pr == 0) mbar_arrive_expect_tx(&full_bar[i], 2 * STAGE_BYTES);
-        tma_load_2d_pair(b_dst, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, (kb_begin + i) * BK,
+        tma_load_2d_pair(b_dst, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, kb_of(i) * BK,
                          p.b_pair ? n0 : n0 + pr * (BN / 2), map_to_cta(smem_u32(&full_bar[i]), lead));
         continue;
       }
       mbar_arrive_expect_tx(&full_bar[i], tx_bytes);
       if (p.b_pair) {
-        tma_load_2d(b_dst, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[i]);
-        tma_load_2d(b_dst + C::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[i]);
+        tma_load_2d(b_dst, &tm_b0, kb_of(i) * BK, n0, &full_bar[i]);
+        tma_load_2d(b_dst + C::B_BYTES / 2, &tm_b1, kb_of(i) * BK, n0, &full_bar[i]);
       } else {
-        tma_load_2d(b_dst, tm_b, (kb_begin + i) * BK, n0, &full_bar[i]);
+        tma_load_2d(b_dst, tm_b, kb_of(i) * BK, n0, &full_bar[i]);
       }
     }
   }
@@ -235,6 +239,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   bool active = true;
   if (p.count != nullptr) {
     const int n = checked_count(*p.count, p.m_total, p.status);
+    if (p.loop_rows) {
+      // The cluster's two CTAs share one row tile (half of the reduction each, partial tiles exchanged) while there is
+      // only one left; with two or more left each takes a row tile of its own over the whole reduction: one pass
+      // over the weights for two tiles instead of two, and nothing to exchange.
+      const int tiles_left = (n + BM - 1) / BM - tiles_done;
+      if (!PAIR && cl_splits == 2 && tiles_left >= 2) { mt = tiles_done + cl_z; splits = 1; z = 0; tile_step = 2; }
+      else mt = tiles_done;
+    }
     t0 = mt * BM;
     active = t0 < n;
     rows_valid = min(BM, n - t0);
@@ -254,6 +266,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   // epilogue geometry
   const int rows_per_cta = BM / splits;           // rows of the tile this CTA finishes
+  const int nkb = KB / splits;                    // k-blocks this CTA walks for the tile
   const int quarter = warp & 3;                   // TMEM lanes a warp may touch: 32*quarter .. +31
   const bool rotate = (EPI == EPI_Q) || (EPI == EPI_KV && !is_b1);
   const int head0 = n0 / HD;
@@ -267,9 +280,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (!gather && elect_one()) {
       for (int i = 0; i < n_early; ++i) {        // the W halves of these stages are already on their way
         if (PAIR)
-          tma_load_2d_pair(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, map_to_cta(smem_u32(&full_bar[i]), lead));
+          tma_load_2d_pair(smem + i * STAGE_BYTES, &tm_a, kb_of(i) * BK, a_row, map_to_cta(smem_u32(&full_bar[i]), lead));
         else
-          tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[i]);
+          tma_load_2d(smem + i * STAGE_BYTES, &tm_a, kb_of(i) * BK, a_row, &full_bar[i]);
       }
     }
     __syncwarp();
@@ -281,17 +294,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (PAIR) {
           const uint32_t fb = map_to_cta(smem_u32(&full_bar[s]), lead);
           if (pr == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * STAGE_BYTES);
-          tma_load_2d_pair(a_dst, &tm_a, (kb_begin + i) * BK, a_row, fb);
-          tma_load_2d_pair(a_dst + A_BYTES, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, (kb_begin + i) * BK,
+          tma_load_2d_pair(a_dst, &tm_a, kb_of(i) * BK, a_row, fb);
+          tma_load_2d_pair(a_dst + A_BYTES, p.b_pair ? (pr == 0 ? &tm_b0 : &tm_b1) : tm_b, kb_of(i) * BK,
                            p.b_pair ? n0 : n0 + pr * (BN / 2), fb);
         } else {
           mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
-          if (!gather) tma_load_2d(a_dst, &tm_a, (kb_begin + i) * BK, a_row, &full_bar[s]);
+          if (!gather) tma_load_2d(a_dst, &tm_a, kb_of(i) * BK, a_row, &full_bar[s]);
           if (p.b_pair) {
-            tma_load_2d(a_dst + A_BYTES, &tm_b0, (kb_begin + i) * BK, n0, &full_bar[s]);
-            tma_load_2d(a_dst + A_BYTES + C::B_BYTES / 2, &tm_b1, (kb_begin + i) * BK, n0, &full_bar[s]);
+            tma_load_2d(a_dst + A_BYTES, &tm_b0, kb_of(i) * BK, n0, &full_bar[s]);
+            tma_load_2d(a_dst + A_BYTES + C::B_BYTES / 2, &tm_b1, kb_of(i) * BK, n0, &full_bar[s]);
           } else {
-            tma_load_2d(a_dst + A_BYTES, tm_b, (kb_begin + i) * BK, n0, &full_bar[s]);
+            tma_load_2d(a_dst + A_BYTES, tm_b, kb_of(i) * BK, n0, &full_bar[s]);
           }
         }
       }
@@ -363,7 +376,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int tok = __shfl_sync(0xffffffffu, tok_own, rw);
         const int srow = tok < 0 ? 0 : (p.gather_cache_rows ? p.g.cache_row(tok) : tok);
         src_k[k] = reinterpret_cast<const uint8_t*>(p.gather_src) + (size_t)srow * p.K * 2 +
-                   (size_t)kb_begin * (BK * 2) + u * 16;
+                   u * 16;
         bytes_k[k] = tok >= 0 ? 16u : 0u;                       // rows past the refresh set are zero-filled
         dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
       }
@@ -374,7 +387,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)i * (BK * 2), bytes_k[k]);
+            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)kb_of(i) * (BK * 2), bytes_k[k]);
         }
         cp_async_commit();                                      // (empty groups at the tail keep the lag uniform)
         if (i >= LAG) {
@@ -566,7 +579,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   } else if (warp == 0 && lane == 0) {
     // a tile past the refresh set: complete the stages whose W halves were started early, then let them land
     if (!gather) {
-      for (int i = 0; i < n_early; ++i) tma_load_2d(smem + i * STAGE_BYTES, &tm_a, (kb_begin + i) * BK, 0, &full_bar[i]);
+      for (int i = 0; i < n_early; ++i) tma_load_2d(smem + i * STAGE_BYTES, &tm_a, kb_of(i) * BK, 0, &full_bar[i]);
       for (int i = 0; i < n_early; ++i) mbar_wait(&full_bar[i], 0, p.status);
     } else {
       // the barrier also counts the four gathering warps, which do not run here: stand in for them
@@ -586,7 +599,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (p.debug != nullptr && threadIdx.x == 0) { atomicMax(&p.debug[6], globaltimer_ns()); atomicAdd(&p.debug[7], 1ull); }
   if (rec && threadIdx.x == 0) p.debug[64 + 3 * lin + 2] = globaltimer_ns();
   if (!p.loop_rows || p.count == nullptr) break;
-  if ((mt + 1) * BM >= checked_count(*p.count, p.m_total, p.status)) break;      // uniform over the cluster
+  tiles_done += tile_step;
+  if (tiles_done * BM >= checked_count(*p.count, p.m_total, p.status)) break;    // uniform over the cluster
   }  // row tiles
   if (warp == 1) {
     if (PAIR) tmem_dealloc2(*tmem_slot, BN);
