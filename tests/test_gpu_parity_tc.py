@@ -76,9 +76,10 @@ def config2():
     return shape, w, hs, x0, o, y0
 
 
-@pytest.mark.parametrize("n_changed", [26, 67, 154, 256, 512])
+@pytest.mark.parametrize("n_changed", [26, 67, 154, 256, 330, 512])
 def test_config2_llada_layer_full_size(dare, config2, n_changed):
-    """Config 2: d=4096, 32 heads x 128, seq 512, bf16; changed fraction 5/13/30/50/100 %, all three reuse modes."""
+    """Config 2: d=4096, 32 heads x 128, seq 512, bf16; changed fraction 5/13/30/50/100 %, all three reuse modes
+    (and 330 rows: three row tiles, of which the gathered projection's clusters take two in one pass and share the third)."""
     shape, w, hs0, x0, o0, y0 = config2
     hs = copy.deepcopy(hs0)
     ch = wl.uniform_positions(hs.rng, shape, n_changed)
