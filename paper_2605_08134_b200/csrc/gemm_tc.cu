@@ -381,13 +381,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         dst_k[k] = smem_u32(smem) + (uint32_t)r * 128u + (uint32_t)((u ^ (r & 7)) << 4);
       }
       constexpr int LAG = STAGES - 2;                           // copy groups in flight per thread
+      uint32_t koff = (uint32_t)kb0 * (BK * 2);                 // byte offset of k-block kb_of(i) in a row
+      const uint32_t kwrap = (uint32_t)KB * (BK * 2);
       for (int i = 0; i < nkb + LAG; ++i) {
         if (i < nkb) {
           const int s = i % STAGES;
           mbar_wait(&empty_bar[s], ((i / STAGES) & 1) ^ 1, p.status);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + (size_t)kb_of(i) * (BK * 2), bytes_k[k]);
+            cp_async_16(dst_k[k] + (uint32_t)s * STAGE_BYTES, src_k[k] + koff, bytes_k[k]);
+          koff += BK * 2;
+          if (koff == kwrap) koff = 0;
         }
         cp_async_commit();                                      // (empty groups at the tail keep the lag uniform)
         if (i >= LAG) {
