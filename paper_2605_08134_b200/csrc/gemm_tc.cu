@@ -130,7 +130,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // it to be uniform over the warp
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   // (a pair launch has the row tiles along x: the two CTAs of an MMA pair are neighbours in x)
-  const int nt = PAIR ? blockIdx.y : blockIdx.x, mt_first = PAIR ? blockIdx.x : blockIdx.y;
+  const int nt = (PAIR ? blockIdx.y : blockIdx.x) + p.nt0, mt_first = PAIR ? blockIdx.x : blockIdx.y;
   const int cl_splits = gridDim.z;              // = cluster size along z: slices of the reduction
   // cluster = (PAIR ? 2 : 1, 1, splits): rank = place in the MMA pair + 2 * reduction slice
   const int crank = (int)cluster_ctarank();

@@ -222,6 +222,7 @@ struct dare_stack {
   const void* emb;
   const float* final_gain;
   StackBuffers buf;
+  int sm_count;               // SMs of the device the stack was created on
   int capture_layer;          // test hook: copy this layer's input and output of every pass (-1 = off)
   void* capture_x;
   void* capture_h;
@@ -273,8 +274,25 @@ dare_status_t forward(dare_stack* S, const int* tokens, int batch, int seq_total
       p.b_pair = 1; p.out0 = B.act; p.ld_out = f;
       const int n_tiles = f / 128;
       const int sp = pick_splits(n_tiles * m_tiles, d / 64);
-      if (launch_gemm_tc(EPI_SWIGLU, 256, S->a_n2, S->maps[l].w_gate, S->maps[l].w_up, p, n_tiles, m_tiles, sp, st,
-                         pairs_pay(n_tiles, m_tiles, sp) ? 1 : 0) != cudaSuccess) return DARE_ERR_CUDA;
+      const bool pairs = pairs_pay(n_tiles, m_tiles, sp);
+      // Pair tiles over the whole reduction fill the SM pairs in waves; a last wave that is less than half full (96
+      // tiles on 74 pairs) is issued as a launch of its own with the reduction split in two, which puts twice as many
+      // SM pairs on it for half as long.  It needs nothing from the launch before it and runs behind it as SMs come
+      // free (it waits for its predecessors only before it leaves).
+      const int wave = S->sm_count / 2;
+      const int rest = pairs && sp == 1 && m_tiles == 2 && wave > 0 ? n_tiles % wave : 0;
+      if (rest > 0 && n_tiles > wave && 2 * rest <= wave) {
+        const int full = n_tiles - rest;
+        if (launch_gemm_tc(EPI_SWIGLU, 256, S->a_n2, S->maps[l].w_gate, S->maps[l].w_up, p, full, m_tiles, 1, st, 1) != cudaSuccess)
+          return DARE_ERR_CUDA;
+        GemmParams q = p;
+        q.nt0 = full; q.wait_at_end = 1;
+        if (launch_gemm_tc(EPI_SWIGLU, 256, S->a_n2, S->maps[l].w_gate, S->maps[l].w_up, q, rest, m_tiles, 2, st, 1) != cudaSuccess)
+          return DARE_ERR_CUDA;
+      } else if (launch_gemm_tc(EPI_SWIGLU, 256, S->a_n2, S->maps[l].w_gate, S->maps[l].w_up, p, n_tiles, m_tiles, sp, st,
+                                pairs ? 1 : 0) != cudaSuccess) {
+        return DARE_ERR_CUDA;
+      }
     }
     // x_next = h + W_D act
     {
@@ -328,6 +346,13 @@ dare_status_t dare_stack_create(const dare_stack_config_t* cfg, const dare_stack
   if (!S) return DARE_ERR_INVALID_ARG;
   S->magic = kStackMagic;
   S->cfg = *cfg;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+      S->sm_count = sms;
+    else
+      S->sm_count = 0;
+  }
   S->cfg.layer.kernel_path = DARE_PATH_TENSOR;
   S->emb = w->emb;
   S->final_gain = w->final_gain;

@@ -115,7 +115,7 @@ dare_status_t step_tc(dare_layer* L, const void* x, const StepGeom& g, int mode,
   base.out_is_cache = 0; base.resid = nullptr; base.ld_resid = 0; base.out_f32 = nullptr; base.b_pair = 0;
   base.rope = reinterpret_cast<const float2*>(B.rope_cs); base.q_prev = B.q_prev;
   base.scores = B.scores; base.has_prev = has_prev ? 1 : 0; base.status = B.status;
-  base.debug = nullptr; base.wait_at_end = 0; base.loop_rows = 0;
+  base.debug = nullptr; base.wait_at_end = 0; base.loop_rows = 0; base.nt0 = 0;
   base.gate_count = nullptr; base.gate_lo = 0; base.gate_hi = 1 << 30; base.store_mask = nullptr;
   // Steps of many row tiles: from these refresh-set sizes on the dense forms of the K/V projection, of attention and of
   // the output projection (results kept for the refreshed rows only) are faster than the listed forms.  Measured on

@@ -54,6 +54,7 @@ struct GemmParams {
   const int* gate_count;
   int gate_lo, gate_hi;
   const int* store_mask;
+  int nt0;               // first column tile of this launch (a projection issued as two launches over its column tiles)
   int loop_rows;         // gathered launch with ONE row of CTAs in the grid: each takes the refresh set's row tiles in turn
   int wait_at_end;       // 1: the launch reads nothing its predecessor in the stream writes and writes nothing that one
                          // reads, so it runs beside it: its CTAs start as soon as the predecessor's have passed their own
