@@ -434,10 +434,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int rl0 = quarter * 32 - owner * rows_per_cta;
     const uint32_t rbar = send ? map_to_cta(smem_u32(recv_bar), rank_of_slice(owner)) : 0u;
     const uint32_t rbase = send ? map_to_cta(smem_u32(smem + RECV_OFFSET), rank_of_slice(owner)) : 0u;
-#pragma unroll 1
-    for (int ch = ch0; ch < ch0 + ch_n; ++ch) {
-      float v[32];
-      tmem_ld_32x32(t_lane + ch * 32, v);
+    // (the next chunk's tensor-memory load is in flight while this chunk is written and sent)
+    float va[32], vb[32];
+    tmem_ld_32x32_nowait(t_lane + ch0 * 32, va);
+#pragma unroll
+    for (int c2 = 0; c2 < ch_n; ++c2) {
+      const int ch = ch0 + c2;
+      float* v = (c2 & 1) ? vb : va;
+      tmem_ld_wait();
+      if (c2 + 1 < ch_n) tmem_ld_32x32_nowait(t_lane + (ch + 1) * 32, (c2 & 1) ? va : vb);
       const uint32_t cdst = dst + (uint32_t)ch * (uint32_t)(BM * 128);
 #pragma unroll
       for (int g4 = 0; g4 < 8; ++g4)
