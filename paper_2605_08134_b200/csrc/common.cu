@@ -100,7 +100,14 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* __restrict__ x, c
     }
   }
   // x may be the output of the previous kernel in the stream (the previous layer of a model), so it is read only
-  // after that kernel has completed.
+  // after that kernel has completed.  Its lines are asked into the L2 before that, though (the L2 is where a later
+  // write of the producer lands too, so nothing stale can come of it): an input that lies in HBM is then on its way
+  // while this CTA waits.
+  if (kEarlyGain) {
+    const char* xb = reinterpret_cast<const char*>(x + (size_t)blockIdx.x * d);
+    const int row_bytes = d * (int)sizeof(T);
+    for (int off = (int)threadIdx.x * 128; off < row_bytes; off += (int)blockDim.x * 128) ptx::prefetch_l2(xb + off);
+  }
   ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   if (dbg && threadIdx.x == 0) {
