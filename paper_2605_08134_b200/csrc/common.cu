@@ -431,10 +431,12 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float* __restr
                                                       int wait_at_end, const float* __restrict__ tau_dev) {
   __shared__ int warp_excl[32];
   __shared__ int chunk_total;
+  const int T = g.tokens();
+  // (the staleness counters are this kernel's own: their lines are asked into the L2 while it waits for the scores)
+  for (int t = threadIdx.x * 32; t < T; t += 1024 * 32) ptx::prefetch_l2(delta + g.cache_row(t));
   if (!wait_at_end) ptx::pdl_wait();
   ptx::pdl_launch_dependents();
   if (tau_dev != nullptr) tau = *tau_dev;
-  const int T = g.tokens();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int base = 0;
   for (int start = 0; start < T; start += 1024) {
