@@ -333,10 +333,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // the epilogue waits for
     const int t_row = r < rows_valid ? (p.idx ? __ldcg(p.idx + row0 + r) : row0 + r) : -1;
 
+    // a warp none of whose 32 rows exists (a partly filled row-sparse tile) only passes the blocks on: its rows of P
+    // and O are whatever the score buffer held, belong to no token and are never stored
+    const bool warp_has_rows = quarter * 32 < rows_valid;
     for (int j = 0; j < n_st; ++j) {
       mbar_wait(&s_full[st], j & 1, p.status);
       tc_fence_after();
       if (dbg && j == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
+      if (!warp_has_rows && ksplit == 1) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[st]);
+        continue;
+      }
       const int key0 = (z + (2 * j + st) * ksplit) * BKV;
       const int n_keys = min(BKV, g.kv_len - key0);   // the last block may be ragged: keys past kv_len do not exist
       // O and the row sum move to a new maximum only when it grew by more than kRescaleStep (in log2 units); the
