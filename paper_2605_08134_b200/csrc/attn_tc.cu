@@ -828,10 +828,17 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     float m = -INFINITY, l = 0.f;
     // (the token whose cache row this thread writes at the end: asked for now, not in the epilogue)
     const int t_row = idx ? __ldcg(idx + row0 + st * BQ + (r < rows_valid ? r : 0)) : row0 + st * BQ + (r < rows_valid ? r : 0);
+    const bool warp_has_rows = quarter * 32 < rows_valid;   // (else: pass the half blocks on; rows of no token, never stored)
     for (int hf = 0; hf < n_half; ++hf) {
       const uint32_t sbuf = tmem_s + (hf & 1) * kHalf + lane_addr;      // scores of half block hf, then its P
       mbar_wait(&s_full[2 * st + (hf & 1)], (hf >> 1) & 1, p.status);
       tc_fence_after();
+      if (!warp_has_rows) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[2 * st + (hf & 1)]);
+        continue;
+      }
 
       if (dbg && hf == 0 && threadIdx.x == 128) p.debug[2] = globaltimer_ns();
       const int n_keys = min(kHalf, g.kv_len - hf * kHalf);
