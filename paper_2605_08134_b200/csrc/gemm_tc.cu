@@ -58,7 +58,7 @@ struct Cfg {
 template <int BN>
 struct Warps {
   static constexpr int N = 8;
-  static constexpr int RB = N == 8 ? 4 : 6;          // rows a warp finishes at a time
+  static constexpr int RB = 4;                       // rows a warp finishes at a time
 };
 template <int RB>
 struct RowBatch {
@@ -417,7 +417,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (splits > 1) cluster_sync_relaxed(); else __syncthreads();
   tc_fence_after();
   if (dbg && EPI == EPI_Q && threadIdx.x == 64) p.debug[32] = globaltimer_ns();
-  if (kWarps == 8 || warp >= 2) {
+  {
     // The partial accumulator: tensor memory -> own shared memory, thread <-> row.  With eight warps the two warps
     // of a lane quarter (w and w + 4) take half of the columns each.
     const int r = quarter * 32 + lane;
@@ -427,8 +427,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // as soon as the warp has written them, so that the copies overlap the rest of the read-out.
     const uint32_t dst = smem_u32(smem) + (uint32_t)r * 128u;
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    constexpr int ch_n = kWarps == 8 ? BN / 64 : BN / 32;
-    const int ch0 = kWarps == 8 ? (warp >> 2) * ch_n : 0;
+    static_assert(kWarps == 8, "two warps per lane quarter share the columns");
+    constexpr int ch_n = BN / 64;
+    const int ch0 = (warp >> 2) * ch_n;
     const int owner = r / rows_per_cta;                              // (uniform over the warp: 32 | rows_per_cta)
     const bool send = splits > 1 && owner != z;
     const int rl0 = quarter * 32 - owner * rows_per_cta;
